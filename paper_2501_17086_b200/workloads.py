@@ -1,0 +1,129 @@
+"""Seeded synthetic workloads (inputs only; none of the method's arithmetic).
+
+The paper trains on CIFAR10, ImageNet32, Wikitext103 and MNLI (Section 5,
+Table 2).  None of those is used here: every tensor below is drawn from a
+seeded counter-based generator and only the *shapes and structure* of the
+paper's models are kept (residual MLP stacks, a pre-LN decoder Transformer
+whose layers are split into attention and feed-forward residual steps, a
+gated recurrent network with a loss at every time step).
+
+Fill order (fixed, so a seed reproduces a workload on a given device type):
+one ``torch.Generator`` per workload, seeded with ``cfg.seed``; tensors are
+drawn in float32 in the order listed in ``make_inputs`` and then rounded once
+to the workload's dtype.  Draws made on "cuda" and on "cpu" differ; both sides
+of a comparison are always fed the same realised tensors.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+
+import torch
+
+
+@dataclasses.dataclass(frozen=True)
+class Workload:
+    name: str
+    block: str            # "mlp" | "preln_mlp" | "rnn_tanh" | "preln_transformer"
+    dtype: str            # "f32" | "bf16"
+    L: int                # residual steps (mlp), time steps (rnn), decoder blocks (transformer)
+    d: int
+    hidden: int = 0
+    in_dim: int = 0
+    n_heads: int = 0
+    head_dim: int = 0
+    seq: int = 0
+    batch: int = 0
+    tokens: int = 0       # rows of a state: batch*seq for token models, batch for the rnn
+    seed: int = 0
+    loss: str = "final_mse"   # "final_half_sse" | "final_mse" | "every_mse"
+    ln_eps: float = 1e-5
+
+    @property
+    def steps(self) -> int:
+        """Residual steps seen by the scan: two per decoder block."""
+        return 2 * self.L if self.block == "preln_transformer" else self.L
+
+    @property
+    def torch_dtype(self):
+        return torch.float32 if self.dtype == "f32" else torch.bfloat16
+
+
+WORKLOADS = {
+    # the five evaluation shapes
+    "c1": Workload("c1", "mlp", "f32", L=8, d=64, hidden=256, tokens=32, seed=1001, loss="final_half_sse"),
+    "c2": Workload("c2", "preln_mlp", "bf16", L=64, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1002),
+    "c3": Workload("c3", "rnn_tanh", "f32", L=4096, d=512, in_dim=256, batch=32, tokens=32, seed=1003, loss="every_mse"),
+    "c4": Workload("c4", "preln_transformer", "bf16", L=24, d=768, hidden=3072, n_heads=12, head_dim=64,
+                   seq=1024, batch=16, tokens=16384, seed=1004),
+    "c5": Workload("c5", "preln_mlp", "bf16", L=128, d=2048, hidden=8192, batch=32, seq=512, tokens=16384, seed=1005),
+    # reduced twins: same structure, sizes the fp64 oracle runs in full; they
+    # span several tiles and leave ragged tails against 128/256-wide tiles.
+    "c2_twin": Workload("c2_twin", "preln_mlp", "bf16", L=5, d=256, hidden=1024, batch=1, seq=328, tokens=328, seed=2002),
+    "c2_twin_f32": Workload("c2_twin_f32", "preln_mlp", "f32", L=5, d=96, hidden=200, batch=1, seq=77, tokens=77, seed=2012),
+    "c3_twin": Workload("c3_twin", "rnn_tanh", "f32", L=200, d=128, in_dim=48, batch=6, tokens=6, seed=2003, loss="every_mse"),
+    "c4_twin": Workload("c4_twin", "preln_transformer", "bf16", L=2, d=128, hidden=512, n_heads=2, head_dim=64,
+                        seq=200, batch=2, tokens=400, seed=2004),
+    "c4_twin_f32": Workload("c4_twin_f32", "preln_transformer", "f32", L=2, d=64, hidden=128, n_heads=2, head_dim=32,
+                            seq=50, batch=2, tokens=100, seed=2014),
+    "c5_twin": Workload("c5_twin", "preln_mlp", "bf16", L=9, d=512, hidden=1536, batch=1, seq=200, tokens=200, seed=2005),
+}
+
+
+def _randn(gen, shape, std, device):
+    return torch.randn(shape, generator=gen, device=device, dtype=torch.float32) * std
+
+
+def make_inputs(cfg: Workload, device="cpu"):
+    """Returns a dict of tensors in ``cfg.dtype`` on ``device``.
+
+    Keys: mlp / preln_mlp: W1 [L,h,d], W2 [L,d,h], x0 [N,d], y [N,d].
+    rnn_tanh: a [d], W [d,d], U [d,in], X [T,B,in], Y [T,B,d], x0 [B,d] (zeros).
+    preln_transformer: Wq, Wk, Wv, Wo [L,d,d], W1 [L,h,d], W2 [L,d,h], x0 [N,d], y [N,d].
+    Standard deviations: 0.02 for Transformer-style inputs weights and
+    0.02 / sqrt(2 * steps) for the weights that write into the residual stream;
+    variance 1/fan_in for the plain MLP; variance 1/in_dim for U; W is 0.5 times
+    an orthogonal matrix (QR of a Gaussian, signs fixed by the diagonal of R)."""
+    dev = torch.device(device)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(cfg.seed)
+    dt = cfg.torch_dtype
+    out = {}
+    if cfg.block in ("mlp", "preln_mlp"):
+        L, d, h, N = cfg.L, cfg.d, cfg.hidden, cfg.tokens
+        if cfg.block == "mlp":
+            s1, s2 = 1.0 / math.sqrt(d), 1.0 / math.sqrt(h)
+        else:
+            s1, s2 = 0.02, 0.02 / math.sqrt(2.0 * cfg.steps)
+        out["W1"] = torch.empty((L, h, d), device=dev, dtype=dt)
+        out["W2"] = torch.empty((L, d, h), device=dev, dtype=dt)
+        for l in range(L):  # per layer: keeps the float32 staging buffer small
+            out["W1"][l] = _randn(gen, (h, d), s1, dev).to(dt)
+            out["W2"][l] = _randn(gen, (d, h), s2, dev).to(dt)
+        out["x0"] = _randn(gen, (N, d), 1.0, dev).to(dt)
+        out["y"] = _randn(gen, (N, d), 1.0, dev).to(dt)
+    elif cfg.block == "rnn_tanh":
+        T, d, B, nin = cfg.L, cfg.d, cfg.batch, cfg.in_dim
+        out["a"] = (0.9 + 0.099 * torch.rand((d,), generator=gen, device=dev, dtype=torch.float32)).to(dt)
+        gauss = _randn(gen, (d, d), 1.0, dev).double().cpu()
+        q, r = torch.linalg.qr(gauss)
+        q = q * torch.sign(torch.diagonal(r)).unsqueeze(0)
+        out["W"] = (0.5 * q).to(dev).to(dt)
+        out["U"] = _randn(gen, (d, nin), 1.0 / math.sqrt(nin), dev).to(dt)
+        out["X"] = _randn(gen, (T, B, nin), 1.0, dev).to(dt)
+        out["Y"] = _randn(gen, (T, B, d), 1.0, dev).to(dt)
+        out["x0"] = torch.zeros((B, d), device=dev, dtype=dt)
+    elif cfg.block == "preln_transformer":
+        L, d, h, N = cfg.L, cfg.d, cfg.hidden, cfg.tokens
+        s_in, s_out = 0.02, 0.02 / math.sqrt(2.0 * cfg.steps)
+        for name, shape, std in (("Wq", (d, d), s_in), ("Wk", (d, d), s_in), ("Wv", (d, d), s_in),
+                                 ("Wo", (d, d), s_out), ("W1", (h, d), s_in), ("W2", (d, h), s_out)):
+            out[name] = torch.empty((L,) + shape, device=dev, dtype=dt)
+        for l in range(L):
+            for name, std in (("Wq", s_in), ("Wk", s_in), ("Wv", s_in), ("Wo", s_out), ("W1", s_in), ("W2", s_out)):
+                out[name][l] = _randn(gen, tuple(out[name].shape[1:]), std, dev).to(dt)
+        out["x0"] = _randn(gen, (N, d), 1.0, dev).to(dt)
+        out["y"] = _randn(gen, (N, d), 1.0, dev).to(dt)
+    else:
+        raise ValueError(f"unknown block kind {cfg.block!r}")
+    return out
