@@ -1,0 +1,159 @@
+/* hbp.h - C ABI of the Highway-backpropagation hot path (arXiv 2501.17086) on one GPU.
+ *
+ * Model (Section 3, Eq. 1-2): a stack of L residual steps
+ *     x_{l+1} = a_l (.) x_l + f_l(x_l),      l = 0..L-1,
+ * where f_l is the expensive block (Jacobian J, only ever multiplied by a
+ * vector) and diag(a_l) is the cheap residual Jacobian K.  The loss is a sum of
+ * per-state losses (Section 3); delta_l = dLoss_l/dx_l is an INPUT of the
+ * backward calls, so any loss can be used.
+ *
+ * Highway-BP (Theorem 2, Section 4.3): g^0 = CumSumProd(delta, K) (Eq. 10); each
+ * iteration computes u_l = J_l^T g_{l+1} for every l from the previous iterate
+ * (Eq. 8) and then g_l = delta_l + a_l (.) g_{l+1} + u_l for l = L-1..0 (Eq. 9
+ * and 11 folded into one recurrence, which is the same thing by linearity).
+ * After k iterations g_l is the sum of all gradient paths through at most k
+ * blocks; it is the exact gradient for l >= L-k, and everywhere once k >= L.
+ * Parameter gradients use the final estimate (last sentence of Section 4.2).
+ *
+ * Conventions
+ *  - Every pointer named below is a DEVICE pointer unless it says "host".
+ *    All device buffers are allocated and owned by the caller and are only
+ *    borrowed until the enqueued work has finished.  The library allocates no
+ *    device memory and frees none.
+ *  - All tensors are row-major with the channel dimension contiguous:
+ *    states [L+1][N][d], weights [layer][out][in].  Element type is
+ *    cfg.dtype (float or bf16); parameter gradients are always float.
+ *  - Device pointers must be 16-byte aligned and d, hidden, in_dim must be
+ *    multiples of 8 (bf16) or 4 (float): all access is 128-bit.
+ *  - Calls enqueue work on `cuda_stream` (a cudaStream_t, may be NULL for the
+ *    default stream) and return without synchronising, except
+ *    hbp_sync_status.  They are not thread-safe per context.
+ *  - Errors are returned as status codes.  Nothing aborts, throws or traps.
+ */
+#ifndef HBP_H_
+#define HBP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hbp_ctx hbp_ctx; /* opaque, host memory, made by hbp_create */
+
+typedef enum {
+  HBP_OK = 0,
+  HBP_ERR_INVALID_ARG = 1, /* NULL where a pointer is required, k < 0, ...          */
+  HBP_ERR_SHAPE = 2,       /* a size is <= 0 or violates the alignment rule        */
+  HBP_ERR_DTYPE = 3,
+  HBP_ERR_STATE = 4,       /* backward / exact before any forward                  */
+  HBP_ERR_WORKSPACE = 5,   /* workspace too small or misaligned                    */
+  HBP_ERR_UNSUPPORTED = 6,
+  HBP_ERR_CUDA = 7,        /* a CUDA runtime call or launch failed                 */
+  HBP_ERR_TIMEOUT = 8      /* a bounded device-side wait expired (status word)     */
+} hbp_status;
+
+/* Block kinds f_l (Table 1; Section 5.1.1 for the Transformer split; Section 5.2 for the RNN).
+ *  MLP               f(x) = W2 gelu(W1 x)                     (exact erf GELU, no biases)
+ *  PRELN_MLP         f(x) = W2 gelu(W1 LN(x))                 (LN without affine, biased variance)
+ *  RNN_TANH          f_t(h) = tanh(W h + U x_t), weights shared over t; L is the sequence length
+ *  PRELN_TRANSFORMER L decoder blocks = 2L residual steps: causal softmax MHA(LN(x)) Wo, then PRELN_MLP */
+typedef enum { HBP_BLOCK_MLP = 0, HBP_BLOCK_PRELN_MLP = 1, HBP_BLOCK_RNN_TANH = 2, HBP_BLOCK_PRELN_TRANSFORMER = 3 } hbp_block;
+typedef enum { HBP_F32 = 0, HBP_BF16 = 1 } hbp_dtype;
+/* Residual gate a_l, the diagonal of K (Eq. 2): all ones, one vector a[d] for every step, or a[steps][d]. */
+typedef enum { HBP_GATE_ONE = 0, HBP_GATE_CHANNEL_SHARED = 1, HBP_GATE_CHANNEL_PER_STEP = 2 } hbp_gate;
+/* Where the loss acts (Section 3): on the last state only (delta is [N][d]) or on every state
+ * (delta is [steps+1][N][d]; delta[0] belongs to x_0 and is usually zero). */
+typedef enum { HBP_LOSS_FINAL = 0, HBP_LOSS_EVERY_STEP = 1 } hbp_loss;
+
+typedef struct {
+  int32_t block;    /* hbp_block */
+  int32_t dtype;    /* hbp_dtype */
+  int32_t gate;     /* hbp_gate  */
+  int32_t loss;     /* hbp_loss  */
+  int32_t L;        /* residual steps (MLP kinds), time steps (RNN), decoder blocks (Transformer) */
+  int32_t d;        /* state width */
+  int32_t hidden;   /* MLP hidden width (MLP kinds, Transformer) */
+  int32_t in_dim;   /* RNN input width */
+  int32_t n_heads;  /* Transformer: n_heads * head_dim == d */
+  int32_t head_dim;
+  int32_t seq;      /* Transformer: tokens == batch * seq */
+  int32_t batch;    /* Transformer: sequences; RNN: rows (== tokens) */
+  int64_t tokens;   /* N: rows of one state */
+  float ln_eps;
+  int32_t reserved;
+} hbp_config;
+
+/* Borrowed parameter pointers; those the block kind does not use are ignored.
+ *  MLP kinds:    W1 [L][hidden][d], W2 [L][d][hidden]
+ *  RNN:          W [d][d], U [d][in_dim]
+ *  Transformer:  Wq, Wk, Wv, Wo [L][d][d], W1 [L][hidden][d], W2 [L][d][hidden]
+ *  gate:         a [d] or [steps][d] when cfg.gate != HBP_GATE_ONE (steps = 2L for the Transformer) */
+typedef struct {
+  const void *W1, *W2;
+  const void *W, *U;
+  const void *Wq, *Wk, *Wv, *Wo;
+  const void *a;
+} hbp_params;
+
+/* Caller-owned float outputs with the shapes of the parameters; OVERWRITTEN, not accumulated.
+ * da has the shape of the gate and may be NULL to skip it. */
+typedef struct {
+  float *dW1, *dW2;
+  float *dW, *dU;
+  float *dWq, *dWk, *dWv, *dWo;
+  float *da;
+} hbp_grads;
+
+/* Bytes of caller-provided device workspace a context for `cfg` needs (activation caches of the
+ * last forward, per-iteration scratch, a status word).  HBP_ERR_SHAPE / _DTYPE / _UNSUPPORTED on a
+ * bad config. */
+hbp_status hbp_workspace_bytes(const hbp_config* cfg, size_t* bytes);
+
+/* Makes a context over `workspace` (device, 256-byte aligned, >= hbp_workspace_bytes).  The
+ * workspace is borrowed until hbp_destroy.  *out is host memory owned by the library. */
+hbp_status hbp_create(const hbp_config* cfg, void* workspace, size_t workspace_bytes, hbp_ctx** out);
+
+/* Section 3, h_i = f_i(h_{i-1}): runs the steps from x0 [N][d] and stores every state in
+ * x_all [steps+1][N][d] (x_all[0] = x0) plus, in the workspace, what the block VJPs need.
+ * `inputs` is the RNN's x [L][batch][in_dim] (NULL otherwise). */
+hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, const void* inputs,
+                       void* x_all, void* cuda_stream);
+
+/* Theorem 2 / Eq. 8-11: k Highway-BP iterations from the caches of the last hbp_forward.
+ * delta: see hbp_loss.  g_all [steps+1][N][d] receives g^k (g_all[steps] = delta_L always).
+ * grads == NULL skips the parameter-gradient pass; otherwise it is computed from g^k (Section 4.2).
+ * k >= steps returns the exact gradient (the loop stops there).  x_all and inputs must be the
+ * buffers the last hbp_forward used. */
+hbp_status hbp_backward(hbp_ctx* ctx, const hbp_params* params, int32_t k, const void* delta,
+                        const void* x_all, const void* inputs, void* g_all, const hbp_grads* grads,
+                        void* cuda_stream);
+
+/* Section 2.2: sequential exact backpropagation, l = L-1..0, through the same block kernels. */
+hbp_status hbp_exact(hbp_ctx* ctx, const hbp_params* params, const void* delta, const void* x_all,
+                     const void* inputs, void* g_all, const hbp_grads* grads, void* cuda_stream);
+
+/* Eq. 9 / Eq. 12 on its own: g[L] = delta_L and g[l] = delta_l + a_l (.) g[l+1] + u[l] for l = L-1..0,
+ * i.e. the reverse CumSumProd with diagonal K.  u [L][rows][d] (NULL = zeros), delta as in hbp_loss
+ * (`loss`), a as in hbp_gate (`gate`), g [L+1][rows][d].  `scratch` is device memory of at least
+ * hbp_cumsumprod_scratch_bytes(...) bytes (may be NULL when that is 0). */
+hbp_status hbp_cumsumprod_scratch_bytes(int32_t dtype, int32_t L, int64_t rows, int32_t d, size_t* bytes);
+hbp_status hbp_cumsumprod(int32_t dtype, int32_t gate, int32_t loss, int32_t L, int64_t rows, int32_t d,
+                          const void* u, const void* delta, const void* a, void* g,
+                          void* scratch, size_t scratch_bytes, void* cuda_stream);
+
+/* Copies the context's device status word to the host after synchronising the stream: HBP_OK, or the
+ * error a kernel recorded (HBP_ERR_TIMEOUT when a bounded wait gave up).  The only synchronising call. */
+hbp_status hbp_sync_status(hbp_ctx* ctx, void* cuda_stream);
+
+/* Number of kernels this context has launched since creation (host counter). */
+int64_t hbp_launch_count(const hbp_ctx* ctx);
+
+const char* hbp_status_string(hbp_status s);
+void hbp_destroy(hbp_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HBP_H_ */
