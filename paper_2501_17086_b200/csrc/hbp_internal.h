@@ -1,0 +1,140 @@
+// Internal declarations shared by the CUDA translation units of libhbp.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hbp.h"
+
+namespace hbp {
+
+typedef __nv_bfloat16 bf16;
+
+// ---------------------------------------------------------------- GEMM description
+// D(m, n) = sum_k A(m, k) * B(n, k) per batch entry, fp32 accumulation, followed by an epilogue.
+// A(m, k) lives at A + batch*a_sb + m*a_sm + k*a_sk (element strides), B(n, k) likewise.
+enum Epilogue {
+  EPI_STORE = 0,     // D = acc
+  EPI_GELU_FWD = 1,  // D = acc (pre-activation Z), D2 = gelu(acc)
+  EPI_RESID = 2,     // v = gate[n] * r + acc with r = R ? R[m,n] : E[m,n];  R = v (if R);  D = v
+  EPI_DGELU = 3,     // D = acc * gelu'(E[m,n]);  D2 = gelu(E[m,n]) if D2
+  EPI_AFFINE = 4,    // D = (E ? E[m,n] : 0) + gate[n] * E2[m,n] + acc
+  EPI_RNN_FWD = 5,   // c = tanh(acc + E[m,n]);  D2 = c;  D = gate[n] * E2[m,n] + c
+};
+
+struct GemmArgs {
+  int M = 0, N = 0, K = 0, batch = 1;
+  int in_dtype = HBP_F32;  // element type of A, A2, B, D2, E, E2, gate and of D unless d_f32
+  const void* A = nullptr;
+  int64_t a_sm = 0, a_sk = 0, a_sb = 0;
+  const void* A2 = nullptr;  // if set, the A operand is A * (1 - A2^2), A2 indexed like A
+  const void* B = nullptr;
+  int64_t b_sn = 0, b_sk = 0, b_sb = 0;
+  int epi = EPI_STORE;
+  void* D = nullptr;
+  int64_t ldd = 0, d_sb = 0;
+  bool d_f32 = false;  // D is float regardless of in_dtype
+  void* D2 = nullptr;
+  int64_t ldd2 = 0, d2_sb = 0;
+  const void* E = nullptr;
+  int64_t lde = 0, e_sb = 0;
+  const void* E2 = nullptr;
+  int64_t lde2 = 0, e2_sb = 0;
+  const void* gate = nullptr;  // [N] per batch entry (stride gate_sb), nullptr = ones
+  int64_t gate_sb = 0;
+  float* R = nullptr;  // fp32 master copy of the residual stream [M][N], leading dim N
+  int splitk = 1;      // > 1: partial sums to `partial` [splitk][batch][M][N], reduced in fixed order
+  float* partial = nullptr;
+};
+
+// Counts launches and remembers the first CUDA error.
+struct Launcher {
+  cudaStream_t stream = nullptr;
+  int64_t* launches = nullptr;
+  cudaError_t err = cudaSuccess;
+  void count(int n = 1) {
+    if (launches) *launches += n;
+  }
+  void check() {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess && err == cudaSuccess) err = e;
+  }
+};
+
+// CUDA-core GEMM for any strides and both dtypes (gemm_simt.cu).
+void gemm_simt(Launcher& lc, const GemmArgs& g);
+// tcgen05 / TMEM / TMA GEMM for bf16 operands; returns false if the problem does not meet its
+// alignment rules, in which case nothing was launched (gemm_tc.cu).
+bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word);
+// Picks gemm_tc when it applies, else gemm_simt.
+void gemm(Launcher& lc, const GemmArgs& g, int* status_word);
+// Set from the environment variable HBP_FORCE_SIMT=1 when a context is created: keeps every GEMM
+// on the CUDA-core kernel (used to cross-check the tensor-core kernel).
+extern bool g_force_simt;
+
+// ---------------------------------------------------------------- scans and elementwise (scan.cu)
+struct ScanArgs {
+  int dtype = HBP_F32;
+  int L = 0;               // number of steps in the buffers
+  int l_lo = 0, l_hi = 0;  // processes l = l_hi-1 .. l_lo, carry-in read from g[l_hi]
+  int64_t rows = 0;
+  int d = 0;
+  const void* u = nullptr;      // [L][rows][d] or nullptr (zeros)
+  const void* delta = nullptr;  // per hbp_loss
+  int loss = HBP_LOSS_FINAL;
+  const void* a = nullptr;  // gate
+  int gate = HBP_GATE_ONE;
+  void* g = nullptr;  // [L+1][rows][d]
+  // LayerNorm-backward finish: u is dY; the kernel forms rstd * (dy - mean(dy) - xhat * mean(dy*xhat)).
+  // xhat [L][rows][d] in dtype, rstd [L][rows] float.
+  const void* xhat = nullptr;
+  const float* rstd = nullptr;
+  void* scratch = nullptr;  // time-chunked variant only
+  size_t scratch_bytes = 0;
+};
+size_t scan_scratch_bytes(int dtype, int L, int64_t rows, int d);
+void scan_reverse(Launcher& lc, const ScanArgs& s);
+void copy_state(Launcher& lc, int dtype, void* dst, const void* src, int64_t elems);
+// LayerNorm forward of one state: x (float master or dtype) -> xhat (dtype), rstd (float).
+void layernorm_fwd(Launcher& lc, int dtype, const void* x, bool x_is_f32, void* xhat, float* rstd, int64_t rows,
+                   int d, float eps);
+void convert_to_f32(Launcher& lc, int dtype, const void* src, float* dst, int64_t elems);
+// da[c] = sum over rows of g[r][c] * x[r][c] (deterministic two-stage reduction; partial holds blocks*d floats).
+void gate_grad(Launcher& lc, int dtype, const void* g, const void* x, int64_t rows_total, int d, float* da,
+               float* partial, int blocks);
+void reduce_splitk(Launcher& lc, const float* partial, float* out, int splits, int64_t elems);
+
+// ---------------------------------------------------------------- attention (attention.cu)
+struct AttnArgs {
+  int dtype = HBP_BF16;
+  int batch = 0, seq = 0, heads = 0, head_dim = 0;
+  // q, k, v are column blocks of one [tokens][3d] buffer (ld = 3d); o, d_o are [tokens][d].
+  const void* qkv = nullptr;
+  void* o = nullptr;
+  float* lse = nullptr;  // [batch][heads][seq]
+  const void* d_o = nullptr;
+  void* d_qkv = nullptr;        // [tokens][3d]
+  float* delta_rows = nullptr;  // scratch [batch][heads][seq]: rowsum(dO * O)
+};
+void attention_fwd(Launcher& lc, const AttnArgs& a);
+void attention_bwd(Launcher& lc, const AttnArgs& a);
+
+// ---------------------------------------------------------------- device math
+__device__ __forceinline__ float gelu_f(float z) { return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f)); }
+__device__ __forceinline__ float gelu_prime_f(float z) {
+  return 0.5f * (1.0f + erff(z * 0.70710678118654752440f)) + z * expf(-0.5f * z * z) * 0.39894228040143267794f;
+}
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+template <typename T>
+__device__ __forceinline__ T from_f(float v);
+template <>
+__device__ __forceinline__ float from_f<float>(float v) {
+  return v;
+}
+template <>
+__device__ __forceinline__ bf16 from_f<bf16>(float v) {
+  return __float2bfloat16_rn(v);
+}
+
+}  // namespace hbp
