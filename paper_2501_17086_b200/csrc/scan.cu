@@ -209,3 +209,242 @@ __global__ void __launch_bounds__(1024) scan_depth_ln_kernel(const ScanArgs s) {
     }
   }
 }
+
+// ---- time-chunked scan for long L and few channels (three phases) ----------------------------------
+// Phase 1: per (chunk, channel group) local scan with zero carry-in -> S (value at the chunk's first
+// step) and P (product of the gates over the chunk).  Phase 2: per channel, serial over the chunks:
+// carry-in of chunk c = G_{c+1}, G_c = S_c + P_c * G_{c+1}.  Phase 3: local scan again with the
+// carry-in, writing g.  Scratch: S (then the carry-ins) [nchunks][rows*d] and P likewise, float.
+constexpr int kChunk = 32;
+
+template <typename T, bool kApply>
+__global__ void __launch_bounds__(128) scan_chunk_kernel(const ScanArgs s, float* __restrict__ S,
+                                                         float* __restrict__ P) {
+  constexpr int V = Vec<T>::N;
+  const int64_t state_elems = s.rows * s.d;
+  const int64_t nvec = state_elems / V;
+  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v >= nvec) return;
+  const int c = blockIdx.y;
+  const int lo = s.l_lo + c * kChunk, hi = min(s.l_hi, lo + kChunk);
+  const int64_t off = v * V;
+  const int ch = (int)(off % s.d);
+  T* g = (T*)s.g;
+  float carry[V], prod[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    carry[i] = kApply ? S[(int64_t)c * state_elems + off + i] : 0.0f;
+    prod[i] = 1.0f;
+  }
+  for (int l = hi - 1; l >= lo; --l) {
+    float val[V];
+    scan_step<T>(s, l, state_elems, off, ch, carry, val);
+    if (kApply) {
+      Vec<T> out;
+      out.set(val);
+      stv<T>(g + (int64_t)l * state_elems + off, out);
+    } else {
+      const T* gp = gate_at<T>(s, l);
+      if (gp) {
+        float a[V];
+        ldv<T>(gp + ch).get(a);
+#pragma unroll
+        for (int i = 0; i < V; ++i) prod[i] *= a[i];
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < V; ++i) carry[i] = val[i];
+  }
+  if (!kApply) {
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      S[(int64_t)c * state_elems + off + i] = carry[i];
+      P[(int64_t)c * state_elems + off + i] = prod[i];
+    }
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(128) scan_carry_kernel(const ScanArgs s, float* __restrict__ S,
+                                                         const float* __restrict__ P, int nchunks) {
+  const int64_t state_elems = s.rows * s.d;
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= state_elems) return;
+  float G = to_f(((const T*)s.g)[(int64_t)s.l_hi * state_elems + e]);
+  for (int c = nchunks - 1; c >= 0; --c) {
+    const float sc = S[(int64_t)c * state_elems + e], pc = P[(int64_t)c * state_elems + e];
+    S[(int64_t)c * state_elems + e] = G;  // carry-in of chunk c
+    G = sc + pc * G;
+  }
+}
+
+// ---- row-wise helpers ----------------------------------------------------------------------------
+template <typename T>
+__global__ void copy_kernel(T* __restrict__ dst, const T* __restrict__ src, int64_t nvec) {
+  int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v < nvec) stv<T>(dst + v * Vec<T>::N, ldv<T>(src + v * Vec<T>::N));
+}
+
+template <typename T>
+__global__ void to_f32_kernel(const T* __restrict__ src, float* __restrict__ dst, int64_t n) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = to_f(src[i]);
+}
+
+// xhat = (x - mean) * rstd over the last axis, biased variance; one block per row, two passes in registers.
+template <typename T, typename X>
+__global__ void __launch_bounds__(1024) layernorm_fwd_kernel(const X* __restrict__ x, T* __restrict__ xhat,
+                                                             float* __restrict__ rstd, int d, float eps) {
+  constexpr int V = Vec<T>::N;
+  __shared__ float red[2][32];
+  const int64_t row = blockIdx.x;
+  const bool active = (int)threadIdx.x * V < d;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
+  float val[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) val[i] = active ? to_f(x[row * d + threadIdx.x * V + i]) : 0.0f;
+  float s1 = 0.0f;
+#pragma unroll
+  for (int i = 0; i < V; ++i) s1 += val[i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+  if (lane == 0) red[0][warp] = s1;
+  __syncthreads();
+  float t = 0.0f;
+  for (int w = 0; w < nwarps; ++w) t += red[0][w];
+  const float mu = t / (float)d;
+  float s2 = 0.0f;
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    const float c = active ? val[i] - mu : 0.0f;
+    s2 = fmaf(c, c, s2);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+  if (lane == 0) red[1][warp] = s2;
+  __syncthreads();
+  t = 0.0f;
+  for (int w = 0; w < nwarps; ++w) t += red[1][w];
+  const float r = rsqrtf(t / (float)d + eps);
+  if (threadIdx.x == 0) rstd[row] = r;
+  if (active) {
+    float o[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) o[i] = (val[i] - mu) * r;
+    Vec<T> out;
+    out.set(o);
+    stv<T>(xhat + row * d + threadIdx.x * V, out);
+  }
+}
+
+// partial[b][c] = sum over the block's rows of g[r][c] * x[r][c]
+template <typename T>
+__global__ void __launch_bounds__(256) gate_grad_kernel(const T* __restrict__ g, const T* __restrict__ x,
+                                                        int64_t rows, int d, float* __restrict__ partial) {
+  const int64_t per = (rows + gridDim.x - 1) / gridDim.x;
+  const int64_t r0 = (int64_t)blockIdx.x * per, r1 = min(rows, r0 + per);
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float acc = 0.0f;
+    for (int64_t r = r0; r < r1; ++r) acc = fmaf(to_f(g[r * d + c]), to_f(x[r * d + c]), acc);
+    partial[(int64_t)blockIdx.x * d + c] = acc;
+  }
+}
+
+inline int row_block_threads(int d, int V) {
+  int t = (d / V + 31) / 32 * 32;
+  return t < 32 ? 32 : t;
+}
+
+}  // namespace
+
+size_t scan_scratch_bytes(int dtype, int L, int64_t rows, int d) {
+  const int V = dtype == HBP_F32 ? 4 : 8;
+  const int64_t nvec = rows * d / V;
+  if (nvec >= 148 * 512 || L < 4 * kChunk) return 0;  // enough channels (or too short) for the serial form
+  const int nchunks = (L + kChunk - 1) / kChunk;
+  return (size_t)2 * nchunks * rows * d * sizeof(float);
+}
+
+void scan_reverse(Launcher& lc, const ScanArgs& s) {
+  if (s.l_hi <= s.l_lo || s.rows <= 0) return;
+  const int V = s.dtype == HBP_F32 ? 4 : 8;
+  const int64_t nvec = s.rows * s.d / V;
+  if (s.xhat) {
+    const int threads = row_block_threads(s.d, V);
+    if (s.dtype == HBP_F32) scan_depth_ln_kernel<float><<<(unsigned)s.rows, threads, 0, lc.stream>>>(s);
+    else scan_depth_ln_kernel<bf16><<<(unsigned)s.rows, threads, 0, lc.stream>>>(s);
+    lc.count();
+    lc.check();
+    return;
+  }
+  const int steps = s.l_hi - s.l_lo;
+  const size_t need = scan_scratch_bytes(s.dtype, steps, s.rows, s.d);
+  if (need > 0 && s.scratch && s.scratch_bytes >= need) {
+    const int nchunks = (steps + kChunk - 1) / kChunk;
+    float* S = (float*)s.scratch;
+    float* P = S + (int64_t)nchunks * s.rows * s.d;
+    dim3 grid((unsigned)((nvec + 127) / 128), nchunks);
+    const unsigned cgrid = (unsigned)((s.rows * s.d + 127) / 128);
+    if (s.dtype == HBP_F32) {
+      scan_chunk_kernel<float, false><<<grid, 128, 0, lc.stream>>>(s, S, P);
+      scan_carry_kernel<float><<<cgrid, 128, 0, lc.stream>>>(s, S, P, nchunks);
+      scan_chunk_kernel<float, true><<<grid, 128, 0, lc.stream>>>(s, S, P);
+    } else {
+      scan_chunk_kernel<bf16, false><<<grid, 128, 0, lc.stream>>>(s, S, P);
+      scan_carry_kernel<bf16><<<cgrid, 128, 0, lc.stream>>>(s, S, P, nchunks);
+      scan_chunk_kernel<bf16, true><<<grid, 128, 0, lc.stream>>>(s, S, P);
+    }
+    lc.count(3);
+    lc.check();
+    return;
+  }
+  const unsigned grid = (unsigned)((nvec + 255) / 256);
+  if (s.dtype == HBP_F32) scan_depth_kernel<float><<<grid, 256, 0, lc.stream>>>(s);
+  else scan_depth_kernel<bf16><<<grid, 256, 0, lc.stream>>>(s);
+  lc.count();
+  lc.check();
+}
+
+void copy_state(Launcher& lc, int dtype, void* dst, const void* src, int64_t elems) {
+  if (dtype == HBP_F32)
+    copy_kernel<float><<<(unsigned)((elems / 4 + 255) / 256), 256, 0, lc.stream>>>((float*)dst, (const float*)src, elems / 4);
+  else
+    copy_kernel<bf16><<<(unsigned)((elems / 8 + 255) / 256), 256, 0, lc.stream>>>((bf16*)dst, (const bf16*)src, elems / 8);
+  lc.count();
+  lc.check();
+}
+
+void convert_to_f32(Launcher& lc, int dtype, const void* src, float* dst, int64_t elems) {
+  const unsigned grid = (unsigned)((elems + 255) / 256);
+  if (dtype == HBP_F32) to_f32_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)src, dst, elems);
+  else to_f32_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)src, dst, elems);
+  lc.count();
+  lc.check();
+}
+
+void layernorm_fwd(Launcher& lc, int dtype, const void* x, bool x_is_f32, void* xhat, float* rstd, int64_t rows,
+                   int d, float eps) {
+  const int V = dtype == HBP_F32 ? 4 : 8;
+  const int threads = row_block_threads(d, V);
+  if (dtype == HBP_F32)
+    layernorm_fwd_kernel<float, float><<<(unsigned)rows, threads, 0, lc.stream>>>((const float*)x, (float*)xhat, rstd, d, eps);
+  else if (x_is_f32)
+    layernorm_fwd_kernel<bf16, float><<<(unsigned)rows, threads, 0, lc.stream>>>((const float*)x, (bf16*)xhat, rstd, d, eps);
+  else
+    layernorm_fwd_kernel<bf16, bf16><<<(unsigned)rows, threads, 0, lc.stream>>>((const bf16*)x, (bf16*)xhat, rstd, d, eps);
+  lc.count();
+  lc.check();
+}
+
+void gate_grad(Launcher& lc, int dtype, const void* g, const void* x, int64_t rows_total, int d, float* da,
+               float* partial, int blocks) {
+  if (dtype == HBP_F32)
+    gate_grad_kernel<float><<<blocks, 256, 0, lc.stream>>>((const float*)g, (const float*)x, rows_total, d, partial);
+  else
+    gate_grad_kernel<bf16><<<blocks, 256, 0, lc.stream>>>((const bf16*)g, (const bf16*)x, rows_total, d, partial);
+  lc.count();
+  lc.check();
+  reduce_splitk(lc, partial, da, blocks, d);
+}
+
+}  // namespace hbp
