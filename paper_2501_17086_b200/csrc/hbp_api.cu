@@ -165,9 +165,6 @@ struct Run {
     if (c->cfg.gate == HBP_GATE_ONE) return nullptr;
     return at(p->a, c->cfg.gate == HBP_GATE_CHANNEL_PER_STEP ? (int64_t)step * d : 0);
   }
-  int64_t gate_stride(int step_stride) const {
-    return c->cfg.gate == HBP_GATE_CHANNEL_PER_STEP ? (int64_t)step_stride * d : 0;
-  }
   GemmArgs base_args() const {
     GemmArgs a;
     a.in_dtype = c->cfg.dtype;
@@ -358,3 +355,304 @@ hbp_status check_grads(const hbp_ctx* ctx, const hbp_grads* g) {
 bool misaligned(const void* p) { return ((uintptr_t)p & 15u) != 0; }
 
 }  // namespace
+
+extern "C" {
+
+const char* hbp_status_string(hbp_status s) {
+  switch (s) {
+    case HBP_OK: return "ok";
+    case HBP_ERR_INVALID_ARG: return "invalid argument";
+    case HBP_ERR_SHAPE: return "bad shape or alignment";
+    case HBP_ERR_DTYPE: return "bad dtype";
+    case HBP_ERR_STATE: return "backward before forward";
+    case HBP_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case HBP_ERR_UNSUPPORTED: return "unsupported configuration";
+    case HBP_ERR_CUDA: return "CUDA error";
+    case HBP_ERR_TIMEOUT: return "bounded device wait expired";
+  }
+  return "unknown status";
+}
+
+hbp_status hbp_workspace_bytes(const hbp_config* cfg, size_t* bytes) {
+  if (!bytes) return HBP_ERR_INVALID_ARG;
+  hbp_status st = check_config(cfg);
+  if (st != HBP_OK) return st;
+  hbp_ctx tmp;
+  tmp.cfg = *cfg;
+  *bytes = carve(&tmp, nullptr);
+  return HBP_OK;
+}
+
+hbp_status hbp_create(const hbp_config* cfg, void* workspace, size_t workspace_bytes, hbp_ctx** out) {
+  if (!out) return HBP_ERR_INVALID_ARG;
+  *out = nullptr;
+  hbp_status st = check_config(cfg);
+  if (st != HBP_OK) return st;
+  if (!workspace || ((uintptr_t)workspace % kAlign)) return HBP_ERR_WORKSPACE;
+  hbp_ctx* c = new (std::nothrow) hbp_ctx;
+  if (!c) return HBP_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  const size_t need = carve(c, (char*)workspace);
+  if (workspace_bytes < need) {
+    delete c;
+    return HBP_ERR_WORKSPACE;
+  }
+  c->ws = (char*)workspace;
+  c->ws_bytes = workspace_bytes;
+  const char* env = std::getenv("HBP_FORCE_SIMT");
+  g_force_simt = env && env[0] == '1';
+  if (cudaMemset(c->status, 0, 256) != cudaSuccess) {
+    delete c;
+    return HBP_ERR_CUDA;
+  }
+  *out = c;
+  return HBP_OK;
+}
+
+void hbp_destroy(hbp_ctx* ctx) { delete ctx; }
+
+int64_t hbp_launch_count(const hbp_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+hbp_status hbp_sync_status(hbp_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return HBP_ERR_INVALID_ARG;
+  int word = 0;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  if (cudaMemcpyAsync(&word, ctx->status, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return HBP_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return HBP_ERR_CUDA;
+  return (hbp_status)word;
+}
+
+hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, const void* inputs, void* x_all,
+                       void* cuda_stream) {
+  hbp_status st = check_call(ctx, params, false);
+  if (st != HBP_OK) return st;
+  if (!x0 || !x_all) return HBP_ERR_INVALID_ARG;
+  if (misaligned(x0) || misaligned(x_all)) return HBP_ERR_SHAPE;
+  const hbp_config& f = ctx->cfg;
+  if (f.block == HBP_BLOCK_RNN_TANH && !inputs) return HBP_ERR_INVALID_ARG;
+  Run r(ctx, params, cuda_stream);
+  r.x_all = (const char*)x_all;
+  char* xa = (char*)x_all;
+  const int64_t N = r.N, d = r.d, h = r.h, state = r.state;
+  copy_state(r.lc, f.dtype, xa, x0, state);
+  if (ctx->xres) convert_to_f32(r.lc, f.dtype, x0, ctx->xres, state);
+
+  if (f.block == HBP_BLOCK_RNN_TANH) {
+    const int T = f.L;
+    GemmArgs a = r.base_args();  // input projection for every t at once
+    a.M = (int)(T * N); a.N = (int)d; a.K = f.in_dim;
+    a.A = inputs; a.a_sm = f.in_dim; a.a_sk = 1;
+    a.B = params->U; a.b_sn = f.in_dim; a.b_sk = 1;
+    a.epi = EPI_STORE; a.D = ctx->C; a.ldd = d;
+    r.run_gemm(a);
+    for (int t = 0; t < T; ++t) {
+      GemmArgs s = r.base_args();
+      s.M = (int)N; s.N = (int)d; s.K = (int)d;
+      s.A = r.at(xa, (int64_t)t * state); s.a_sm = d; s.a_sk = 1;
+      s.B = params->W; s.b_sn = d; s.b_sk = 1;
+      s.epi = EPI_RNN_FWD;
+      s.E = r.at(ctx->C, (int64_t)t * state); s.lde = d;
+      s.E2 = r.at(xa, (int64_t)t * state); s.lde2 = d;
+      s.gate = r.gate_ptr(t);
+      s.D2 = r.at(ctx->C, (int64_t)t * state); s.ldd2 = d;
+      s.D = r.at(xa, (int64_t)(t + 1) * state); s.ldd = d;
+      r.run_gemm(s);
+    }
+  } else {
+    const bool tr = f.block == HBP_BLOCK_PRELN_TRANSFORMER;
+    if (tr) {  // stack Wq, Wk, Wv per layer so that QKV and its VJP are single GEMMs
+      const size_t blk = (size_t)d * d * r.es;
+      const void* src[3] = {params->Wq, params->Wk, params->Wv};
+      for (int w = 0; w < 3; ++w) {
+        cudaError_t e = cudaMemcpy2DAsync(ctx->Wqkv + w * blk, 3 * blk, src[w], blk, blk, (size_t)f.L,
+                                          cudaMemcpyDeviceToDevice, r.lc.stream);
+        if (e != cudaSuccess && r.lc.err == cudaSuccess) r.lc.err = e;
+      }
+    }
+    // residual update x_{l+1} = a * x_l + F through the float master copy when there is one
+    auto resid_epilogue = [&](GemmArgs& a, int step) {
+      a.epi = EPI_RESID;
+      a.gate = r.gate_ptr(step);
+      if (ctx->xres) a.R = ctx->xres;
+      else { a.E = r.at(xa, (int64_t)step * state); a.lde = d; }
+      a.D = r.at(xa, (int64_t)(step + 1) * state); a.ldd = d;
+    };
+    auto ln_of = [&](int step) {
+      const void* src = ctx->xres ? (const void*)ctx->xres : (const void*)r.at(xa, (int64_t)step * state);
+      layernorm_fwd(r.lc, f.dtype, src, ctx->xres != nullptr, r.at(ctx->Y, (int64_t)step * state),
+                    ctx->rstd + (int64_t)step * N, N, (int)d, f.ln_eps);
+    };
+    for (int b = 0; b < f.L; ++b) {
+      if (tr) {
+        const int step = 2 * b;
+        ln_of(step);
+        GemmArgs q = r.base_args();
+        q.M = (int)N; q.N = (int)(3 * d); q.K = (int)d;
+        q.A = r.at(ctx->Y, (int64_t)step * state); q.a_sm = d; q.a_sk = 1;
+        q.B = r.at(ctx->Wqkv, (int64_t)b * 3 * d * d); q.b_sn = d; q.b_sk = 1;
+        q.epi = EPI_STORE; q.D = r.at(ctx->QKV, (int64_t)b * 3 * state); q.ldd = 3 * d;
+        r.run_gemm(q);
+        AttnArgs t;
+        t.dtype = f.dtype; t.batch = f.batch; t.seq = f.seq; t.heads = f.n_heads; t.head_dim = f.head_dim;
+        t.qkv = r.at(ctx->QKV, (int64_t)b * 3 * state);
+        t.o = r.at(ctx->O, (int64_t)b * state);
+        t.lse = ctx->lse + (int64_t)b * f.batch * f.n_heads * f.seq;
+        attention_fwd(r.lc, t);
+        GemmArgs o = r.base_args();
+        o.M = (int)N; o.N = (int)d; o.K = (int)d;
+        o.A = r.at(ctx->O, (int64_t)b * state); o.a_sm = d; o.a_sk = 1;
+        o.B = r.at(params->Wo, (int64_t)b * d * d); o.b_sn = d; o.b_sk = 1;
+        resid_epilogue(o, step);
+        r.run_gemm(o);
+      }
+      const int step = r.mlp_step(b);
+      if (ctx->preln) ln_of(step);
+      GemmArgs a = r.base_args();
+      a.M = (int)N; a.N = (int)h; a.K = (int)d;
+      a.A = r.mlp_operand(b); a.a_sm = d; a.a_sk = 1;
+      a.B = r.at(params->W1, (int64_t)b * h * d); a.b_sn = d; a.b_sk = 1;
+      a.epi = EPI_GELU_FWD;
+      a.D = r.at(ctx->Z, (int64_t)b * N * h); a.ldd = h;
+      a.D2 = ctx->H2; a.ldd2 = h;
+      r.run_gemm(a);
+      GemmArgs c2 = r.base_args();
+      c2.M = (int)N; c2.N = (int)d; c2.K = (int)h;
+      c2.A = ctx->H2; c2.a_sm = h; c2.a_sk = 1;
+      c2.B = r.at(params->W2, (int64_t)b * d * h); c2.b_sn = h; c2.b_sk = 1;
+      resid_epilogue(c2, step);
+      r.run_gemm(c2);
+    }
+  }
+  ctx->forward_done = true;
+  return r.result();
+}
+
+static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_t k, bool exact, const void* delta,
+                                  const void* x_all, const void* inputs, void* g_all, const hbp_grads* grads,
+                                  void* cuda_stream) {
+  hbp_status st = check_call(ctx, params, true);
+  if (st != HBP_OK) return st;
+  if (!delta || !x_all || !g_all || k < 0) return HBP_ERR_INVALID_ARG;
+  if (misaligned(delta) || misaligned(x_all) || misaligned(g_all)) return HBP_ERR_SHAPE;
+  st = check_grads(ctx, grads);
+  if (st != HBP_OK) return st;
+  const hbp_config& f = ctx->cfg;
+  if (f.block == HBP_BLOCK_RNN_TANH && grads && !inputs) return HBP_ERR_INVALID_ARG;
+  Run r(ctx, params, cuda_stream);
+  r.x_all = (const char*)x_all;
+  r.inputs = (const char*)inputs;
+  r.g = (char*)g_all;
+  r.delta = (const char*)delta;
+  const int steps = ctx->steps, layers = ctx->layers, grp = ctx->group;
+  const bool tr = f.block == HBP_BLOCK_PRELN_TRANSFORMER, rnn = f.block == HBP_BLOCK_RNN_TANH;
+  r.set_last_state();
+
+  if (!exact) {
+    // g^0 = CumSumProd(delta, K) (Eq. 10), then k iterations of {all-step VJP (Eq. 8); reverse scan (Eq. 9, 11)}
+    scan_reverse(r.lc, r.scan_args(0, steps, false));
+    const int iters = k < steps ? k : steps;
+    for (int it = 0; it < iters; ++it) {
+      if (rnn) {
+        r.rnn_vjp_all();
+      } else {
+        for (int b0 = 0; b0 < layers; b0 += grp) r.mlp_vjp(b0, b0 + grp < layers ? b0 + grp : layers, false, true);
+        if (tr) r.attn_vjp(0, layers, true);
+      }
+      scan_reverse(r.lc, r.scan_args(0, steps, true));
+    }
+    if (grads) {  // Section 4.2: parameter gradients from the final estimate
+      if (rnn) {
+        r.rnn_wgrad(grads);
+      } else {
+        for (int b0 = 0; b0 < layers; b0 += grp) {
+          const int b1 = b0 + grp < layers ? b0 + grp : layers;
+          r.mlp_vjp(b0, b1, true, false);
+          r.mlp_wgrad(b0, b1, grads);
+        }
+        if (tr) {
+          r.attn_vjp(0, layers, false);
+          r.attn_wgrad(0, layers, grads);
+        }
+      }
+      r.gate_grads(grads);
+    }
+  } else {
+    // Section 2.2: g_l = delta_l + a_l g_{l+1} + J_l^T g_{l+1}, one step at a time
+    if (rnn) {
+      for (int t = steps - 1; t >= 0; --t) {
+        GemmArgs a = r.base_args();
+        a.M = (int)r.N; a.N = (int)r.d; a.K = (int)r.d;
+        a.A = r.at(r.g, (int64_t)(t + 1) * r.state); a.A2 = r.at(ctx->C, (int64_t)t * r.state); a.a_sm = r.d; a.a_sk = 1;
+        a.B = params->W; a.b_sn = 1; a.b_sk = r.d;
+        a.epi = EPI_AFFINE;
+        a.E = f.loss == HBP_LOSS_EVERY_STEP ? r.at(r.delta, (int64_t)t * r.state) : nullptr; a.lde = r.d;
+        a.E2 = r.at(r.g, (int64_t)(t + 1) * r.state); a.lde2 = r.d;
+        a.gate = r.gate_ptr(t);
+        a.D = r.at(r.g, (int64_t)t * r.state); a.ldd = r.d;
+        r.run_gemm(a);
+      }
+      if (grads) r.rnn_wgrad(grads);
+    } else {
+      for (int l = steps - 1; l >= 0; --l) {
+        const int b = tr ? l / 2 : l;
+        const bool is_mlp = !tr || (l % 2 == 1);
+        if (is_mlp) {
+          r.mlp_vjp(b, b + 1, grads != nullptr, true);
+          if (grads) r.mlp_wgrad(b, b + 1, grads);
+        } else {
+          r.attn_vjp(b, b + 1, true);
+          if (grads) r.attn_wgrad(b, b + 1, grads);
+        }
+        scan_reverse(r.lc, r.scan_args(l, l + 1, true));
+      }
+    }
+    if (grads) r.gate_grads(grads);
+  }
+  return r.result();
+}
+
+hbp_status hbp_backward(hbp_ctx* ctx, const hbp_params* params, int32_t k, const void* delta, const void* x_all,
+                        const void* inputs, void* g_all, const hbp_grads* grads, void* cuda_stream) {
+  return backward_common(ctx, params, k, false, delta, x_all, inputs, g_all, grads, cuda_stream);
+}
+
+hbp_status hbp_exact(hbp_ctx* ctx, const hbp_params* params, const void* delta, const void* x_all, const void* inputs,
+                     void* g_all, const hbp_grads* grads, void* cuda_stream) {
+  return backward_common(ctx, params, 0, true, delta, x_all, inputs, g_all, grads, cuda_stream);
+}
+
+hbp_status hbp_cumsumprod_scratch_bytes(int32_t dtype, int32_t L, int64_t rows, int32_t d, size_t* bytes) {
+  if (!bytes) return HBP_ERR_INVALID_ARG;
+  if (dtype != HBP_F32 && dtype != HBP_BF16) return HBP_ERR_DTYPE;
+  if (L <= 0 || rows <= 0 || d <= 0 || d % (dtype == HBP_F32 ? 4 : 8)) return HBP_ERR_SHAPE;
+  *bytes = scan_scratch_bytes(dtype, L, rows, d);
+  return HBP_OK;
+}
+
+hbp_status hbp_cumsumprod(int32_t dtype, int32_t gate, int32_t loss, int32_t L, int64_t rows, int32_t d, const void* u,
+                          const void* delta, const void* a, void* g, void* scratch, size_t scratch_bytes,
+                          void* cuda_stream) {
+  size_t need = 0;
+  hbp_status st = hbp_cumsumprod_scratch_bytes(dtype, L, rows, d, &need);
+  if (st != HBP_OK) return st;
+  if (!delta || !g) return HBP_ERR_INVALID_ARG;
+  if (gate < 0 || gate > HBP_GATE_CHANNEL_PER_STEP || (loss != HBP_LOSS_FINAL && loss != HBP_LOSS_EVERY_STEP))
+    return HBP_ERR_UNSUPPORTED;
+  if (gate != HBP_GATE_ONE && !a) return HBP_ERR_INVALID_ARG;
+  if (misaligned(u) || misaligned(delta) || misaligned(a) || misaligned(g) || misaligned(scratch)) return HBP_ERR_SHAPE;
+  if (need > 0 && (!scratch || scratch_bytes < need)) return HBP_ERR_WORKSPACE;
+  Launcher lc;
+  lc.stream = (cudaStream_t)cuda_stream;
+  const int64_t state = rows * d;
+  const size_t es = dtype == HBP_F32 ? 4 : 2;
+  const char* dl = loss == HBP_LOSS_EVERY_STEP ? (const char*)delta + (size_t)L * state * es : (const char*)delta;
+  copy_state(lc, dtype, (char*)g + (size_t)L * state * es, dl, state);
+  ScanArgs s;
+  s.dtype = dtype; s.L = L; s.l_lo = 0; s.l_hi = L; s.rows = rows; s.d = d;
+  s.u = u; s.delta = delta; s.loss = loss; s.a = a; s.gate = gate; s.g = g;
+  s.scratch = scratch; s.scratch_bytes = scratch_bytes;
+  scan_reverse(lc, s);
+  return lc.err == cudaSuccess ? HBP_OK : HBP_ERR_CUDA;
+}
+
+}  // extern "C"
