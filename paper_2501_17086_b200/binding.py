@@ -1,0 +1,239 @@
+"""ctypes binding over libhbp.so: argument marshalling only.
+
+torch is used for device memory and streams; every step of the path runs in
+the library's CUDA kernels.  Importing this module without a built
+``libhbp.so`` raises: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhbp.so")
+
+HBP_F32, HBP_BF16 = 0, 1
+BLOCKS = {"mlp": 0, "preln_mlp": 1, "rnn_tanh": 2, "preln_transformer": 3}
+GATE_ONE, GATE_CHANNEL_SHARED, GATE_CHANNEL_PER_STEP = 0, 1, 2
+LOSS_FINAL, LOSS_EVERY_STEP = 0, 1
+
+EXPORTS = ["hbp_workspace_bytes", "hbp_create", "hbp_forward", "hbp_backward", "hbp_exact",
+           "hbp_cumsumprod_scratch_bytes", "hbp_cumsumprod", "hbp_sync_status", "hbp_launch_count",
+           "hbp_status_string", "hbp_destroy"]
+
+
+class HbpError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = int(code)
+        super().__init__(f"{where}: hbp status {self.code} ({status_string(self.code)})")
+
+
+class hbp_config(C.Structure):
+    _fields_ = [("block", C.c_int32), ("dtype", C.c_int32), ("gate", C.c_int32), ("loss", C.c_int32),
+                ("L", C.c_int32), ("d", C.c_int32), ("hidden", C.c_int32), ("in_dim", C.c_int32),
+                ("n_heads", C.c_int32), ("head_dim", C.c_int32), ("seq", C.c_int32), ("batch", C.c_int32),
+                ("tokens", C.c_int64), ("ln_eps", C.c_float), ("reserved", C.c_int32)]
+
+
+class hbp_params(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("W1", "W2", "W", "U", "Wq", "Wk", "Wv", "Wo", "a")]
+
+
+class hbp_grads(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("dW1", "dW2", "dW", "dU", "dWq", "dWk", "dWv", "dWo", "da")]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2501_17086_b200.build` "
+                          "(the library has no fallback path)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+    lib.hbp_workspace_bytes.argtypes = [C.POINTER(hbp_config), C.POINTER(sz)]
+    lib.hbp_create.argtypes = [C.POINTER(hbp_config), vp, sz, C.POINTER(vp)]
+    lib.hbp_forward.argtypes = [vp, C.POINTER(hbp_params), vp, vp, vp, vp]
+    lib.hbp_backward.argtypes = [vp, C.POINTER(hbp_params), i32, vp, vp, vp, vp, C.POINTER(hbp_grads), vp]
+    lib.hbp_exact.argtypes = [vp, C.POINTER(hbp_params), vp, vp, vp, vp, C.POINTER(hbp_grads), vp]
+    lib.hbp_cumsumprod_scratch_bytes.argtypes = [i32, i32, i64, i32, C.POINTER(sz)]
+    lib.hbp_cumsumprod.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.hbp_sync_status.argtypes = [vp, vp]
+    lib.hbp_launch_count.argtypes = [vp]
+    lib.hbp_launch_count.restype = i64
+    lib.hbp_status_string.argtypes = [C.c_int]
+    lib.hbp_status_string.restype = C.c_char_p
+    lib.hbp_destroy.argtypes = [vp]
+    lib.hbp_destroy.restype = None
+    for name in EXPORTS:
+        if name not in ("hbp_launch_count", "hbp_status_string", "hbp_destroy"):
+            getattr(lib, name).restype = C.c_int
+    return lib
+
+
+lib = _load()
+
+
+def status_string(code: int) -> str:
+    return lib.hbp_status_string(int(code)).decode()
+
+
+def _check(code, where):
+    if code != 0:
+        raise HbpError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(dt):
+    if dt == torch.float32:
+        return HBP_F32
+    if dt == torch.bfloat16:
+        return HBP_BF16
+    raise HbpError(3, "dtype")
+
+
+def make_config(block, dtype, L, d, tokens, hidden=0, in_dim=0, n_heads=0, head_dim=0, seq=0, batch=0,
+                gate=GATE_ONE, loss=LOSS_FINAL, ln_eps=1e-5) -> hbp_config:
+    return hbp_config(BLOCKS[block], HBP_F32 if dtype in ("f32", torch.float32) else HBP_BF16, gate, loss, L, d,
+                      hidden, in_dim, n_heads, head_dim, seq, batch, tokens, ln_eps, 0)
+
+
+def config_from_workload(w) -> hbp_config:
+    """hbp_config of a ``workloads.Workload``."""
+    gate = GATE_CHANNEL_SHARED if w.block == "rnn_tanh" else GATE_ONE
+    loss = LOSS_EVERY_STEP if w.loss == "every_mse" else LOSS_FINAL
+    return make_config(w.block, w.dtype, w.L, w.d, w.tokens, w.hidden, w.in_dim, w.n_heads, w.head_dim, w.seq,
+                       w.batch, gate, loss, w.ln_eps)
+
+
+def workspace_bytes(cfg: hbp_config) -> int:
+    n = C.c_size_t(0)
+    _check(lib.hbp_workspace_bytes(C.byref(cfg), C.byref(n)), "hbp_workspace_bytes")
+    return n.value
+
+
+_GRAD_SHAPES = {
+    "mlp": lambda c: {"dW1": (c.L, c.hidden, c.d), "dW2": (c.L, c.d, c.hidden)},
+    "rnn_tanh": lambda c: {"dW": (c.d, c.d), "dU": (c.d, c.in_dim)},
+    "preln_transformer": lambda c: {"dW1": (c.L, c.hidden, c.d), "dW2": (c.L, c.d, c.hidden),
+                                    **{n: (c.L, c.d, c.d) for n in ("dWq", "dWk", "dWv", "dWo")}},
+}
+_GRAD_SHAPES["preln_mlp"] = _GRAD_SHAPES["mlp"]
+_BLOCK_NAMES = {v: k for k, v in BLOCKS.items()}
+
+
+class Context:
+    """One hbp_ctx over a torch-allocated workspace on the current CUDA device."""
+
+    def __init__(self, cfg: hbp_config, device="cuda"):
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.dtype = torch.float32 if cfg.dtype == HBP_F32 else torch.bfloat16
+        self.block = _BLOCK_NAMES[cfg.block]
+        self.steps = 2 * cfg.L if self.block == "preln_transformer" else cfg.L
+        nbytes = workspace_bytes(cfg)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        handle = C.c_void_p()
+        _check(lib.hbp_create(C.byref(cfg), C.c_void_p(base), nbytes, C.byref(handle)), "hbp_create")
+        self._h = handle
+        self._keep = None
+
+    def close(self):
+        if self._h is not None:
+            lib.hbp_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- marshalling ----------------------------------------------------
+    def _params(self, params):
+        p = hbp_params()
+        for name, _ in hbp_params._fields_:
+            t = params.get(name)
+            if t is not None:
+                assert t.is_cuda and t.is_contiguous() and t.dtype == self.dtype, name
+                setattr(p, name, t.data_ptr())
+        return p
+
+    def new_grads(self, with_gate=False):
+        c = self.cfg
+        out = {n: torch.empty(s, dtype=torch.float32, device=self.device) for n, s in _GRAD_SHAPES[self.block](c).items()}
+        if with_gate and c.gate != GATE_ONE:
+            out["da"] = torch.empty((c.d,) if c.gate == GATE_CHANNEL_SHARED else (self.steps, c.d),
+                                    dtype=torch.float32, device=self.device)
+        return out
+
+    def _grads(self, grads):
+        if grads is None:
+            return None
+        g = hbp_grads()
+        for name, t in grads.items():
+            assert t.is_cuda and t.is_contiguous() and t.dtype == torch.float32, name
+            setattr(g, name, t.data_ptr())
+        return C.byref(g)
+
+    def new_states(self):
+        return torch.empty((self.steps + 1, self.cfg.tokens, self.cfg.d), dtype=self.dtype, device=self.device)
+
+    # -- the three calls --------------------------------------------------
+    def forward(self, params, x0, inputs=None, x_all=None):
+        x_all = self.new_states() if x_all is None else x_all
+        p = self._params(params)
+        _check(lib.hbp_forward(self._h, C.byref(p), _ptr(x0), _ptr(inputs), _ptr(x_all), _stream()), "hbp_forward")
+        return x_all
+
+    def backward(self, params, k, delta, x_all, inputs=None, g_all=None, grads=None):
+        g_all = self.new_states() if g_all is None else g_all
+        p = self._params(params)
+        _check(lib.hbp_backward(self._h, C.byref(p), int(k), _ptr(delta), _ptr(x_all), _ptr(inputs), _ptr(g_all),
+                                self._grads(grads), _stream()), "hbp_backward")
+        return g_all
+
+    def exact(self, params, delta, x_all, inputs=None, g_all=None, grads=None):
+        g_all = self.new_states() if g_all is None else g_all
+        p = self._params(params)
+        _check(lib.hbp_exact(self._h, C.byref(p), _ptr(delta), _ptr(x_all), _ptr(inputs), _ptr(g_all),
+                             self._grads(grads), _stream()), "hbp_exact")
+        return g_all
+
+    def sync_status(self):
+        _check(lib.hbp_sync_status(self._h, _stream()), "hbp_sync_status")
+
+    @property
+    def launches(self) -> int:
+        return int(lib.hbp_launch_count(self._h))
+
+
+def cumsumprod_scratch_bytes(dtype, L, rows, d) -> int:
+    n = C.c_size_t(0)
+    _check(lib.hbp_cumsumprod_scratch_bytes(_dtype_code(dtype), L, rows, d, C.byref(n)), "hbp_cumsumprod_scratch_bytes")
+    return n.value
+
+
+def cumsumprod(u, delta, a=None, gate=None, loss=LOSS_FINAL, g=None, scratch=None):
+    """g[L] = delta_L, g[l] = delta_l + a_l * g[l+1] + u[l]; u is [L, rows, d] (or None with ``g`` given)."""
+    ref = u if u is not None else g
+    L = ref.shape[0] - (0 if u is not None else 1)
+    rows, d = ref.shape[1], ref.shape[2]
+    if gate is None:
+        gate = GATE_ONE if a is None else (GATE_CHANNEL_SHARED if a.dim() == 1 else GATE_CHANNEL_PER_STEP)
+    if g is None:
+        g = torch.empty((L + 1, rows, d), dtype=ref.dtype, device=ref.device)
+    need = cumsumprod_scratch_bytes(ref.dtype, L, rows, d)
+    if scratch is None and need:
+        scratch = torch.empty(need, dtype=torch.uint8, device=ref.device)
+    _check(lib.hbp_cumsumprod(_dtype_code(ref.dtype), gate, loss, L, rows, d, _ptr(u), _ptr(delta), _ptr(a), _ptr(g),
+                              _ptr(scratch), 0 if scratch is None else scratch.numel(), _stream()), "hbp_cumsumprod")
+    return g
