@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhbp.so")
-SOURCES = ["hbp_api.cu", "gemm_simt.cu", "gemm_tc.cu", "scan.cu", "attention.cu"]
+SOURCES = ["hbp_api.cu", "gemm_simt.cu", "gemm_tc.cu", "scan.cu", "attention.cu", "rnn.cu"]
 
 
 def _stale() -> bool:
@@ -46,7 +46,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
             failed = True
     if failed:
         raise RuntimeError("nvcc failed")
-    subprocess.check_call([nvcc, "-shared", "-o", LIB] + objs + ["-lcudart"])
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB] + objs + ["-lcudart"])
     return LIB
 
 

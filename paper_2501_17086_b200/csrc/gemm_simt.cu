@@ -10,10 +10,7 @@ namespace {
 template <typename T>
 __device__ __forceinline__ float load_a(const T* A, const T* A2, int64_t off) {
   float v = to_f(A[off]);
-  if (A2) {
-    float c = to_f(A2[off]);
-    v *= (1.0f - c * c);
-  }
+  if (A2) v *= to_f(A2[off]);
   return v;
 }
 
@@ -50,9 +47,11 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int b, int m, 
     case EPI_RNN_FWD: {
       float gate = g.gate ? to_f(((const T*)g.gate)[b * g.gate_sb + n]) : 1.0f;
       float z = acc + to_f(((const T*)g.E)[b * g.e_sb + (int64_t)m * g.lde + n]);
-      float c = tanhf(z);
+      // tanh and its derivative 1 - tanh^2 = 4e / (1 + e)^2 with e = exp(-2|z|): no cancellation near |c| = 1
+      float e = expf(-2.0f * fabsf(z));
+      float c = copysignf((1.0f - e) / (1.0f + e), z);
       float h = to_f(((const T*)g.E2)[b * g.e2_sb + (int64_t)m * g.lde2 + n]);
-      ((T*)g.D2)[b * g.d2_sb + (int64_t)m * g.ldd2 + n] = from_f<T>(c);
+      ((T*)g.D2)[b * g.d2_sb + (int64_t)m * g.ldd2 + n] = from_f<T>(4.0f * e / ((1.0f + e) * (1.0f + e)));
       ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(gate * h + c);
     } break;
   }

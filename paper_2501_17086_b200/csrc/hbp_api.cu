@@ -35,10 +35,11 @@ struct hbp_ctx {
   float* rstd = nullptr;   // [steps][N]
   char* Z = nullptr;       // [layers][N][h] MLP pre-activations
   float* xres = nullptr;   // [N][d] float master of the residual stream (bf16 only)
+  double* hres = nullptr;  // RNN: 2 x [B][d] double master of the recurrent state (ping-pong)
   char* U = nullptr;       // [steps][N][d] block VJP outputs (dY before the LayerNorm finish)
   char* H1 = nullptr;      // [group][N][h] dZ
   char* H2 = nullptr;      // [group][N][h] gelu(Z)
-  char* C = nullptr;       // RNN: [T][B][d] tanh outputs
+  char* C = nullptr;       // RNN: [T][B][d] tanh'(z_t) = 1 - tanh(z_t)^2
   char* scan_scratch = nullptr;
   size_t scan_scratch_bytes = 0;
   float* partial = nullptr;  // split-K / gate-gradient partial sums
@@ -107,6 +108,7 @@ size_t carve(hbp_ctx* c, char* base) {
   c->partial_floats = (size_t)kGateBlocks * d;
   if (f.block == HBP_BLOCK_RNN_TANH) {
     c->C = take(steps * N * d * es);
+    c->hres = (double*)take(2 * N * d * 8);
     c->scan_scratch_bytes = scan_scratch_bytes(f.dtype, f.L, f.tokens, f.d);
     c->scan_scratch = take(c->scan_scratch_bytes);
     const size_t wmax = d * (d > (size_t)f.in_dim ? d : (size_t)f.in_dim);
@@ -273,7 +275,7 @@ struct Run {
   }
 
   // ---- RNN ---------------------------------------------------------------------------------------
-  // u_t = (g_{t+1} * (1 - c_t^2)) W for every t at once (one GEMM over T*B rows)
+  // u_t = (g_{t+1} * tanh'(z_t)) W for every t at once (one GEMM over T*B rows)
   void rnn_vjp_all() {
     const int T = c->cfg.L;
     GemmArgs a = base_args();
@@ -439,24 +441,13 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
 
   if (f.block == HBP_BLOCK_RNN_TANH) {
     const int T = f.L;
-    GemmArgs a = r.base_args();  // input projection for every t at once
-    a.M = (int)(T * N); a.N = (int)d; a.K = f.in_dim;
-    a.A = inputs; a.a_sm = f.in_dim; a.a_sk = 1;
-    a.B = params->U; a.b_sn = f.in_dim; a.b_sk = 1;
-    a.epi = EPI_STORE; a.D = ctx->C; a.ldd = d;
-    r.run_gemm(a);
+    convert_to_f64(r.lc, f.dtype, x0, ctx->hres, state);
     for (int t = 0; t < T; ++t) {
-      GemmArgs s = r.base_args();
-      s.M = (int)N; s.N = (int)d; s.K = (int)d;
-      s.A = r.at(xa, (int64_t)t * state); s.a_sm = d; s.a_sk = 1;
-      s.B = params->W; s.b_sn = d; s.b_sk = 1;
-      s.epi = EPI_RNN_FWD;
-      s.E = r.at(ctx->C, (int64_t)t * state); s.lde = d;
-      s.E2 = r.at(xa, (int64_t)t * state); s.lde2 = d;
-      s.gate = r.gate_ptr(t);
-      s.D2 = r.at(ctx->C, (int64_t)t * state); s.ldd2 = d;
-      s.D = r.at(xa, (int64_t)(t + 1) * state); s.ldd = d;
-      r.run_gemm(s);
+      const double* hin = ctx->hres + (int64_t)(t & 1) * state;
+      double* hout = ctx->hres + (int64_t)((t + 1) & 1) * state;
+      rnn_forward_step(r.lc, f.dtype, params->W, params->U, r.at(inputs, (int64_t)t * N * f.in_dim), r.gate_ptr(t), hin,
+                       hout, r.at(ctx->C, (int64_t)t * state), r.at(xa, (int64_t)(t + 1) * state), (int)N, (int)d,
+                       f.in_dim);
     }
   } else {
     const bool tr = f.block == HBP_BLOCK_PRELN_TRANSFORMER;

@@ -19,7 +19,7 @@ enum Epilogue {
   EPI_RESID = 2,     // v = gate[n] * r + acc with r = R ? R[m,n] : E[m,n];  R = v (if R);  D = v
   EPI_DGELU = 3,     // D = acc * gelu'(E[m,n]);  D2 = gelu(E[m,n]) if D2
   EPI_AFFINE = 4,    // D = (E ? E[m,n] : 0) + gate[n] * E2[m,n] + acc
-  EPI_RNN_FWD = 5,   // c = tanh(acc + E[m,n]);  D2 = c;  D = gate[n] * E2[m,n] + c
+  EPI_RNN_FWD = 5,   // c = tanh(acc + E[m,n]);  D2 = 1 - c^2;  D = gate[n] * E2[m,n] + c
 };
 
 struct GemmArgs {
@@ -27,7 +27,7 @@ struct GemmArgs {
   int in_dtype = HBP_F32;  // element type of A, A2, B, D2, E, E2, gate and of D unless d_f32
   const void* A = nullptr;
   int64_t a_sm = 0, a_sk = 0, a_sb = 0;
-  const void* A2 = nullptr;  // if set, the A operand is A * (1 - A2^2), A2 indexed like A
+  const void* A2 = nullptr;  // if set, the A operand is the elementwise product A * A2, A2 indexed like A
   const void* B = nullptr;
   int64_t b_sn = 0, b_sk = 0, b_sb = 0;
   int epi = EPI_STORE;
@@ -103,6 +103,13 @@ void convert_to_f32(Launcher& lc, int dtype, const void* src, float* dst, int64_
 void gate_grad(Launcher& lc, int dtype, const void* g, const void* x, int64_t rows_total, int d, float* da,
                float* partial, int blocks);
 void reduce_splitk(Launcher& lc, const float* partial, float* out, int splits, int64_t elems);
+
+// ---------------------------------------------------------------- RNN forward step (rnn.cu)
+// z = W h + U x_t in double from the double master state h_in; writes h_out (double), the cached
+// derivative 1 - tanh(z)^2 and the next stored state (both in dtype).
+void rnn_forward_step(Launcher& lc, int dtype, const void* W, const void* U, const void* x_t, const void* gate,
+                      const double* h_in, double* h_out, void* deriv, void* state_out, int B, int d, int in_dim);
+void convert_to_f64(Launcher& lc, int dtype, const void* src, double* dst, int64_t elems);
 
 // ---------------------------------------------------------------- attention (attention.cu)
 struct AttnArgs {

@@ -108,7 +108,7 @@ def make_inputs(cfg: Workload, device="cpu"):
         gauss = _randn(gen, (d, d), 1.0, dev).double().cpu()
         q, r = torch.linalg.qr(gauss)
         q = q * torch.sign(torch.diagonal(r)).unsqueeze(0)
-        out["W"] = (0.5 * q).to(dev).to(dt)
+        out["W"] = (0.5 * q).contiguous().to(dev).to(dt)
         out["U"] = _randn(gen, (d, nin), 1.0 / math.sqrt(nin), dev).to(dt)
         out["X"] = _randn(gen, (T, B, nin), 1.0, dev).to(dt)
         out["Y"] = _randn(gen, (T, B, d), 1.0, dev).to(dt)
