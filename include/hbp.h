@@ -147,6 +147,15 @@ hbp_status hbp_cumsumprod(int32_t dtype, int32_t gate, int32_t loss, int32_t L, 
  * error a kernel recorded (HBP_ERR_TIMEOUT when a bounded wait gave up).  The only synchronising call. */
 hbp_status hbp_sync_status(hbp_ctx* ctx, void* cuda_stream);
 
+/* Device time per phase of the path, for the backward / exact calls made while profiling is on.  CUDA
+ * events are recorded on the call's stream around each phase: the reverse scans (Eq. 9-11), the block VJPs
+ * (Eq. 8), the parameter-gradient pass (Section 4.2) and everything else.  hbp_profile_enable(ctx, 1)
+ * clears the totals; hbp_profile_read waits for the recorded events, adds them up into ms[HBP_PHASE_COUNT]
+ * and launches[HBP_PHASE_COUNT] (either may be NULL) and clears the record. */
+typedef enum { HBP_PHASE_SCAN = 0, HBP_PHASE_VJP = 1, HBP_PHASE_WGRAD = 2, HBP_PHASE_OTHER = 3, HBP_PHASE_COUNT = 4 } hbp_phase;
+hbp_status hbp_profile_enable(hbp_ctx* ctx, int32_t on);
+hbp_status hbp_profile_read(hbp_ctx* ctx, float* ms, int64_t* launches);
+
 /* Number of kernels this context has launched since creation (host counter). */
 int64_t hbp_launch_count(const hbp_ctx* ctx);
 

@@ -21,6 +21,7 @@ LOSS_FINAL, LOSS_EVERY_STEP = 0, 1
 
 EXPORTS = ["hbp_workspace_bytes", "hbp_create", "hbp_forward", "hbp_backward", "hbp_exact",
            "hbp_cumsumprod_scratch_bytes", "hbp_cumsumprod", "hbp_sync_status", "hbp_launch_count",
+           "hbp_profile_enable", "hbp_profile_read",
            "hbp_status_string", "hbp_destroy"]
 
 
@@ -59,6 +60,8 @@ def _load():
     lib.hbp_cumsumprod_scratch_bytes.argtypes = [i32, i32, i64, i32, C.POINTER(sz)]
     lib.hbp_cumsumprod.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.hbp_sync_status.argtypes = [vp, vp]
+    lib.hbp_profile_enable.argtypes = [vp, i32]
+    lib.hbp_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(i64)]
     lib.hbp_launch_count.argtypes = [vp]
     lib.hbp_launch_count.restype = i64
     lib.hbp_status_string.argtypes = [C.c_int]
@@ -210,6 +213,16 @@ class Context:
 
     def sync_status(self):
         _check(lib.hbp_sync_status(self._h, _stream()), "hbp_sync_status")
+
+    def profile_enable(self, on=True):
+        _check(lib.hbp_profile_enable(self._h, 1 if on else 0), "hbp_profile_enable")
+
+    def profile_read(self):
+        """{'scan'|'vjp'|'wgrad'|'other': (ms, launches)} since the last read; waits for the recorded events."""
+        ms = (C.c_float * 4)()
+        n = (C.c_int64 * 4)()
+        _check(lib.hbp_profile_read(self._h, ms, n), "hbp_profile_read")
+        return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(("scan", "vjp", "wgrad", "other"))}
 
     @property
     def launches(self) -> int:

@@ -1,6 +1,515 @@
-// tcgen05 / TMEM / TMA GEMM for bf16 operands (placeholder until the kernel lands: takes no problem).
+// bf16 GEMM on the 5th-generation tensor cores: tcgen05.mma with the accumulator in tensor memory,
+// operands staged in shared memory by TMA (128-byte swizzle), fused epilogues read back with tcgen05.ld.
+//
+//   D(m, n) = sum_k A(m, k) B(n, k), fp32 accumulate, batched (one launch covers all layers of a group).
+//
+// Persistent kernel, one CTA per SM, 320 threads:
+//   warp 0      TMA producer (one lane): fills a 4-stage ring of {A 128x64, B 256x64} bf16 tiles
+//   warp 1      MMA issuer (one lane): 4 x tcgen05.mma 128x256x16 per stage; owns the TMEM allocation
+//   warps 2..9  epilogue: two warps per 32-lane TMEM quarter, 128 accumulator columns each
+// The 512 TMEM columns hold two 128x256 fp32 accumulators, so the epilogue of tile i overlaps the main
+// loop of tile i+1.  Either operand may be K-major (contraction index contiguous in memory) or MN-major
+// (row/column index contiguous); both are supported natively through the matrix descriptors, so neither
+// weights nor activations are ever transposed in memory.
+//
+// Every wait on an mbarrier is bounded: after ~4 s it raises a shared abort flag, records
+// HBP_ERR_TIMEOUT in the status word, and all roles drain and leave through the common exit that
+// frees the tensor memory.
+#include <cuda.h>
+
 #include "hbp_internal.h"
 
 namespace hbp {
-bool gemm_tc(Launcher&, const GemmArgs&, int*) { return false; }
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int EPI_WARPS = 8, THREADS = 64 + 32 * EPI_WARPS;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr uint64_t WAIT_LIMIT_NS = 4000000000ull;
+
+struct TcParams {
+  int M, N, K, batch;
+  int m_tiles, n_tiles, num_tiles, k_blocks;
+  int a_mn, b_mn;  // 1: the operand is MN-major
+  int epi, d_f32;
+  void* D; int64_t ldd, d_sb;
+  void* D2; int64_t ldd2, d2_sb;
+  const void* E; int64_t lde, e_sb;
+  const void* gate; int64_t gate_sb;
+  float* R;
+  int* status;
+};
+
+// ------------------------------------------------------------------------------------------- PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if another role raised the abort flag or the time limit passed.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  uint64_t t0 = 0;
+  for (uint32_t spin = 0;; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 255u) == 255u) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        atomicExch(status, (int)HBP_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  Offsets are in 16-byte units.
+//  K-major : rows of 128 bytes (64 elements of K), 8-row groups 1024 bytes apart (stride offset).
+//  MN-major: 64 contiguous MN elements per 128-byte row, 8 rows of K per 1024-byte group (stride
+//            offset), further blocks of 64 MN elements 8192 bytes apart (leading offset).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lead_bytes, uint32_t stride_bytes) {
+  uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lead_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((stride_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;  // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;  // 128-byte swizzle
+  return d;
+}
+
+// ------------------------------------------------------------------------------------------- epilogue math
+// Phi(z) and the normal density for bf16 outputs: erf by Abramowitz & Stegun 7.1.26 (|error| < 1.5e-7),
+// sharing exp(-z^2/2) between erf and the density; the tail is formed without cancellation.
+__device__ __forceinline__ void normal_cdf_pdf(float z, float& cdf, float& pdf) {
+  const float ax = fabsf(z) * 0.70710678118654752440f;
+  const float t = __frcp_rn(fmaf(0.3275911f, ax, 1.0f));
+  const float e = __expf(-0.5f * z * z);
+  float poly = fmaf(t, 1.061405429f, -1.453152027f);
+  poly = fmaf(t, poly, 1.421413741f);
+  poly = fmaf(t, poly, -0.284496736f);
+  poly = fmaf(t, poly, 0.254829592f);
+  const float half_tail = 0.5f * poly * t * e;  // 0.5 * erfc(|z| / sqrt 2)
+  cdf = z < 0.0f ? half_tail : 1.0f - half_tail;
+  pdf = e * 0.39894228040143267794f;
+}
+
+__device__ __forceinline__ void unpack8(const uint4& raw, float* f) {
+  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 t = __bfloat1622float2(p[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+  uint4 raw;
+  __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+  return raw;
+}
+
+// One thread owns `row` and the 32 accumulator columns starting at col0.
+__device__ __forceinline__ void epilogue_chunk(const TcParams& p, int b, int row, int col0, float* v) {
+  if (row >= p.M) return;
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    const int col = col0 + 8 * g;
+    if (col >= p.N) break;  // N is a multiple of 8: groups are all-in or all-out
+    float* a = v + 8 * g;
+    const int64_t di = (int64_t)b * p.d_sb + (int64_t)row * p.ldd + col;
+    switch (p.epi) {
+      case EPI_STORE: {
+        if (p.d_f32) {
+          float4* o = reinterpret_cast<float4*>((float*)p.D + di);
+          o[0] = make_float4(a[0], a[1], a[2], a[3]);
+          o[1] = make_float4(a[4], a[5], a[6], a[7]);
+        } else {
+          *reinterpret_cast<uint4*>((bf16*)p.D + di) = pack8(a);
+        }
+      } break;
+      case EPI_GELU_FWD: {
+        *reinterpret_cast<uint4*>((bf16*)p.D + di) = pack8(a);
+        float act[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float cdf, pdf;
+          normal_cdf_pdf(a[i], cdf, pdf);
+          act[i] = a[i] * cdf;
+        }
+        *reinterpret_cast<uint4*>((bf16*)p.D2 + (int64_t)b * p.d2_sb + (int64_t)row * p.ldd2 + col) = pack8(act);
+      } break;
+      case EPI_DGELU: {
+        float z[8], dz[8], act[8];
+        unpack8(*reinterpret_cast<const uint4*>((const bf16*)p.E + (int64_t)b * p.e_sb + (int64_t)row * p.lde + col), z);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float cdf, pdf;
+          normal_cdf_pdf(z[i], cdf, pdf);
+          dz[i] = a[i] * fmaf(z[i], pdf, cdf);
+          act[i] = z[i] * cdf;
+        }
+        *reinterpret_cast<uint4*>((bf16*)p.D + di) = pack8(dz);
+        if (p.D2) *reinterpret_cast<uint4*>((bf16*)p.D2 + (int64_t)b * p.d2_sb + (int64_t)row * p.ldd2 + col) = pack8(act);
+      } break;
+      case EPI_RESID: {
+        float gt[8], r[8];
+        if (p.gate) {
+          unpack8(*reinterpret_cast<const uint4*>((const bf16*)p.gate + (int64_t)b * p.gate_sb + col), gt);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) gt[i] = 1.0f;
+        }
+        if (p.R) {
+          float4* rp = reinterpret_cast<float4*>(p.R + (int64_t)row * p.N + col);
+          const float4 r0 = rp[0], r1 = rp[1];
+          r[0] = r0.x; r[1] = r0.y; r[2] = r0.z; r[3] = r0.w;
+          r[4] = r1.x; r[5] = r1.y; r[6] = r1.z; r[7] = r1.w;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) a[i] = fmaf(gt[i], r[i], a[i]);
+          rp[0] = make_float4(a[0], a[1], a[2], a[3]);
+          rp[1] = make_float4(a[4], a[5], a[6], a[7]);
+        } else {
+          unpack8(*reinterpret_cast<const uint4*>((const bf16*)p.E + (int64_t)b * p.e_sb + (int64_t)row * p.lde + col), r);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) a[i] = fmaf(gt[i], r[i], a[i]);
+        }
+        *reinterpret_cast<uint4*>((bf16*)p.D + di) = pack8(a);
+      } break;
+      default: break;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------- kernel
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // the swizzled tiles need 1024-byte alignment
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(aligned + STAGES * STAGE_BYTES);
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty, [2S+4] drain
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * STAGES + 4);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(accf_bar(a), 1);
+      mbar_init(acce_bar(a), EPI_WARPS);
+    }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int tiles_per_batch = p.m_tiles * p.n_tiles;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t issued_mask = 0, issued_parity = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+        const int b = tile / tiles_per_batch, r = tile % tiles_per_batch;
+        const int m0 = (r % p.m_tiles) * BM, n0 = (r / p.m_tiles) * BN;
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t sA = base + stage * STAGE_BYTES, sB = sA + A_BYTES;
+          const uint32_t fb = full_bar(stage);
+          mbar_expect_tx(fb, STAGE_BYTES);
+          issued_mask |= 1u << stage;
+          issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+          const int k0 = kb * BK;
+          if (p.a_mn) {
+#pragma unroll
+            for (int i = 0; i < BM / 64; ++i) tma_load_3d(sA + i * 8192, &tmA, fb, m0 + 64 * i, k0, b);
+          } else {
+            tma_load_3d(sA, &tmA, fb, k0, m0, b);
+          }
+          if (p.b_mn) {
+#pragma unroll
+            for (int i = 0; i < BN / 64; ++i) tma_load_3d(sB + i * 8192, &tmB, fb, n0 + 64 * i, k0, b);
+          } else {
+            tma_load_3d(sB, &tmB, fb, k0, n0, b);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // leave no copy of ours in flight: wait (bounded) for every stage armed last
+        for (int s = 0; s < STAGES; ++s)
+          if (issued_mask & (1u << s)) {
+            uint64_t t0 = global_ns();
+            while (!mbar_try_wait(full_bar(s), (issued_parity >> s) & 1u) && global_ns() - t0 < 100000000ull) {
+            }
+          }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) /*fp32 accumulate*/ | (1u << 7) /*A bf16*/ | (1u << 10) /*B bf16*/ |
+                             ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) | ((uint32_t)(BN >> 3) << 17) |
+                             ((uint32_t)(BM >> 4) << 24);
+      const uint32_t a_step = p.a_mn ? 2048u : 32u, b_step = p.b_mn ? 2048u : 32u;  // bytes per 16 of K
+      const uint32_t a_lead = p.a_mn ? 8192u : 16u, b_lead = p.b_mn ? 8192u : 16u;
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+        if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)acc * BN;
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sA = base + stage * STAGE_BYTES, sB = sA + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t ad = make_desc(sA + k * a_step, a_lead, 1024u);
+            const uint64_t bd = make_desc(sB + k * b_step, b_lead, 1024u);
+            tc_mma(tmem_d, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(accf_bar(acc));  // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (!ok) {  // let issued MMAs finish before the tensor memory is freed
+        tc_commit(drain_bar);
+        uint64_t t0 = global_ns();
+        while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < 100000000ull) {
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int quarter = warp & 3, half = (warp - 2) >> 2;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+      const int b = tile / tiles_per_batch, r = tile % tiles_per_batch;
+      const int m0 = (r % p.m_tiles) * BM, n0 = (r / p.m_tiles) * BN;
+      if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag, p.status)) break;
+      tc_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        const int col = half * 128 + c * 32;
+        float v[32];
+        tc_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + col), v);
+        epilogue_chunk(p, b, row, n0 + col, v);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acce_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------- host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)ptr;
+  }
+  return fn;
+}
+
+// Tensor map of one operand: element (mn, k, b) at base + b*sb + mn*s_mn + k*s_k (element strides).
+bool make_map(CUtensorMap* tm, const void* base, int extent_mn, int K, int batch, int64_t s_mn, int64_t s_k,
+              int64_t s_b, bool mn_major, int box_mn) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3], strides[2];
+  cuuint32_t box[3], estr[3] = {1, 1, 1};
+  const int64_t row_stride = mn_major ? s_k : s_mn;
+  dims[0] = mn_major ? (cuuint64_t)extent_mn : (cuuint64_t)K;
+  dims[1] = mn_major ? (cuuint64_t)K : (cuuint64_t)extent_mn;
+  dims[2] = (cuuint64_t)batch;
+  strides[0] = (cuuint64_t)row_stride * 2;
+  strides[1] = batch > 1 ? (cuuint64_t)s_b * 2 : (cuuint64_t)row_stride * 2 * dims[1];
+  box[0] = 64;
+  box[1] = mn_major ? 64 : (cuuint32_t)box_mn;
+  box[2] = 1;
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+// An operand qualifies if one of its two strides is 1 and the others keep every row 16-byte aligned.
+bool operand_ok(const void* base, int64_t s_mn, int64_t s_k, int64_t s_b, int batch, bool* mn_major) {
+  if (!aligned16(base)) return false;
+  if (batch > 1 && (s_b % 8 != 0 || s_b <= 0)) return false;
+  if (s_k == 1 && s_mn % 8 == 0 && s_mn > 0) { *mn_major = false; return true; }
+  if (s_mn == 1 && s_k % 8 == 0 && s_k > 0) { *mn_major = true; return true; }
+  return false;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 1;
+  }
+  return n;
+}
+
+}  // namespace
+
+bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
+  if (g.in_dtype != HBP_BF16 || g.A2 || g.splitk > 1 || !status_word) return false;
+  if (g.M <= 0 || g.N <= 0 || g.K <= 0 || g.batch <= 0) return false;
+  if (g.N % 8 || g.K % 8) return false;
+  if (g.epi != EPI_STORE && g.epi != EPI_GELU_FWD && g.epi != EPI_DGELU && g.epi != EPI_RESID) return false;
+  bool a_mn = false, b_mn = false;
+  if (!operand_ok(g.A, g.a_sm, g.a_sk, g.a_sb, g.batch, &a_mn)) return false;
+  if (!operand_ok(g.B, g.b_sn, g.b_sk, g.b_sb, g.batch, &b_mn)) return false;
+  if (a_mn && g.M % 8) return false;
+  // epilogue operands: 16-byte vectors
+  const int dv = g.d_f32 ? 4 : 8;
+  if (!aligned16(g.D) || g.ldd % dv || g.d_sb % dv) return false;
+  if (g.D2 && (!aligned16(g.D2) || g.ldd2 % 8 || g.d2_sb % 8)) return false;
+  if (g.E && (!aligned16(g.E) || g.lde % 8 || g.e_sb % 8)) return false;
+  if (g.gate && (!aligned16(g.gate) || g.gate_sb % 8)) return false;
+  if (g.R && (!aligned16(g.R) || g.N % 4)) return false;
+  if (g.epi == EPI_GELU_FWD && !g.D2) return false;
+  if (g.epi == EPI_DGELU && !g.E) return false;
+  if (g.epi == EPI_RESID && !g.R && !g.E) return false;
+
+  CUtensorMap tmA, tmB;
+  if (!make_map(&tmA, g.A, g.M, g.K, g.batch, g.a_sm, g.a_sk, g.a_sb, a_mn, BM)) return false;
+  if (!make_map(&tmB, g.B, g.N, g.K, g.batch, g.b_sn, g.b_sk, g.b_sb, b_mn, BN)) return false;
+
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    attr_set = true;
+  }
+  TcParams p;
+  p.M = g.M; p.N = g.N; p.K = g.K; p.batch = g.batch;
+  p.m_tiles = (g.M + BM - 1) / BM;
+  p.n_tiles = (g.N + BN - 1) / BN;
+  p.num_tiles = p.m_tiles * p.n_tiles * g.batch;
+  p.k_blocks = (g.K + BK - 1) / BK;
+  p.a_mn = a_mn; p.b_mn = b_mn;
+  p.epi = g.epi; p.d_f32 = g.d_f32;
+  p.D = g.D; p.ldd = g.ldd; p.d_sb = g.d_sb;
+  p.D2 = g.D2; p.ldd2 = g.ldd2; p.d2_sb = g.d2_sb;
+  p.E = g.E; p.lde = g.lde; p.e_sb = g.e_sb;
+  p.gate = g.gate; p.gate_sb = g.gate_sb;
+  p.R = g.R;
+  p.status = status_word;
+  const int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
+  gemm_tc_kernel<<<grid, THREADS, SMEM_BYTES, lc.stream>>>(tmA, tmB, p);
+  lc.count();
+  lc.check();
+  return true;
+}
+
 }  // namespace hbp

@@ -4,6 +4,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "hbp_internal.h"
 
@@ -18,8 +19,17 @@ void gemm(Launcher& lc, const GemmArgs& g, int* status_word) {
 
 using namespace hbp;
 
+struct ProfSeg {
+  cudaEvent_t beg, end;
+  int phase;
+  int64_t launches;
+};
+
 struct hbp_ctx {
   hbp_config cfg;
+  bool profiling = false;
+  std::vector<ProfSeg> segs;       // recorded, not yet read
+  std::vector<ProfSeg> free_segs;  // event pairs ready for reuse
   char* ws = nullptr;
   size_t ws_bytes = 0;
   bool forward_done = false;
@@ -331,6 +341,33 @@ struct Run {
   }
 };
 
+// Records a pair of events around one phase of a call while profiling is on.
+struct PhaseScope {
+  hbp_ctx* c;
+  cudaStream_t stream;
+  ProfSeg seg;
+  bool live = false;
+  int64_t launches0 = 0;
+  PhaseScope(Run& r, int phase) : c(r.c), stream(r.lc.stream) {
+    if (!c->profiling || c->segs.size() >= 8192) return;
+    if (!c->free_segs.empty()) {
+      seg = c->free_segs.back();
+      c->free_segs.pop_back();
+    } else if (cudaEventCreate(&seg.beg) != cudaSuccess || cudaEventCreate(&seg.end) != cudaSuccess) {
+      return;
+    }
+    seg.phase = phase;
+    launches0 = c->launches;
+    live = cudaEventRecord(seg.beg, stream) == cudaSuccess;
+  }
+  ~PhaseScope() {
+    if (!live) return;
+    cudaEventRecord(seg.end, stream);
+    seg.launches = c->launches - launches0;
+    c->segs.push_back(seg);
+  }
+};
+
 hbp_status check_call(hbp_ctx* ctx, const hbp_params* p, bool need_forward) {
   if (!ctx || !p) return HBP_ERR_INVALID_ARG;
   if (need_forward && !ctx->forward_done) return HBP_ERR_STATE;
@@ -411,7 +448,43 @@ hbp_status hbp_create(const hbp_config* cfg, void* workspace, size_t workspace_b
   return HBP_OK;
 }
 
-void hbp_destroy(hbp_ctx* ctx) { delete ctx; }
+void hbp_destroy(hbp_ctx* ctx) {
+  if (!ctx) return;
+  for (auto* v : {&ctx->segs, &ctx->free_segs})
+    for (ProfSeg& s : *v) {
+      cudaEventDestroy(s.beg);
+      cudaEventDestroy(s.end);
+    }
+  delete ctx;
+}
+
+hbp_status hbp_profile_enable(hbp_ctx* ctx, int32_t on) {
+  if (!ctx) return HBP_ERR_INVALID_ARG;
+  ctx->profiling = on != 0;
+  for (ProfSeg& s : ctx->segs) ctx->free_segs.push_back(s);
+  ctx->segs.clear();
+  return HBP_OK;
+}
+
+hbp_status hbp_profile_read(hbp_ctx* ctx, float* ms, int64_t* launches) {
+  if (!ctx) return HBP_ERR_INVALID_ARG;
+  float t[HBP_PHASE_COUNT] = {0, 0, 0, 0};
+  int64_t n[HBP_PHASE_COUNT] = {0, 0, 0, 0};
+  hbp_status st = HBP_OK;
+  for (ProfSeg& s : ctx->segs) {
+    float e = 0.0f;
+    if (cudaEventSynchronize(s.end) != cudaSuccess || cudaEventElapsedTime(&e, s.beg, s.end) != cudaSuccess) st = HBP_ERR_CUDA;
+    t[s.phase] += e;
+    n[s.phase] += s.launches;
+    ctx->free_segs.push_back(s);
+  }
+  ctx->segs.clear();
+  for (int i = 0; i < HBP_PHASE_COUNT; ++i) {
+    if (ms) ms[i] = t[i];
+    if (launches) launches[i] = n[i];
+  }
+  return st;
+}
 
 int64_t hbp_launch_count(const hbp_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
@@ -536,22 +609,33 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
   r.delta = (const char*)delta;
   const int steps = ctx->steps, layers = ctx->layers, grp = ctx->group;
   const bool tr = f.block == HBP_BLOCK_PRELN_TRANSFORMER, rnn = f.block == HBP_BLOCK_RNN_TANH;
-  r.set_last_state();
+  {
+    PhaseScope ph(r, HBP_PHASE_SCAN);
+    r.set_last_state();
+  }
 
   if (!exact) {
     // g^0 = CumSumProd(delta, K) (Eq. 10), then k iterations of {all-step VJP (Eq. 8); reverse scan (Eq. 9, 11)}
-    scan_reverse(r.lc, r.scan_args(0, steps, false));
+    {
+      PhaseScope ph(r, HBP_PHASE_SCAN);
+      scan_reverse(r.lc, r.scan_args(0, steps, false));
+    }
     const int iters = k < steps ? k : steps;
     for (int it = 0; it < iters; ++it) {
-      if (rnn) {
-        r.rnn_vjp_all();
-      } else {
-        for (int b0 = 0; b0 < layers; b0 += grp) r.mlp_vjp(b0, b0 + grp < layers ? b0 + grp : layers, false, true);
-        if (tr) r.attn_vjp(0, layers, true);
+      {
+        PhaseScope ph(r, HBP_PHASE_VJP);
+        if (rnn) {
+          r.rnn_vjp_all();
+        } else {
+          for (int b0 = 0; b0 < layers; b0 += grp) r.mlp_vjp(b0, b0 + grp < layers ? b0 + grp : layers, false, true);
+          if (tr) r.attn_vjp(0, layers, true);
+        }
       }
+      PhaseScope ph(r, HBP_PHASE_SCAN);
       scan_reverse(r.lc, r.scan_args(0, steps, true));
     }
     if (grads) {  // Section 4.2: parameter gradients from the final estimate
+      PhaseScope ph(r, HBP_PHASE_WGRAD);
       if (rnn) {
         r.rnn_wgrad(grads);
       } else {
@@ -569,6 +653,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
     }
   } else {
     // Section 2.2: g_l = delta_l + a_l g_{l+1} + J_l^T g_{l+1}, one step at a time
+    PhaseScope ph(r, HBP_PHASE_OTHER);
     if (rnn) {
       for (int t = steps - 1; t >= 0; --t) {
         GemmArgs a = r.base_args();
