@@ -23,8 +23,8 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int b, int m, 
       else ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(acc);
     } break;
     case EPI_GELU_FWD: {
-      ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(acc);
-      ((T*)g.D2)[b * g.d2_sb + (int64_t)m * g.ldd2 + n] = from_f<T>(gelu_f(acc));
+      ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(gelu_f(acc));
+      ((T*)g.D2)[b * g.d2_sb + (int64_t)m * g.ldd2 + n] = from_f<T>(gelu_prime_f(acc));
     } break;
     case EPI_RESID: {
       float gate = g.gate ? to_f(((const T*)g.gate)[b * g.gate_sb + n]) : 1.0f;
@@ -33,10 +33,9 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int b, int m, 
       if (g.R) g.R[(int64_t)m * g.N + n] = v;
       ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(v);
     } break;
-    case EPI_DGELU: {
-      float z = to_f(((const T*)g.E)[b * g.e_sb + (int64_t)m * g.lde + n]);
-      ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(acc * gelu_prime_f(z));
-      if (g.D2) ((T*)g.D2)[b * g.d2_sb + (int64_t)m * g.ldd2 + n] = from_f<T>(gelu_f(z));
+    case EPI_MUL: {
+      float e = to_f(((const T*)g.E)[b * g.e_sb + (int64_t)m * g.lde + n]);
+      ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(acc * e);
     } break;
     case EPI_AFFINE: {
       float gate = g.gate ? to_f(((const T*)g.gate)[b * g.gate_sb + n]) : 1.0f;

@@ -6,7 +6,9 @@
 // Persistent kernel, one CTA per SM, 320 threads:
 //   warp 0      TMA producer (one lane): fills a 4-stage ring of {A 128x64, B 256x64} bf16 tiles
 //   warp 1      MMA issuer (one lane): 4 x tcgen05.mma 128x256x16 per stage; owns the TMEM allocation
-//   warps 2..9  epilogue: two warps per 32-lane TMEM quarter, 128 accumulator columns each
+//   warps 2..9  epilogue: two warps per 32-lane TMEM quarter, 128 accumulator columns each; each warp
+//               stages 32-row chunks through a private 4 KB swizzled buffer, so every global access of
+//               the epilogue is a TMA tile copy (the cached gelu' in, the result out)
 // The 512 TMEM columns hold two 128x256 fp32 accumulators, so the epilogue of tile i overlaps the main
 // loop of tile i+1.  Either operand may be K-major (contraction index contiguous in memory) or MN-major
 // (row/column index contiguous); both are supported natively through the matrix descriptors, so neither
@@ -27,7 +29,8 @@ constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int EPI_WARPS = 8, THREADS = 64 + 32 * EPI_WARPS;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int EPI_BUF_BYTES = 4096;  // 32 rows x 128 bytes per epilogue warp
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * EPI_BUF_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr uint64_t WAIT_LIMIT_NS = 4000000000ull;
 
 struct TcParams {
@@ -91,6 +94,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
       ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(tm), "r"(src),
+               "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -163,94 +175,73 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
   return raw;
 }
 
-// One thread owns `row` and the 32 accumulator columns starting at col0.
-__device__ __forceinline__ void epilogue_chunk(const TcParams& p, int b, int row, int col0, float* v) {
+// Residual update of the forward pass, written straight from registers (not on the hot path):
+// one thread owns `row` and the 32 accumulator columns starting at col0.
+__device__ __forceinline__ void residual_chunk(const TcParams& p, int b, int row, int col0, float* v) {
   if (row >= p.M) return;
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
     const int col = col0 + 8 * g;
     if (col >= p.N) break;  // N is a multiple of 8: groups are all-in or all-out
     float* a = v + 8 * g;
-    const int64_t di = (int64_t)b * p.d_sb + (int64_t)row * p.ldd + col;
-    switch (p.epi) {
-      case EPI_STORE: {
-        if (p.d_f32) {
-          float4* o = reinterpret_cast<float4*>((float*)p.D + di);
-          o[0] = make_float4(a[0], a[1], a[2], a[3]);
-          o[1] = make_float4(a[4], a[5], a[6], a[7]);
-        } else {
-          *reinterpret_cast<uint4*>((bf16*)p.D + di) = pack8(a);
-        }
-      } break;
-      case EPI_GELU_FWD: {
-        *reinterpret_cast<uint4*>((bf16*)p.D + di) = pack8(a);
-        float act[8];
+    float gt[8], r[8];
+    if (p.gate) {
+      unpack8(*reinterpret_cast<const uint4*>((const bf16*)p.gate + (int64_t)b * p.gate_sb + col), gt);
+    } else {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          float cdf, pdf;
-          normal_cdf_pdf(a[i], cdf, pdf);
-          act[i] = a[i] * cdf;
-        }
-        *reinterpret_cast<uint4*>((bf16*)p.D2 + (int64_t)b * p.d2_sb + (int64_t)row * p.ldd2 + col) = pack8(act);
-      } break;
-      case EPI_DGELU: {
-        float z[8], dz[8], act[8];
-        unpack8(*reinterpret_cast<const uint4*>((const bf16*)p.E + (int64_t)b * p.e_sb + (int64_t)row * p.lde + col), z);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          float cdf, pdf;
-          normal_cdf_pdf(z[i], cdf, pdf);
-          dz[i] = a[i] * fmaf(z[i], pdf, cdf);
-          act[i] = z[i] * cdf;
-        }
-        *reinterpret_cast<uint4*>((bf16*)p.D + di) = pack8(dz);
-        if (p.D2) *reinterpret_cast<uint4*>((bf16*)p.D2 + (int64_t)b * p.d2_sb + (int64_t)row * p.ldd2 + col) = pack8(act);
-      } break;
-      case EPI_RESID: {
-        float gt[8], r[8];
-        if (p.gate) {
-          unpack8(*reinterpret_cast<const uint4*>((const bf16*)p.gate + (int64_t)b * p.gate_sb + col), gt);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) gt[i] = 1.0f;
-        }
-        if (p.R) {
-          float4* rp = reinterpret_cast<float4*>(p.R + (int64_t)row * p.N + col);
-          const float4 r0 = rp[0], r1 = rp[1];
-          r[0] = r0.x; r[1] = r0.y; r[2] = r0.z; r[3] = r0.w;
-          r[4] = r1.x; r[5] = r1.y; r[6] = r1.z; r[7] = r1.w;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) a[i] = fmaf(gt[i], r[i], a[i]);
-          rp[0] = make_float4(a[0], a[1], a[2], a[3]);
-          rp[1] = make_float4(a[4], a[5], a[6], a[7]);
-        } else {
-          unpack8(*reinterpret_cast<const uint4*>((const bf16*)p.E + (int64_t)b * p.e_sb + (int64_t)row * p.lde + col), r);
-#pragma unroll
-          for (int i = 0; i < 8; ++i) a[i] = fmaf(gt[i], r[i], a[i]);
-        }
-        *reinterpret_cast<uint4*>((bf16*)p.D + di) = pack8(a);
-      } break;
-      default: break;
+      for (int i = 0; i < 8; ++i) gt[i] = 1.0f;
     }
+    if (p.R) {
+      float4* rp = reinterpret_cast<float4*>(p.R + (int64_t)row * p.N + col);
+      const float4 r0 = rp[0], r1 = rp[1];
+      r[0] = r0.x; r[1] = r0.y; r[2] = r0.z; r[3] = r0.w;
+      r[4] = r1.x; r[5] = r1.y; r[6] = r1.z; r[7] = r1.w;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) a[i] = fmaf(gt[i], r[i], a[i]);
+      rp[0] = make_float4(a[0], a[1], a[2], a[3]);
+      rp[1] = make_float4(a[4], a[5], a[6], a[7]);
+    } else {
+      unpack8(*reinterpret_cast<const uint4*>((const bf16*)p.E + (int64_t)b * p.e_sb + (int64_t)row * p.lde + col), r);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) a[i] = fmaf(gt[i], r[i], a[i]);
+    }
+    *reinterpret_cast<uint4*>((bf16*)p.D + (int64_t)b * p.d_sb + (int64_t)row * p.ldd + col) = pack8(a);
   }
+}
+
+// Address of 16-byte unit `u` of row `r` in a 32-row x 128-byte buffer laid out with the 128-byte swizzle
+// the tensor maps use: conflict-free for one-row-per-lane access.
+__device__ __forceinline__ uint32_t swz(uint32_t buf, int r, int u) { return buf + r * 128 + ((u ^ (r & 7)) << 4); }
+__device__ __forceinline__ void st_shared16(uint32_t addr, const uint4& v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 ld_shared16(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
 }
 
 // ------------------------------------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmD2,
+               const __grid_constant__ CUtensorMap tmE, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   // the swizzled tiles need 1024-byte alignment
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(aligned + STAGES * STAGE_BYTES);
-  // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty, [2S+4] drain
+  const uint32_t epi_base = base + STAGES * STAGE_BYTES;  // EPI_WARPS x 4 KB, each 1024-byte aligned
+  uint64_t* bars = reinterpret_cast<uint64_t*>(aligned + STAGES * STAGE_BYTES + EPI_WARPS * EPI_BUF_BYTES);
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty, [2S+4] drain,
+  // [2S+5 .. 2S+5+EPI_WARPS) one per epilogue warp for its staged operand loads
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
   auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
   auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
   const uint32_t drain_bar = bar0 + 8u * (2 * STAGES + 4);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5);
+  auto epi_bar = [&](int w) { return bar0 + 8u * (2 * STAGES + 5 + w); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5 + EPI_WARPS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -264,6 +255,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(acce_bar(a), EPI_WARPS);
     }
     mbar_init(drain_bar, 1);
+    for (int w = 0; w < EPI_WARPS; ++w) mbar_init(epi_bar(w), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -364,26 +356,117 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else {
     // ------------------------------------------------------------------ epilogue
-    const int quarter = warp & 3, half = (warp - 2) >> 2;
+    const int quarter = warp & 3, half = (warp - 2) >> 2, ew = warp - 2;
+    const uint32_t buf = epi_base + ew * EPI_BUF_BYTES;
+    const uint32_t ebar = epi_bar(ew);
+    uint32_t e_phase = 0;
+    bool e_pending = false;  // lane 0: a staged operand load is in flight
     int acc = 0;
     uint32_t acc_phase = 0;
+    const bool staged = p.epi != EPI_RESID;
+    const bool has_e = p.epi == EPI_MUL;
+    const int cw = p.d_f32 ? 32 : 64;      // accumulator columns per staged chunk (128 bytes of output per row)
+    const int nchunks = 128 / cw;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       const int b = tile / tiles_per_batch, r = tile % tiles_per_batch;
       const int m0 = (r % p.m_tiles) * BM, n0 = (r / p.m_tiles) * BN;
+      const int row0 = m0 + quarter * 32, colw = n0 + half * 128;
+      if (has_e && lane == 0) {  // the buffer is free here: fetch the first chunk of E while the MMAs still run
+        mbar_expect_tx(ebar, EPI_BUF_BYTES);
+        tma_load_3d(buf, &tmE, ebar, colw, row0, b);
+        e_pending = true;
+      }
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag, p.status)) break;
       tc_fence_after();
-      const int row = m0 + quarter * 32 + lane;
+      const uint32_t tsrc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + half * 128);
+      if (!staged) {
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        const int col = half * 128 + c * 32;
-        float v[32];
-        tc_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + col), v);
-        epilogue_chunk(p, b, row, n0 + col, v);
+        for (int c = 0; c < 4; ++c) {
+          float v[32];
+          tc_ld32(tsrc + c * 32, v);
+          residual_chunk(p, b, row0 + lane, colw + c * 32, v);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce_bar(acc));
+      } else {
+        bool ok = true;
+#pragma unroll 1
+        for (int c = 0; c < nchunks; ++c) {
+          float v[64];
+          tc_ld32(tsrc + c * cw, v);
+          if (!p.d_f32) tc_ld32(tsrc + c * cw + 32, v + 32);
+          if (c == nchunks - 1) {  // last read of this accumulator: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce_bar(acc));
+          }
+          const int col = colw + c * cw;
+          if (has_e) {
+            if (!mbar_wait(ebar, e_phase, abort_flag, p.status)) { ok = false; break; }
+            e_phase ^= 1u;
+            e_pending = false;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              float e[8];
+              unpack8(ld_shared16(swz(buf, lane, u)), e);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) v[8 * u + i] *= e[i];
+            }
+          }
+          if (p.d_f32) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+              st_shared16(swz(buf, lane, u), make_uint4(__float_as_uint(v[4 * u]), __float_as_uint(v[4 * u + 1]),
+                                                        __float_as_uint(v[4 * u + 2]), __float_as_uint(v[4 * u + 3])));
+          } else if (p.epi == EPI_GELU_FWD) {
+            float dv[64];
+#pragma unroll
+            for (int i = 0; i < 64; ++i) {
+              float cdf, pdf;
+              normal_cdf_pdf(v[i], cdf, pdf);
+              dv[i] = fmaf(v[i], pdf, cdf);
+              v[i] *= cdf;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) st_shared16(swz(buf, lane, u), pack8(dv + 8 * u));
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_3d(&tmD2, buf, col, row0, b);
+              tma_store_wait_read();
+            }
+            __syncwarp();
+#pragma unroll
+            for (int u = 0; u < 8; ++u) st_shared16(swz(buf, lane, u), pack8(v + 8 * u));
+          } else {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) st_shared16(swz(buf, lane, u), pack8(v + 8 * u));
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_3d(&tmD, buf, col, row0, b);
+            tma_store_wait_read();  // the buffer may be overwritten once the copy has read it
+            if (has_e && c + 1 < nchunks) {
+              mbar_expect_tx(ebar, EPI_BUF_BYTES);
+              tma_load_3d(buf, &tmE, ebar, col + cw, row0, b);
+              e_pending = true;
+            }
+          }
+          __syncwarp();
+        }
+        if (!ok) break;
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acce_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+    if (lane == 0) {
+      tma_store_wait_all();
+      if (e_pending) {  // only after an abort: do not leave with a copy into our buffer in flight
+        uint64_t t0 = global_ns();
+        while (!mbar_try_wait(ebar, e_phase) && global_ns() - t0 < 100000000ull) {
+        }
+      }
     }
   }
 
@@ -435,6 +518,20 @@ bool make_map(CUtensorMap* tm, const void* base, int extent_mn, int K, int batch
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of an epilogue operand [batch][M][N] (leading dimension ld, batch stride sb, in elements):
+// boxes of 32 rows x 128 bytes, the chunk one epilogue warp stages.
+bool make_map_epi(CUtensorMap* tm, const void* base, bool f32, int M, int N, int batch, int64_t ld, int64_t sb) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t es = f32 ? 4 : 2;
+  cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)M, (cuuint64_t)batch};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * es, batch > 1 ? (cuuint64_t)sb * es : (cuuint64_t)ld * es * (cuuint64_t)M};
+  cuuint32_t box[3] = {f32 ? 32u : 64u, 32u, 1u}, estr[3] = {1, 1, 1};
+  return fn(tm, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 // An operand qualifies if one of its two strides is 1 and the others keep every row 16-byte aligned.
@@ -463,7 +560,8 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   if (g.in_dtype != HBP_BF16 || g.A2 || g.splitk > 1 || !status_word) return false;
   if (g.M <= 0 || g.N <= 0 || g.K <= 0 || g.batch <= 0) return false;
   if (g.N % 8 || g.K % 8) return false;
-  if (g.epi != EPI_STORE && g.epi != EPI_GELU_FWD && g.epi != EPI_DGELU && g.epi != EPI_RESID) return false;
+  if (g.epi != EPI_STORE && g.epi != EPI_GELU_FWD && g.epi != EPI_MUL && g.epi != EPI_RESID) return false;
+  if (g.d_f32 && g.epi != EPI_STORE) return false;
   bool a_mn = false, b_mn = false;
   if (!operand_ok(g.A, g.a_sm, g.a_sk, g.a_sb, g.batch, &a_mn)) return false;
   if (!operand_ok(g.B, g.b_sn, g.b_sk, g.b_sb, g.batch, &b_mn)) return false;
@@ -476,12 +574,20 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   if (g.gate && (!aligned16(g.gate) || g.gate_sb % 8)) return false;
   if (g.R && (!aligned16(g.R) || g.N % 4)) return false;
   if (g.epi == EPI_GELU_FWD && !g.D2) return false;
-  if (g.epi == EPI_DGELU && !g.E) return false;
+  if (g.epi == EPI_MUL && !g.E) return false;
   if (g.epi == EPI_RESID && !g.R && !g.E) return false;
 
   CUtensorMap tmA, tmB;
   if (!make_map(&tmA, g.A, g.M, g.K, g.batch, g.a_sm, g.a_sk, g.a_sb, a_mn, BM)) return false;
   if (!make_map(&tmB, g.B, g.N, g.K, g.batch, g.b_sn, g.b_sk, g.b_sb, b_mn, BN)) return false;
+  // epilogue operands that are staged through shared memory (everything but the forward residual update)
+  CUtensorMap tmD = tmA, tmD2 = tmA, tmE = tmA;  // placeholders when unused
+  if (g.epi != EPI_RESID) {
+    if (g.batch > 1 && g.d_sb <= 0) return false;
+    if (!make_map_epi(&tmD, g.D, g.d_f32, g.M, g.N, g.batch, g.ldd, g.d_sb)) return false;
+    if (g.epi == EPI_GELU_FWD && !make_map_epi(&tmD2, g.D2, false, g.M, g.N, g.batch, g.ldd2, g.d2_sb)) return false;
+    if (g.epi == EPI_MUL && !make_map_epi(&tmE, g.E, false, g.M, g.N, g.batch, g.lde, g.e_sb)) return false;
+  }
 
   static bool attr_set = false;
   if (!attr_set) {
@@ -506,7 +612,7 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   p.R = g.R;
   p.status = status_word;
   const int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
-  gemm_tc_kernel<<<grid, THREADS, SMEM_BYTES, lc.stream>>>(tmA, tmB, p);
+  gemm_tc_kernel<<<grid, THREADS, SMEM_BYTES, lc.stream>>>(tmA, tmB, tmD, tmD2, tmE, p);
   lc.count();
   lc.check();
   return true;

@@ -43,12 +43,12 @@ struct hbp_ctx {
   int* status = nullptr;
   char* Y = nullptr;       // [steps][N][d] LayerNorm output xhat
   float* rstd = nullptr;   // [steps][N]
-  char* Z = nullptr;       // [layers][N][h] MLP pre-activations
+  char* ACT = nullptr;     // [layers][N][h] gelu(Z)
+  char* DACT = nullptr;    // [layers][N][h] gelu'(Z)
   float* xres = nullptr;   // [N][d] float master of the residual stream (bf16 only)
   double* hres = nullptr;  // RNN: 2 x [B][d] double master of the recurrent state (ping-pong)
   char* U = nullptr;       // [steps][N][d] block VJP outputs (dY before the LayerNorm finish)
   char* H1 = nullptr;      // [group][N][h] dZ
-  char* H2 = nullptr;      // [group][N][h] gelu(Z)
   char* C = nullptr;       // RNN: [T][B][d] tanh'(z_t) = 1 - tanh(z_t)^2
   char* scan_scratch = nullptr;
   size_t scan_scratch_bytes = 0;
@@ -128,14 +128,14 @@ size_t carve(hbp_ctx* c, char* base) {
       c->Y = take(steps * N * d * es);
       c->rstd = (float*)take(steps * N * 4);
     }
-    c->Z = take((size_t)c->layers * N * h * es);
+    c->ACT = take((size_t)c->layers * N * h * es);
+    c->DACT = take((size_t)c->layers * N * h * es);
     const size_t per_layer = N * h * es;
     size_t grp = ((size_t)6 << 30) / per_layer;
     if (grp < 1) grp = 1;
     if (grp > (size_t)c->layers) grp = (size_t)c->layers;
     c->group = (int)grp;
     c->H1 = take(grp * per_layer);
-    c->H2 = take(grp * per_layer);
   }
   if (f.block == HBP_BLOCK_PRELN_TRANSFORMER) {
     const size_t Lb = (size_t)f.L;
@@ -194,17 +194,16 @@ struct Run {
   }
 
   // ---- MLP block: u = J^T g for layers [b0, b1) (b1 - b0 <= group), from states g[step+1] -------
-  // dA = G W2, dZ = dA * gelu'(Z) -> H1;  dY = dZ W1 -> U[step].  want_act also writes gelu(Z) -> H2.
-  void mlp_vjp(int b0, int b1, bool want_act, bool want_dy) {
+  // dA = G W2, dZ = dA * gelu'(Z) -> H1 (cached derivative);  dY = dZ W1 -> U[step].
+  void mlp_vjp(int b0, int b1, bool want_dy) {
     const int nb = b1 - b0, ss = step_stride();
     GemmArgs a = base_args();
     a.M = (int)N; a.N = (int)h; a.K = (int)d; a.batch = nb;
     a.A = at(g, (int64_t)(mlp_step(b0) + 1) * state); a.a_sm = d; a.a_sk = 1; a.a_sb = ss * state;
     a.B = at(p->W2, (int64_t)b0 * d * h); a.b_sn = 1; a.b_sk = h; a.b_sb = d * h;
-    a.epi = EPI_DGELU;
-    a.E = at(c->Z, (int64_t)b0 * N * h); a.lde = h; a.e_sb = N * h;
+    a.epi = EPI_MUL;
+    a.E = at(c->DACT, (int64_t)b0 * N * h); a.lde = h; a.e_sb = N * h;
     a.D = c->H1; a.ldd = h; a.d_sb = N * h;
-    if (want_act) { a.D2 = c->H2; a.ldd2 = h; a.d2_sb = N * h; }
     run_gemm(a);
     if (!want_dy) return;
     GemmArgs b = base_args();
@@ -215,13 +214,13 @@ struct Run {
     b.D = at(c->U, (int64_t)mlp_step(b0) * state); b.ldd = d; b.d_sb = ss * state;
     run_gemm(b);
   }
-  // dW2 = G^T gelu(Z), dW1 = dZ^T y for layers [b0, b1); needs H1, H2 from mlp_vjp(want_act).
+  // dW2 = G^T gelu(Z), dW1 = dZ^T y for layers [b0, b1); needs dZ in H1 from mlp_vjp.
   void mlp_wgrad(int b0, int b1, const hbp_grads* gr) {
     const int nb = b1 - b0, ss = step_stride();
     GemmArgs a = base_args();
     a.M = (int)d; a.N = (int)h; a.K = (int)N; a.batch = nb;
     a.A = at(g, (int64_t)(mlp_step(b0) + 1) * state); a.a_sm = 1; a.a_sk = d; a.a_sb = ss * state;
-    a.B = c->H2; a.b_sn = 1; a.b_sk = h; a.b_sb = N * h;
+    a.B = at(c->ACT, (int64_t)b0 * N * h); a.b_sn = 1; a.b_sk = h; a.b_sb = N * h;
     a.epi = EPI_STORE; a.d_f32 = true;
     a.D = gr->dW2 + (int64_t)b0 * d * h; a.ldd = h; a.d_sb = d * h;
     run_gemm(a);
@@ -576,12 +575,12 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
       a.A = r.mlp_operand(b); a.a_sm = d; a.a_sk = 1;
       a.B = r.at(params->W1, (int64_t)b * h * d); a.b_sn = d; a.b_sk = 1;
       a.epi = EPI_GELU_FWD;
-      a.D = r.at(ctx->Z, (int64_t)b * N * h); a.ldd = h;
-      a.D2 = ctx->H2; a.ldd2 = h;
+      a.D = r.at(ctx->ACT, (int64_t)b * N * h); a.ldd = h;
+      a.D2 = r.at(ctx->DACT, (int64_t)b * N * h); a.ldd2 = h;
       r.run_gemm(a);
       GemmArgs c2 = r.base_args();
       c2.M = (int)N; c2.N = (int)d; c2.K = (int)h;
-      c2.A = ctx->H2; c2.a_sm = h; c2.a_sk = 1;
+      c2.A = r.at(ctx->ACT, (int64_t)b * N * h); c2.a_sm = h; c2.a_sk = 1;
       c2.B = r.at(params->W2, (int64_t)b * d * h); c2.b_sn = h; c2.b_sk = 1;
       resid_epilogue(c2, step);
       r.run_gemm(c2);
@@ -627,7 +626,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
         if (rnn) {
           r.rnn_vjp_all();
         } else {
-          for (int b0 = 0; b0 < layers; b0 += grp) r.mlp_vjp(b0, b0 + grp < layers ? b0 + grp : layers, false, true);
+          for (int b0 = 0; b0 < layers; b0 += grp) r.mlp_vjp(b0, b0 + grp < layers ? b0 + grp : layers, true);
           if (tr) r.attn_vjp(0, layers, true);
         }
       }
@@ -641,7 +640,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
       } else {
         for (int b0 = 0; b0 < layers; b0 += grp) {
           const int b1 = b0 + grp < layers ? b0 + grp : layers;
-          r.mlp_vjp(b0, b1, true, false);
+          r.mlp_vjp(b0, b1, false);
           r.mlp_wgrad(b0, b1, grads);
         }
         if (tr) {
@@ -673,7 +672,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
         const int b = tr ? l / 2 : l;
         const bool is_mlp = !tr || (l % 2 == 1);
         if (is_mlp) {
-          r.mlp_vjp(b, b + 1, grads != nullptr, true);
+          r.mlp_vjp(b, b + 1, true);
           if (grads) r.mlp_wgrad(b, b + 1, grads);
         } else {
           r.attn_vjp(b, b + 1, true);

@@ -15,9 +15,9 @@ typedef __nv_bfloat16 bf16;
 // A(m, k) lives at A + batch*a_sb + m*a_sm + k*a_sk (element strides), B(n, k) likewise.
 enum Epilogue {
   EPI_STORE = 0,     // D = acc
-  EPI_GELU_FWD = 1,  // D = acc (pre-activation Z), D2 = gelu(acc)
+  EPI_GELU_FWD = 1,  // D = gelu(acc), D2 = gelu'(acc): the two activation caches of the MLP block
   EPI_RESID = 2,     // v = gate[n] * r + acc with r = R ? R[m,n] : E[m,n];  R = v (if R);  D = v
-  EPI_DGELU = 3,     // D = acc * gelu'(E[m,n]);  D2 = gelu(E[m,n]) if D2
+  EPI_MUL = 3,       // D = acc * E[m,n]   (dZ = dA * gelu'(Z) with the cached derivative)
   EPI_AFFINE = 4,    // D = (E ? E[m,n] : 0) + gate[n] * E2[m,n] + acc
   EPI_RNN_FWD = 5,   // c = tanh(acc + E[m,n]);  D2 = 1 - c^2;  D = gate[n] * E2[m,n] + c
 };
