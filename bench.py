@@ -260,8 +260,8 @@ def run_ours(args):
     hbm = peaks.get("hbm_gbs", 6650.0)
     scan_iter_ms = None
     if kk > 0 and scan_ms > 0:
-        # the first scan of a call (g^0) has no u: count the k full scans at their share
-        scan_iter_ms = scan_ms / args.steps / (kk + 0.5)
+        # the scan phase holds exactly the k scans of the iterations (g^0 is booked under "other")
+        scan_iter_ms = scan_ms / args.steps / kk
     scan_roof = {"bound": "hbm", "kernel": "scan_depth_ln_kernel" if tensors >= 3 and w.loss != "every_mse" else "scan kernels",
                  "achieved": (scan_bytes / (scan_iter_ms * 1e-3) / 1e9) if scan_iter_ms else None, "peak": hbm, "unit": "GB/s",
                  "bytes_per_scan": scan_bytes, "tensors_counted": tensors, "traffic": None}

@@ -18,6 +18,7 @@ template <typename T>
 __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int b, int m, int n, float acc) {
   const int64_t dn = (int64_t)m * g.ldd + n;
   switch (g.epi) {
+    case EPI_STORE_LN:
     case EPI_STORE: {
       if (g.d_f32) ((float*)g.D)[b * g.d_sb + dn] = acc;
       else ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(acc);

@@ -43,6 +43,7 @@ struct TcParams {
   const void* E; int64_t lde, e_sb;
   const void* gate; int64_t gate_sb;
   float* R;
+  float2* stats; int64_t stats_sb;
   int* status;
 };
 
@@ -364,7 +365,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     int acc = 0;
     uint32_t acc_phase = 0;
     const bool staged = p.epi != EPI_RESID;
-    const bool has_e = p.epi == EPI_MUL;
+    const bool has_e = p.epi == EPI_MUL || p.epi == EPI_STORE_LN;
     const int cw = p.d_f32 ? 32 : 64;      // accumulator columns per staged chunk (128 bytes of output per row)
     const int nchunks = 128 / cw;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
@@ -391,6 +392,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) mbar_arrive(acce_bar(acc));
       } else {
         bool ok = true;
+        float s1 = 0.0f, s2 = 0.0f;  // EPI_STORE_LN: row sums of acc and acc * E over this warp's 128 columns
 #pragma unroll 1
         for (int c = 0; c < nchunks; ++c) {
           float v[64];
@@ -410,8 +412,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int u = 0; u < 8; ++u) {
               float e[8];
               unpack8(ld_shared16(swz(buf, lane, u)), e);
+              if (p.epi == EPI_MUL) {
 #pragma unroll
-              for (int i = 0; i < 8; ++i) v[8 * u + i] *= e[i];
+                for (int i = 0; i < 8; ++i) v[8 * u + i] *= e[i];
+              } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  s1 += v[8 * u + i];
+                  s2 = fmaf(v[8 * u + i], e[i], s2);
+                }
+              }
             }
           }
           if (p.d_f32) {
@@ -457,6 +467,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           __syncwarp();
         }
         if (!ok) break;
+        if (p.epi == EPI_STORE_LN && row0 + lane < p.M)
+          p.stats[(int64_t)b * p.stats_sb + (int64_t)(row0 + lane) * (2 * p.n_tiles) + 2 * (n0 / BN) + half] =
+              make_float2(s1, s2);
       }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
@@ -556,11 +569,15 @@ int sm_count() {
 
 }  // namespace
 
+int gemm_tc_stats_slots(int N) { return 2 * ((N + BN - 1) / BN); }
+
 bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   if (g.in_dtype != HBP_BF16 || g.A2 || g.splitk > 1 || !status_word) return false;
   if (g.M <= 0 || g.N <= 0 || g.K <= 0 || g.batch <= 0) return false;
   if (g.N % 8 || g.K % 8) return false;
-  if (g.epi != EPI_STORE && g.epi != EPI_GELU_FWD && g.epi != EPI_MUL && g.epi != EPI_RESID) return false;
+  if (g.epi != EPI_STORE && g.epi != EPI_GELU_FWD && g.epi != EPI_MUL && g.epi != EPI_RESID && g.epi != EPI_STORE_LN)
+    return false;
+  if (g.epi == EPI_STORE_LN && (!g.stats || !g.E)) return false;
   if (g.d_f32 && g.epi != EPI_STORE) return false;
   bool a_mn = false, b_mn = false;
   if (!operand_ok(g.A, g.a_sm, g.a_sk, g.a_sb, g.batch, &a_mn)) return false;
@@ -586,7 +603,8 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
     if (g.batch > 1 && g.d_sb <= 0) return false;
     if (!make_map_epi(&tmD, g.D, g.d_f32, g.M, g.N, g.batch, g.ldd, g.d_sb)) return false;
     if (g.epi == EPI_GELU_FWD && !make_map_epi(&tmD2, g.D2, false, g.M, g.N, g.batch, g.ldd2, g.d2_sb)) return false;
-    if (g.epi == EPI_MUL && !make_map_epi(&tmE, g.E, false, g.M, g.N, g.batch, g.lde, g.e_sb)) return false;
+    if ((g.epi == EPI_MUL || g.epi == EPI_STORE_LN) && !make_map_epi(&tmE, g.E, false, g.M, g.N, g.batch, g.lde, g.e_sb))
+      return false;
   }
 
   static bool attr_set = false;
@@ -610,6 +628,7 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   p.E = g.E; p.lde = g.lde; p.e_sb = g.e_sb;
   p.gate = g.gate; p.gate_sb = g.gate_sb;
   p.R = g.R;
+  p.stats = g.stats; p.stats_sb = g.stats_sb;
   p.status = status_word;
   const int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
   gemm_tc_kernel<<<grid, THREADS, SMEM_BYTES, lc.stream>>>(tmA, tmB, tmD, tmD2, tmE, p);

@@ -11,9 +11,10 @@
 namespace hbp {
 bool g_force_simt = false;
 
-void gemm(Launcher& lc, const GemmArgs& g, int* status_word) {
-  if (!g_force_simt && g.in_dtype == HBP_BF16 && gemm_tc(lc, g, status_word)) return;
+bool gemm(Launcher& lc, const GemmArgs& g, int* status_word) {
+  if (!g_force_simt && g.in_dtype == HBP_BF16 && gemm_tc(lc, g, status_word)) return true;
   gemm_simt(lc, g);
+  return false;
 }
 }  // namespace hbp
 
@@ -49,6 +50,9 @@ struct hbp_ctx {
   double* hres = nullptr;  // RNN: 2 x [B][d] double master of the recurrent state (ping-pong)
   char* U = nullptr;       // [steps][N][d] block VJP outputs (dY before the LayerNorm finish)
   char* H1 = nullptr;      // [group][N][h] dZ
+  float2* lnpart = nullptr;  // [steps][N][slots] partial row sums of dY and dY * xhat from the GEMM epilogue
+  float4* lnstat = nullptr;  // [steps][N] {rstd, mean dY, mean dY * xhat, 0}
+  int ln_slots = 0;
   char* C = nullptr;       // RNN: [T][B][d] tanh'(z_t) = 1 - tanh(z_t)^2
   char* scan_scratch = nullptr;
   size_t scan_scratch_bytes = 0;
@@ -127,6 +131,11 @@ size_t carve(hbp_ctx* c, char* base) {
     if (c->preln) {
       c->Y = take(steps * N * d * es);
       c->rstd = (float*)take(steps * N * 4);
+      if (f.dtype == HBP_BF16) {
+        c->ln_slots = gemm_tc_stats_slots(f.d);
+        c->lnpart = (float2*)take(steps * N * c->ln_slots * sizeof(float2));
+        c->lnstat = (float4*)take(steps * N * sizeof(float4));
+      }
     }
     c->ACT = take((size_t)c->layers * N * h * es);
     c->DACT = take((size_t)c->layers * N * h * es);
@@ -182,7 +191,8 @@ struct Run {
     a.in_dtype = c->cfg.dtype;
     return a;
   }
-  void run_gemm(const GemmArgs& a) { gemm(lc, a, c->status); }
+  bool stats_ok = true;  // every dY GEMM since the last reset also produced the LayerNorm row sums
+  bool run_gemm(const GemmArgs& a) { return gemm(lc, a, c->status); }
   hbp_status result() const { return lc.err == cudaSuccess ? HBP_OK : HBP_ERR_CUDA; }
 
   // state/step index of MLP layer b and of attention layer b
@@ -191,6 +201,15 @@ struct Run {
   // operand of W1 for layer b: LayerNorm output or the raw state
   const char* mlp_operand(int b) const {
     return c->preln ? at(c->Y, (int64_t)mlp_step(b) * state) : at(x_all, (int64_t)mlp_step(b) * state);
+  }
+
+  // Asks the dY GEMM (first step `step`, `ss` steps between batch entries) for the LayerNorm row sums too.
+  void ln_epilogue(GemmArgs& b, int step, int ss) {
+    if (!c->lnpart) return;
+    b.epi = EPI_STORE_LN;
+    b.E = at(c->Y, (int64_t)step * state); b.lde = d; b.e_sb = ss * state;
+    b.stats = c->lnpart + (int64_t)step * N * c->ln_slots;
+    b.stats_sb = (int64_t)ss * N * c->ln_slots;
   }
 
   // ---- MLP block: u = J^T g for layers [b0, b1) (b1 - b0 <= group), from states g[step+1] -------
@@ -212,7 +231,9 @@ struct Run {
     b.B = at(p->W1, (int64_t)b0 * h * d); b.b_sn = 1; b.b_sk = d; b.b_sb = h * d;
     b.epi = EPI_STORE;
     b.D = at(c->U, (int64_t)mlp_step(b0) * state); b.ldd = d; b.d_sb = ss * state;
-    run_gemm(b);
+    ln_epilogue(b, mlp_step(b0), ss);
+    const bool tc = run_gemm(b);
+    stats_ok = stats_ok && (tc || !c->lnpart);
   }
   // dW2 = G^T gelu(Z), dW1 = dZ^T y for layers [b0, b1); needs dZ in H1 from mlp_vjp.
   void mlp_wgrad(int b0, int b1, const hbp_grads* gr) {
@@ -260,7 +281,9 @@ struct Run {
     b.B = at(c->Wqkv, (int64_t)b0 * 3 * d * d); b.b_sn = 1; b.b_sk = d; b.b_sb = 3 * d * d;
     b.epi = EPI_STORE;
     b.D = at(c->U, (int64_t)(2 * b0) * state); b.ldd = d; b.d_sb = 2 * state;
-    run_gemm(b);
+    ln_epilogue(b, 2 * b0, 2);
+    const bool tc = run_gemm(b);
+    stats_ok = stats_ok && (tc || !c->lnpart);
   }
   void attn_wgrad(int b0, int b1, const hbp_grads* gr) {
     const int nb = b1 - b0;
@@ -323,6 +346,14 @@ struct Run {
     }
   }
 
+  // Reverse scan over steps [lo, hi) that adds the block VJPs in U (finishing LayerNorm-backward on the way).
+  void scan_with_u(int lo, int hi) {
+    if (c->preln && c->lnpart && stats_ok)
+      ln_stats_finish(lc, c->lnpart + (int64_t)lo * N * c->ln_slots, c->ln_slots, c->rstd + (int64_t)lo * N,
+                      c->lnstat + (int64_t)lo * N, (int64_t)(hi - lo) * N, (int)d);
+    scan_reverse(lc, scan_args(lo, hi, true));
+    stats_ok = true;
+  }
   ScanArgs scan_args(int lo, int hi, bool with_u) const {
     ScanArgs s;
     s.dtype = c->cfg.dtype; s.L = c->steps; s.l_lo = lo; s.l_hi = hi; s.rows = N; s.d = (int)d;
@@ -330,7 +361,10 @@ struct Run {
     s.delta = delta; s.loss = c->cfg.loss;
     s.a = p->a; s.gate = c->cfg.gate;
     s.g = g;
-    if (with_u && c->preln) { s.xhat = c->Y; s.rstd = c->rstd; }
+    if (with_u && c->preln) {
+      s.xhat = c->Y; s.rstd = c->rstd;
+      if (c->lnpart && stats_ok) s.lnstat = c->lnstat;
+    }
     s.scratch = c->scan_scratch; s.scratch_bytes = c->scan_scratch_bytes;
     return s;
   }
@@ -609,14 +643,14 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
   const int steps = ctx->steps, layers = ctx->layers, grp = ctx->group;
   const bool tr = f.block == HBP_BLOCK_PRELN_TRANSFORMER, rnn = f.block == HBP_BLOCK_RNN_TANH;
   {
-    PhaseScope ph(r, HBP_PHASE_SCAN);
+    PhaseScope ph(r, HBP_PHASE_OTHER);
     r.set_last_state();
   }
 
   if (!exact) {
     // g^0 = CumSumProd(delta, K) (Eq. 10), then k iterations of {all-step VJP (Eq. 8); reverse scan (Eq. 9, 11)}
     {
-      PhaseScope ph(r, HBP_PHASE_SCAN);
+      PhaseScope ph(r, HBP_PHASE_OTHER);  // g^0: a scan without VJPs (a broadcast of delta_L when a = 1)
       scan_reverse(r.lc, r.scan_args(0, steps, false));
     }
     const int iters = k < steps ? k : steps;
@@ -631,7 +665,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
         }
       }
       PhaseScope ph(r, HBP_PHASE_SCAN);
-      scan_reverse(r.lc, r.scan_args(0, steps, true));
+      r.scan_with_u(0, steps);
     }
     if (grads) {  // Section 4.2: parameter gradients from the final estimate
       PhaseScope ph(r, HBP_PHASE_WGRAD);
@@ -678,7 +712,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
           r.attn_vjp(b, b + 1, true);
           if (grads) r.attn_wgrad(b, b + 1, grads);
         }
-        scan_reverse(r.lc, r.scan_args(l, l + 1, true));
+        r.scan_with_u(l, l + 1);
       }
     }
     if (grads) r.gate_grads(grads);

@@ -19,6 +19,7 @@ enum Epilogue {
   EPI_RESID = 2,     // v = gate[n] * r + acc with r = R ? R[m,n] : E[m,n];  R = v (if R);  D = v
   EPI_MUL = 3,       // D = acc * E[m,n]   (dZ = dA * gelu'(Z) with the cached derivative)
   EPI_AFFINE = 4,    // D = (E ? E[m,n] : 0) + gate[n] * E2[m,n] + acc
+  EPI_STORE_LN = 6,  // D = acc, plus per-row partial sums (sum acc, sum acc * E[m,n]) per 128 columns -> stats
   EPI_RNN_FWD = 5,   // c = tanh(acc + E[m,n]);  D2 = 1 - c^2;  D = gate[n] * E2[m,n] + c
 };
 
@@ -43,6 +44,8 @@ struct GemmArgs {
   const void* gate = nullptr;  // [N] per batch entry (stride gate_sb), nullptr = ones
   int64_t gate_sb = 0;
   float* R = nullptr;  // fp32 master copy of the residual stream [M][N], leading dim N
+  float2* stats = nullptr;  // EPI_STORE_LN: [batch][M][stats_slots] partial sums; batch stride stats_sb (in float2)
+  int64_t stats_sb = 0;
   int splitk = 1;      // > 1: partial sums to `partial` [splitk][batch][M][N], reduced in fixed order
   float* partial = nullptr;
 };
@@ -66,8 +69,11 @@ void gemm_simt(Launcher& lc, const GemmArgs& g);
 // tcgen05 / TMEM / TMA GEMM for bf16 operands; returns false if the problem does not meet its
 // alignment rules, in which case nothing was launched (gemm_tc.cu).
 bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word);
-// Picks gemm_tc when it applies, else gemm_simt.
-void gemm(Launcher& lc, const GemmArgs& g, int* status_word);
+// Picks gemm_tc when it applies, else gemm_simt (EPI_STORE_LN then degrades to EPI_STORE); returns
+// whether the tensor-core kernel ran.
+bool gemm(Launcher& lc, const GemmArgs& g, int* status_word);
+// Number of 128-column slots of partial sums the tensor-core kernel writes per row for N columns.
+int gemm_tc_stats_slots(int N);
 // Set from the environment variable HBP_FORCE_SIMT=1 when a context is created: keeps every GEMM
 // on the CUDA-core kernel (used to cross-check the tensor-core kernel).
 extern bool g_force_simt;
@@ -89,11 +95,17 @@ struct ScanArgs {
   // xhat [L][rows][d] in dtype, rstd [L][rows] float.
   const void* xhat = nullptr;
   const float* rstd = nullptr;
+  // If set, [L][rows] of {rstd, mean(dy), mean(dy*xhat), 0} prepared by ln_stats_finish: the kernel then
+  // needs no reduction of its own and streams like the plain scan.
+  const float4* lnstat = nullptr;
   void* scratch = nullptr;  // time-chunked variant only
   size_t scratch_bytes = 0;
 };
 size_t scan_scratch_bytes(int dtype, int L, int64_t rows, int d);
 void scan_reverse(Launcher& lc, const ScanArgs& s);
+// lnstat[l][row] = {rstd, sum_slots s1 / d, sum_slots s2 / d, 0} from the GEMM's partial sums.
+void ln_stats_finish(Launcher& lc, const float2* stats, int slots, const float* rstd, float4* lnstat, int64_t count,
+                     int d);
 void copy_state(Launcher& lc, int dtype, void* dst, const void* src, int64_t elems);
 // LayerNorm forward of one state: x (float master or dtype) -> xhat (dtype), rstd (float).
 void layernorm_fwd(Launcher& lc, int dtype, const void* x, bool x_is_f32, void* xhat, float* rstd, int64_t rows,

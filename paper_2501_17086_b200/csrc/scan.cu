@@ -120,6 +120,67 @@ __global__ void __launch_bounds__(256) scan_depth_kernel(const ScanArgs s) {
   }
 }
 
+// ---- depth scan with the LayerNorm-backward finish from prepared row statistics ---------------------
+// Same streaming form as above: lnstat[l][row] = {rstd, mean(dy), mean(dy * xhat)} comes from the GEMM that
+// produced dy, so no reduction is needed here.  u holds dy, the VJP is rstd * (dy - m1 - xhat * m2).
+template <typename T>
+__global__ void __launch_bounds__(256) scan_depth_lnstat_kernel(const ScanArgs s) {
+  constexpr int V = Vec<T>::N;
+  const int64_t state_elems = s.rows * s.d;
+  const int64_t nvec = state_elems / V;
+  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v >= nvec) return;
+  const int64_t off = v * V;
+  const int64_t row = off / s.d;
+  const int ch = (int)(off - row * s.d);
+  T* g = (T*)s.g;
+  float carry[V];
+  ldv<T>(g + (int64_t)s.l_hi * state_elems + off).get(carry);
+  for (int l = s.l_hi - 1; l >= s.l_lo; --l) {
+    float dy[V], xh[V], val[V];
+    ldv_stream<T>((const T*)s.u + (int64_t)l * state_elems + off).get(dy);
+    ldv_stream<T>((const T*)s.xhat + (int64_t)l * state_elems + off).get(xh);
+    const float4 st = __ldg(s.lnstat + (int64_t)l * s.rows + row);
+    const T* gp = gate_at<T>(s, l);
+    if (gp) {
+      float a[V];
+      ldv<T>(gp + ch).get(a);
+#pragma unroll
+      for (int i = 0; i < V; ++i) val[i] = a[i] * carry[i];
+    } else {
+#pragma unroll
+      for (int i = 0; i < V; ++i) val[i] = carry[i];
+    }
+#pragma unroll
+    for (int i = 0; i < V; ++i) val[i] += st.x * (dy[i] - st.y - xh[i] * st.z);
+    const T* dp = delta_at<T>(s, l, state_elems);
+    if (dp) {
+      float dl[V];
+      ldv_stream<T>(dp + off).get(dl);
+#pragma unroll
+      for (int i = 0; i < V; ++i) val[i] += dl[i];
+    }
+    Vec<T> out;
+    out.set(val);
+    stv<T>(g + (int64_t)l * state_elems + off, out);
+#pragma unroll
+    for (int i = 0; i < V; ++i) carry[i] = val[i];
+  }
+}
+
+__global__ void ln_stats_finish_kernel(const float2* __restrict__ stats, int slots, const float* __restrict__ rstd,
+                                       float4* __restrict__ lnstat, int64_t count, float inv_d) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  float s1 = 0.0f, s2 = 0.0f;
+  for (int k = 0; k < slots; ++k) {  // fixed order: deterministic
+    const float2 t = stats[i * slots + k];
+    s1 += t.x;
+    s2 += t.y;
+  }
+  lnstat[i] = make_float4(rstd[i], s1 * inv_d, s2 * inv_d, 0.0f);
+}
+
 // ---- depth scan with the LayerNorm-backward finish: one block per row ------------------------------
 // u holds dY = dL/d(LN(x)); the step's VJP is rstd * (dy - mean(dy) - xhat * mean(dy * xhat)).
 template <typename T>
@@ -369,6 +430,14 @@ void scan_reverse(Launcher& lc, const ScanArgs& s) {
   if (s.l_hi <= s.l_lo || s.rows <= 0) return;
   const int V = s.dtype == HBP_F32 ? 4 : 8;
   const int64_t nvec = s.rows * s.d / V;
+  if (s.xhat && s.lnstat) {
+    const unsigned grid = (unsigned)((nvec + 255) / 256);
+    if (s.dtype == HBP_F32) scan_depth_lnstat_kernel<float><<<grid, 256, 0, lc.stream>>>(s);
+    else scan_depth_lnstat_kernel<bf16><<<grid, 256, 0, lc.stream>>>(s);
+    lc.count();
+    lc.check();
+    return;
+  }
   if (s.xhat) {
     const int threads = row_block_threads(s.d, V);
     if (s.dtype == HBP_F32) scan_depth_ln_kernel<float><<<(unsigned)s.rows, threads, 0, lc.stream>>>(s);
@@ -401,6 +470,14 @@ void scan_reverse(Launcher& lc, const ScanArgs& s) {
   const unsigned grid = (unsigned)((nvec + 255) / 256);
   if (s.dtype == HBP_F32) scan_depth_kernel<float><<<grid, 256, 0, lc.stream>>>(s);
   else scan_depth_kernel<bf16><<<grid, 256, 0, lc.stream>>>(s);
+  lc.count();
+  lc.check();
+}
+
+void ln_stats_finish(Launcher& lc, const float2* stats, int slots, const float* rstd, float4* lnstat, int64_t count,
+                     int d) {
+  ln_stats_finish_kernel<<<(unsigned)((count + 255) / 256), 256, 0, lc.stream>>>(stats, slots, rstd, lnstat, count,
+                                                                                1.0f / (float)d);
   lc.count();
   lc.check();
 }
