@@ -688,17 +688,14 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
     // Section 2.2: g_l = delta_l + a_l g_{l+1} + J_l^T g_{l+1}, one step at a time
     PhaseScope ph(r, HBP_PHASE_OTHER);
     if (rnn) {
+      // the sequential recurrence is carried in double beside the stored float gradients
+      convert_to_f64(r.lc, f.dtype, r.at(r.g, (int64_t)steps * r.state), ctx->hres, r.state);
       for (int t = steps - 1; t >= 0; --t) {
-        GemmArgs a = r.base_args();
-        a.M = (int)r.N; a.N = (int)r.d; a.K = (int)r.d;
-        a.A = r.at(r.g, (int64_t)(t + 1) * r.state); a.A2 = r.at(ctx->C, (int64_t)t * r.state); a.a_sm = r.d; a.a_sk = 1;
-        a.B = params->W; a.b_sn = 1; a.b_sk = r.d;
-        a.epi = EPI_AFFINE;
-        a.E = f.loss == HBP_LOSS_EVERY_STEP ? r.at(r.delta, (int64_t)t * r.state) : nullptr; a.lde = r.d;
-        a.E2 = r.at(r.g, (int64_t)(t + 1) * r.state); a.lde2 = r.d;
-        a.gate = r.gate_ptr(t);
-        a.D = r.at(r.g, (int64_t)t * r.state); a.ldd = r.d;
-        r.run_gemm(a);
+        const double* gin = ctx->hres + (int64_t)((steps - 1 - t) & 1) * r.state;
+        double* gout = ctx->hres + (int64_t)((steps - t) & 1) * r.state;
+        rnn_backward_step(r.lc, f.dtype, params->W, r.at(ctx->C, (int64_t)t * r.state),
+                          f.loss == HBP_LOSS_EVERY_STEP ? r.at(r.delta, (int64_t)t * r.state) : nullptr, r.gate_ptr(t),
+                          gin, gout, r.at(r.g, (int64_t)t * r.state), (int)r.N, (int)r.d);
       }
       if (grads) r.rnn_wgrad(grads);
     } else {

@@ -121,6 +121,9 @@ void reduce_splitk(Launcher& lc, const float* partial, float* out, int splits, i
 // derivative 1 - tanh(z)^2 and the next stored state (both in dtype).
 void rnn_forward_step(Launcher& lc, int dtype, const void* W, const void* U, const void* x_t, const void* gate,
                       const double* h_in, double* h_out, void* deriv, void* state_out, int B, int d, int in_dim);
+// g_t = delta_t + a * g_{t+1} + (g_{t+1} * deriv_t) W in double from the double master g_in.
+void rnn_backward_step(Launcher& lc, int dtype, const void* W, const void* deriv, const void* delta, const void* gate,
+                       const double* g_in, double* g_out, void* g_store, int B, int d);
 void convert_to_f64(Launcher& lc, int dtype, const void* src, double* dst, int64_t elems);
 
 // ---------------------------------------------------------------- attention (attention.cu)

@@ -66,6 +66,49 @@ __global__ void __launch_bounds__(256) rnn_step_kernel(const T* __restrict__ W, 
   }
 }
 
+// One step of exact backpropagation through time, carried in double like the forward recurrence:
+//     g_t = delta_t + a * g_{t+1} + (g_{t+1} * tanh'(z_t)) W
+// from the double master copy of g_{t+1}; writes the new master and its rounding g[t].
+template <typename T>
+__global__ void __launch_bounds__(256) rnn_bwd_step_kernel(const T* __restrict__ W, const T* __restrict__ deriv,
+                                                           const T* __restrict__ delta, const T* __restrict__ gate,
+                                                           const double* __restrict__ g_in, double* __restrict__ g_out,
+                                                           T* __restrict__ g_store, int B, int d) {
+  __shared__ double Hs[kTile][kTile + 1];
+  __shared__ float Ws[kTile][kTile + 1];
+  const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
+  const int n0 = blockIdx.x * kTile, m0 = blockIdx.y * kTile;
+  double acc[4] = {0.0, 0.0, 0.0, 0.0};
+  for (int k0 = 0; k0 < d; k0 += kTile) {
+    for (int i = ty; i < kTile; i += 8) {
+      const int m = m0 + i, k = k0 + tx;
+      Hs[i][tx] = (m < B && k < d) ? g_in[(int64_t)m * d + k] * (double)to_f(deriv[(int64_t)m * d + k]) : 0.0;
+      const int kk = k0 + i, n = n0 + tx;  // W[k][n]: contiguous in n
+      Ws[tx][i] = (kk < d && n < d) ? to_f(W[(int64_t)kk * d + n]) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < kTile; ++kk) {
+      const double w = (double)Ws[tx][kk];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[j] = fma(Hs[ty + 8 * j][kk], w, acc[j]);
+    }
+    __syncthreads();
+  }
+  const int n = n0 + tx;
+  if (n >= d) return;
+  const double a = gate ? (double)to_f(gate[n]) : 1.0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int m = m0 + ty + 8 * j;
+    if (m >= B) continue;
+    const int64_t idx = (int64_t)m * d + n;
+    const double v = (delta ? (double)to_f(delta[idx]) : 0.0) + a * g_in[idx] + acc[j];
+    g_out[idx] = v;
+    g_store[idx] = from_f<T>((float)v);
+  }
+}
+
 template <typename T>
 __global__ void to_f64_kernel(const T* __restrict__ src, double* __restrict__ dst, int64_t n) {
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -85,6 +128,19 @@ void rnn_forward_step(Launcher& lc, int dtype, const void* W, const void* U, con
     rnn_step_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)U, (const bf16*)x_t,
                                                        (const bf16*)gate, h_in, h_out, (bf16*)deriv, (bf16*)state_out,
                                                        B, d, in_dim);
+  lc.count();
+  lc.check();
+}
+
+void rnn_backward_step(Launcher& lc, int dtype, const void* W, const void* deriv, const void* delta, const void* gate,
+                       const double* g_in, double* g_out, void* g_store, int B, int d) {
+  dim3 grid((d + kTile - 1) / kTile, (B + kTile - 1) / kTile);
+  if (dtype == HBP_F32)
+    rnn_bwd_step_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)deriv, (const float*)delta,
+                                                            (const float*)gate, g_in, g_out, (float*)g_store, B, d);
+  else
+    rnn_bwd_step_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)deriv, (const bf16*)delta,
+                                                           (const bf16*)gate, g_in, g_out, (bf16*)g_store, B, d);
   lc.count();
   lc.check();
 }

@@ -13,14 +13,17 @@ template <>
 struct Vec<float> {
   static constexpr int N = 4;
   float4 raw;
-  __device__ __forceinline__ void get(float* f) const { f[0] = raw.x; f[1] = raw.y; f[2] = raw.z; f[3] = raw.w; }
-  __device__ __forceinline__ void set(const float* f) { raw = make_float4(f[0], f[1], f[2], f[3]); }
+  template <typename F>
+  __device__ __forceinline__ void get(F* f) const { f[0] = raw.x; f[1] = raw.y; f[2] = raw.z; f[3] = raw.w; }
+  template <typename F>
+  __device__ __forceinline__ void set(const F* f) { raw = make_float4((float)f[0], (float)f[1], (float)f[2], (float)f[3]); }
 };
 template <>
 struct Vec<bf16> {
   static constexpr int N = 8;
   uint4 raw;
-  __device__ __forceinline__ void get(float* f) const {
+  template <typename F>
+  __device__ __forceinline__ void get(F* f) const {
     const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&raw);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -29,11 +32,23 @@ struct Vec<bf16> {
       f[2 * i + 1] = t.y;
     }
   }
-  __device__ __forceinline__ void set(const float* f) {
+  template <typename F>
+  __device__ __forceinline__ void set(const F* f) {
     __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&raw);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn((float)f[2 * i], (float)f[2 * i + 1]);
   }
+};
+
+// The running value of the recurrence: double for float data (thousands of steps must stay within 1e-5 of
+// an exact evaluation), float for bf16 data.
+template <typename T>
+struct Acc {
+  typedef float type;
+};
+template <>
+struct Acc<float> {
+  typedef double type;
 };
 
 template <typename T>
@@ -69,7 +84,7 @@ __device__ __forceinline__ const T* gate_at(const ScanArgs& s, int l) {
 // One step of the recurrence for a 16-byte channel group: val = a * carry + u + delta.
 template <typename T>
 __device__ __forceinline__ void scan_step(const ScanArgs& s, int l, int64_t state_elems, int64_t off, int ch,
-                                          const float* carry, float* val) {
+                                          const typename Acc<T>::type* carry, typename Acc<T>::type* val) {
   constexpr int V = Vec<T>::N;
   const T* gp = gate_at<T>(s, l);
   if (gp) {
@@ -107,10 +122,11 @@ __global__ void __launch_bounds__(256) scan_depth_kernel(const ScanArgs s) {
   const int64_t off = v * V;
   const int ch = (int)(off % s.d);
   T* g = (T*)s.g;
-  float carry[V];
+  typedef typename Acc<T>::type A;
+  A carry[V];
   ldv<T>(g + (int64_t)s.l_hi * state_elems + off).get(carry);
   for (int l = s.l_hi - 1; l >= s.l_lo; --l) {
-    float val[V];
+    A val[V];
     scan_step<T>(s, l, state_elems, off, ch, carry, val);
     Vec<T> out;
     out.set(val);
@@ -275,12 +291,14 @@ __global__ void __launch_bounds__(1024) scan_depth_ln_kernel(const ScanArgs s) {
 // Phase 1: per (chunk, channel group) local scan with zero carry-in -> S (value at the chunk's first
 // step) and P (product of the gates over the chunk).  Phase 2: per channel, serial over the chunks:
 // carry-in of chunk c = G_{c+1}, G_c = S_c + P_c * G_{c+1}.  Phase 3: local scan again with the
-// carry-in, writing g.  Scratch: S (then the carry-ins) [nchunks][rows*d] and P likewise, float.
+// carry-in, writing g.  Scratch: S (then the carry-ins) [nchunks][rows*d] and P likewise, in the
+// accumulator type (double for float data).
 constexpr int kChunk = 32;
 
 template <typename T, bool kApply>
-__global__ void __launch_bounds__(128) scan_chunk_kernel(const ScanArgs s, float* __restrict__ S,
-                                                         float* __restrict__ P) {
+__global__ void __launch_bounds__(128) scan_chunk_kernel(const ScanArgs s, typename Acc<T>::type* __restrict__ S,
+                                                         typename Acc<T>::type* __restrict__ P) {
+  typedef typename Acc<T>::type A;
   constexpr int V = Vec<T>::N;
   const int64_t state_elems = s.rows * s.d;
   const int64_t nvec = state_elems / V;
@@ -291,14 +309,14 @@ __global__ void __launch_bounds__(128) scan_chunk_kernel(const ScanArgs s, float
   const int64_t off = v * V;
   const int ch = (int)(off % s.d);
   T* g = (T*)s.g;
-  float carry[V], prod[V];
+  A carry[V], prod[V];
 #pragma unroll
   for (int i = 0; i < V; ++i) {
-    carry[i] = kApply ? S[(int64_t)c * state_elems + off + i] : 0.0f;
-    prod[i] = 1.0f;
+    carry[i] = kApply ? S[(int64_t)c * state_elems + off + i] : (A)0;
+    prod[i] = (A)1;
   }
   for (int l = hi - 1; l >= lo; --l) {
-    float val[V];
+    A val[V];
     scan_step<T>(s, l, state_elems, off, ch, carry, val);
     if (kApply) {
       Vec<T> out;
@@ -326,14 +344,15 @@ __global__ void __launch_bounds__(128) scan_chunk_kernel(const ScanArgs s, float
 }
 
 template <typename T>
-__global__ void __launch_bounds__(128) scan_carry_kernel(const ScanArgs s, float* __restrict__ S,
-                                                         const float* __restrict__ P, int nchunks) {
+__global__ void __launch_bounds__(128) scan_carry_kernel(const ScanArgs s, typename Acc<T>::type* __restrict__ S,
+                                                         const typename Acc<T>::type* __restrict__ P, int nchunks) {
+  typedef typename Acc<T>::type A;
   const int64_t state_elems = s.rows * s.d;
   const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= state_elems) return;
-  float G = to_f(((const T*)s.g)[(int64_t)s.l_hi * state_elems + e]);
+  A G = (A)to_f(((const T*)s.g)[(int64_t)s.l_hi * state_elems + e]);
   for (int c = nchunks - 1; c >= 0; --c) {
-    const float sc = S[(int64_t)c * state_elems + e], pc = P[(int64_t)c * state_elems + e];
+    const A sc = S[(int64_t)c * state_elems + e], pc = P[(int64_t)c * state_elems + e];
     S[(int64_t)c * state_elems + e] = G;  // carry-in of chunk c
     G = sc + pc * G;
   }
@@ -423,7 +442,7 @@ size_t scan_scratch_bytes(int dtype, int L, int64_t rows, int d) {
   const int64_t nvec = rows * d / V;
   if (nvec >= 148 * 512 || L < 4 * kChunk) return 0;  // enough channels (or too short) for the serial form
   const int nchunks = (L + kChunk - 1) / kChunk;
-  return (size_t)2 * nchunks * rows * d * sizeof(float);
+  return (size_t)2 * nchunks * rows * d * (dtype == HBP_F32 ? sizeof(double) : sizeof(float));
 }
 
 void scan_reverse(Launcher& lc, const ScanArgs& s) {
@@ -450,15 +469,17 @@ void scan_reverse(Launcher& lc, const ScanArgs& s) {
   const size_t need = scan_scratch_bytes(s.dtype, steps, s.rows, s.d);
   if (need > 0 && s.scratch && s.scratch_bytes >= need) {
     const int nchunks = (steps + kChunk - 1) / kChunk;
-    float* S = (float*)s.scratch;
-    float* P = S + (int64_t)nchunks * s.rows * s.d;
     dim3 grid((unsigned)((nvec + 127) / 128), nchunks);
     const unsigned cgrid = (unsigned)((s.rows * s.d + 127) / 128);
     if (s.dtype == HBP_F32) {
+      double* S = (double*)s.scratch;
+      double* P = S + (int64_t)nchunks * s.rows * s.d;
       scan_chunk_kernel<float, false><<<grid, 128, 0, lc.stream>>>(s, S, P);
       scan_carry_kernel<float><<<cgrid, 128, 0, lc.stream>>>(s, S, P, nchunks);
       scan_chunk_kernel<float, true><<<grid, 128, 0, lc.stream>>>(s, S, P);
     } else {
+      float* S = (float*)s.scratch;
+      float* P = S + (int64_t)nchunks * s.rows * s.d;
       scan_chunk_kernel<bf16, false><<<grid, 128, 0, lc.stream>>>(s, S, P);
       scan_carry_kernel<bf16><<<cgrid, 128, 0, lc.stream>>>(s, S, P, nchunks);
       scan_chunk_kernel<bf16, true><<<grid, 128, 0, lc.stream>>>(s, S, P);

@@ -1,0 +1,82 @@
+"""Full-size workloads on the GPU, in the launch configuration the benchmark times, checked against the
+fp64 oracle on sampled independent units (tokens / sequences / batch rows): the blocks act on each unit
+independently, so the oracle run on a subset with the full weights gives exactly those rows of every g_l."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import run as orun
+from paper_2501_17086_b200.workloads import WORKLOADS, make_inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-5, "bf16": 2e-2}
+# Exact BPTT on c3 is ill-conditioned: with a in U(0.9, 0.999) plus 0.5 x orthogonal recurrent weights the step
+# Jacobian a + tanh'(z) W has growth ~1.007 per step, so ||g_0|| / ||g_T|| ~ 1e13 over 4096 steps and the float
+# rounding of the stored states (2.6e-7 between the two forward passes) is amplified through hundreds of
+# factors.  Highway-BP with k <= 8 applies at most 8 block Jacobians and keeps the 1e-5 bar; exact BPTT at the
+# full length is held to this looser bound (it meets 1e-5 on the T = 200 twin).
+TOL_EXACT_LONG_RNN = 5e-4
+
+
+def _rows_of(w, t, rows):
+    """[steps+1, N, d] -> the sampled units, shaped like the oracle's states."""
+    if w.block == "preln_transformer":
+        return t.reshape(t.shape[0], w.batch, w.seq, w.d)[:, rows]
+    return t[:, rows]
+
+
+@pytest.mark.parametrize("name,ks,rows", [
+    ("c2", (1, 2, 4, 8), [0, 1, 127, 128, 4097, 8191]),
+    ("c3", (1, 2, 4, 8), [0, 31]),
+    ("c4", (1, 2, 4), [5]),
+    ("c5", (1, 2), [0, 129, 8200, 16383]),
+])
+def test_full_size_sampled_units(name, ks, rows):
+    from paper_2501_17086_b200 import harness
+    w = WORKLOADS[name]
+    need_gb = {"c2": 30, "c3": 4, "c4": 40, "c5": 150}[name]
+    free, _ = torch.cuda.mem_get_info()
+    if free < need_gb * 2**30:
+        pytest.skip(f"needs about {need_gb} GB of free device memory")
+    inp = make_inputs(w, "cuda")
+    ctx = harness.make_context(w)
+    params = harness.params_for(w, inp)
+    xin = harness.rnn_inputs(w, inp)
+    x_all = ctx.forward(params, inp["x0"], xin)
+    delta = harness.loss_delta(w, x_all, inp)
+    rows_t = torch.tensor(rows, device="cuda")
+    got = {}
+    g_all = ctx.new_states()
+    for k in ks:
+        ctx.backward(params, k, delta, x_all, xin, g_all=g_all)
+        got[k] = _rows_of(w, g_all, rows_t).float().cpu().double().numpy()
+    grads = ctx.new_grads(with_gate=True)
+    ctx.exact(params, delta, x_all, xin, g_all=g_all, grads=grads)
+    got["exact"] = _rows_of(w, g_all, rows_t).float().cpu().double().numpy()
+    ctx.sync_status()
+    xs_gpu = _rows_of(w, x_all, rows_t).float().cpu().double().numpy()
+    for t in grads.values():
+        assert torch.isfinite(t).all()
+    del ctx, g_all, x_all, grads
+    torch.cuda.empty_cache()
+
+    ref = orun.run(w, inp, ks=ks, rows=rows_t.cpu())
+    tol = TOL[w.dtype]
+
+    def rel(a, b):
+        nb = np.linalg.norm(b)
+        return float(np.linalg.norm(a.reshape(b.shape) - b) / nb) if nb else float(np.linalg.norm(a))
+
+    worst_x = max(rel(xs_gpu[l], ref["xs"][l]) for l in range(w.steps + 1))
+    assert worst_x < tol, f"states: {worst_x:.3e}"
+    for k in ks:
+        worst = max(rel(got[k][l], ref["hbp"][k][l]) for l in range(w.steps + 1))
+        assert worst < tol, f"k={k}: max rel-L2 {worst:.3e}"
+    worst = max(rel(got["exact"][l], ref["exact"][l]) for l in range(w.steps + 1))
+    tol_exact = TOL_EXACT_LONG_RNN if name == "c3" else tol
+    assert worst < tol_exact, f"exact: max rel-L2 {worst:.3e}"
+    # tail exactness on the GPU itself (Theorem 2): g^k_l is already exact for l >= steps - k
+    kmax = max(ks)
+    for l in range(w.steps - kmax, w.steps + 1):
+        assert rel(got[kmax][l], got["exact"][l]) < tol_exact
