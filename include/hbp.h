@@ -143,6 +143,22 @@ hbp_status hbp_cumsumprod(int32_t dtype, int32_t gate, int32_t loss, int32_t L, 
                           const void* u, const void* delta, const void* a, void* g,
                           void* scratch, size_t scratch_bytes, void* cuda_stream);
 
+/* The same scan for callers that cannot allocate device memory.  (The paper has no counterpart: this is a
+ * packaging variant of hbp_cumsumprod, not a step of the method.)  Some hosts hand all device memory to
+ * their own pool at start-up, or forbid cudaMalloc/cudaFree once they are running (latency-critical loops,
+ * sandboxed plug-ins); they have no way to provide the scratch that the time-chunked scan needs.  Here the
+ * scratch is a fixed array inside the library's device image of hbp_cumsumprod_static_max_bytes() bytes
+ * (32 MiB), held by every GPU that loads the library until the process exits.  The call allocates nothing and
+ * frees nothing.  Problems whose hbp_cumsumprod_scratch_bytes(...) exceeds the fixed size are refused with
+ * HBP_ERR_WORKSPACE.  The first call on each device looks the array's device address up (a one-time set-up
+ * with that device current): make that first call before starting any stream capture.  All calls share the
+ * one array per device, so two calls whose kernels may overlap on the GPU (different streams) race on it;
+ * serialise them.  Contents left by an earlier call are harmless: the scan writes every partial result
+ * before reading it. */
+size_t hbp_cumsumprod_static_max_bytes(void);
+hbp_status hbp_cumsumprod_static(int32_t dtype, int32_t gate, int32_t loss, int32_t L, int64_t rows, int32_t d,
+                                 const void* u, const void* delta, const void* a, void* g, void* cuda_stream);
+
 /* Copies the context's device status word to the host after synchronising the stream: HBP_OK, or the
  * error a kernel recorded (HBP_ERR_TIMEOUT when a bounded wait gave up).  The only synchronising call. */
 hbp_status hbp_sync_status(hbp_ctx* ctx, void* cuda_stream);

@@ -21,7 +21,7 @@ LOSS_FINAL, LOSS_EVERY_STEP = 0, 1
 
 EXPORTS = ["hbp_workspace_bytes", "hbp_create", "hbp_forward", "hbp_backward", "hbp_exact",
            "hbp_cumsumprod_scratch_bytes", "hbp_cumsumprod", "hbp_sync_status", "hbp_launch_count",
-           "hbp_profile_enable", "hbp_profile_read",
+           "hbp_profile_enable", "hbp_profile_read", "hbp_cumsumprod_static", "hbp_cumsumprod_static_max_bytes",
            "hbp_status_string", "hbp_destroy"]
 
 
@@ -59,6 +59,8 @@ def _load():
     lib.hbp_exact.argtypes = [vp, C.POINTER(hbp_params), vp, vp, vp, vp, C.POINTER(hbp_grads), vp]
     lib.hbp_cumsumprod_scratch_bytes.argtypes = [i32, i32, i64, i32, C.POINTER(sz)]
     lib.hbp_cumsumprod.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.hbp_cumsumprod_static.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp]
+    lib.hbp_cumsumprod_static_max_bytes.argtypes = []
     lib.hbp_sync_status.argtypes = [vp, vp]
     lib.hbp_profile_enable.argtypes = [vp, i32]
     lib.hbp_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(i64)]
@@ -69,7 +71,9 @@ def _load():
     lib.hbp_destroy.argtypes = [vp]
     lib.hbp_destroy.restype = None
     for name in EXPORTS:
-        if name not in ("hbp_launch_count", "hbp_status_string", "hbp_destroy"):
+        if name == "hbp_cumsumprod_static_max_bytes":
+            lib.hbp_cumsumprod_static_max_bytes.restype = sz
+        elif name not in ("hbp_launch_count", "hbp_status_string", "hbp_destroy"):
             getattr(lib, name).restype = C.c_int
     return lib
 
@@ -249,4 +253,23 @@ def cumsumprod(u, delta, a=None, gate=None, loss=LOSS_FINAL, g=None, scratch=Non
         scratch = torch.empty(need, dtype=torch.uint8, device=ref.device)
     _check(lib.hbp_cumsumprod(_dtype_code(ref.dtype), gate, loss, L, rows, d, _ptr(u), _ptr(delta), _ptr(a), _ptr(g),
                               _ptr(scratch), 0 if scratch is None else scratch.numel(), _stream()), "hbp_cumsumprod")
+    return g
+
+
+def cumsumprod_static_max_bytes() -> int:
+    return int(lib.hbp_cumsumprod_static_max_bytes())
+
+
+def cumsumprod_static(u, delta, a=None, gate=None, loss=LOSS_FINAL, g=None):
+    """hbp_cumsumprod for callers that cannot allocate: the scratch of the time-chunked scan lives in a
+    fixed 32 MiB array inside the library, so only inputs and the output are passed.  ``g`` must be given
+    by such callers (this wrapper makes one with torch only when it is omitted).  Raises HbpError with
+    status 5 when the problem needs more scratch than the fixed array holds."""
+    L, rows, d = u.shape
+    if gate is None:
+        gate = GATE_ONE if a is None else (GATE_CHANNEL_SHARED if a.dim() == 1 else GATE_CHANNEL_PER_STEP)
+    if g is None:
+        g = torch.empty((L + 1, rows, d), dtype=u.dtype, device=u.device)
+    _check(lib.hbp_cumsumprod_static(_dtype_code(u.dtype), gate, loss, L, rows, d, _ptr(u), _ptr(delta), _ptr(a),
+                                     _ptr(g), _stream()), "hbp_cumsumprod_static")
     return g
