@@ -262,7 +262,7 @@ def run_ours(args):
     if kk > 0 and scan_ms > 0:
         # the scan phase holds exactly the k scans of the iterations (g^0 is booked under "other")
         scan_iter_ms = scan_ms / args.steps / kk
-    scan_roof = {"bound": "hbm", "kernel": "scan_depth_ln_kernel" if tensors >= 3 and w.loss != "every_mse" else "scan kernels",
+    scan_roof = {"bound": "hbm", "kernel": "scan_depth_lnstat_kernel" if tensors >= 3 and w.loss != "every_mse" else "scan kernels",
                  "achieved": (scan_bytes / (scan_iter_ms * 1e-3) / 1e9) if scan_iter_ms else None, "peak": hbm, "unit": "GB/s",
                  "bytes_per_scan": scan_bytes, "tensors_counted": tensors, "traffic": None}
     if scan_roof["achieved"]:
