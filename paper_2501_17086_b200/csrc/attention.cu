@@ -243,9 +243,12 @@ template <typename T, int DH>
 void launch_bwd(Launcher& lc, const AttnArgs& a) {
   dim3 grid((a.seq + kRows - 1) / kRows, a.heads, a.batch);
   attn_rowdot_kernel<T, DH><<<grid, kThreads, 0, lc.stream>>>(a);
+  lc.count();
+  lc.check();
+  if (!g_force_simt && attention_bwd_tc(lc, a, a.status)) return;  // bf16, head dimension 64: tensor cores
   attn_bwd_dq_kernel<T, DH><<<grid, kThreads, 0, lc.stream>>>(a);
   attn_bwd_dkv_kernel<T, DH><<<grid, kThreads, 0, lc.stream>>>(a);
-  lc.count(3);
+  lc.count(2);
   lc.check();
 }
 

@@ -1,0 +1,346 @@
+// Flash-style causal attention backward on the tensor cores (bf16, head dimension 64).
+//
+// The S x S score matrix is never stored: each CTA recomputes the blocks it needs from Q, K and the
+// forward's log-sum-exp.  Two kernels, so that every output is owned by exactly one CTA (no atomics, runs
+// are bitwise reproducible):
+//   attn_dkv_kernel  one CTA per 128 keys; loops over blocks of 64 queries that can see them:
+//                       S^T = K Q^T, dP^T = V dO^T            (tcgen05.mma 128x64x16, accumulators in TMEM)
+//                       P^T = exp(S^T/sqrt(dh) - lse), dS^T = P^T * (dP^T - D)   (4 warps, one key row per lane)
+//                       dV += P^T dO,  dK += dS^T Q           (P^T, dS^T go back through shared memory as bf16)
+//   attn_dq_kernel   one CTA per 128 queries; loops over blocks of 64 keys up to the diagonal:
+//                       S = Q K^T, dP = dO V^T, dS = P * (dP - D),  dQ += dS K
+// with D_i = sum(dO_i * O_i).  All tiles are moved by TMA (128-byte swizzle); the same shared-memory tile
+// serves as a K-major operand (contraction over the head dimension) and as an MN-major operand (contraction
+// over its rows).  Each CTA uses at most 256 TMEM columns and ~100 KB of shared memory, so two CTAs share an
+// SM and the softmax of one overlaps the MMAs of the other.  All mbarrier waits are bounded.
+#include "tc_common.cuh"
+
+namespace hbp {
+
+using namespace tc;
+
+namespace {
+
+constexpr int DH = 64;
+constexpr int BIG = 128, SMALL = 64;
+constexpr int BIG_BYTES = BIG * DH * 2, SMALL_BYTES = SMALL * DH * 2, PS_BYTES = BIG * SMALL * 2;
+constexpr int THREADS = 192;  // warp 0 TMA, warp 1 MMA, warps 2..5 softmax / epilogue
+constexpr uint32_t TMEM_COLS = 256;
+constexpr float LOG2E = 1.4426950408889634f;
+
+struct AttnTcParams {
+  int S, H, B;
+  const float* lse;   // [B][H][S]
+  const float* drow;  // [B][H][S]
+  float scale;
+  int* status;
+};
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void named_barrier_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 64, A K-major, B K-major or MN-major
+constexpr uint32_t make_idesc(int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(SMALL >> 3) << 17) |
+         ((uint32_t)(BIG >> 4) << 24);
+}
+constexpr uint32_t IDESC_KK = make_idesc(0), IDESC_KMN = make_idesc(1);
+
+// Barrier slots (8 bytes each):
+// 0 big tiles loaded, 1-2 full[2], 3-4 empty[2], 5 scores ready, 6 probabilities ready, 7 all MMAs done.
+__device__ __forceinline__ uint32_t bar_at(uint32_t bars, int i) { return bars + 8u * i; }
+
+template <bool kDKV>
+__global__ void __launch_bounds__(THREADS, 2)
+attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_constant__ CUtensorMap tmBig1,
+                   const __grid_constant__ CUtensorMap tmSmall0, const __grid_constant__ CUtensorMap tmSmall1,
+                   const __grid_constant__ CUtensorMap tmOut0, const __grid_constant__ CUtensorMap tmOut1,
+                   const AttnTcParams p) {
+  // kDKV: big tiles = K, V (rows = keys), small tiles = Q, dO (rows = queries), outputs dK (Out0), dV (Out1).
+  // else: big tiles = Q, dO (rows = queries), small tiles = K, V (rows = keys), output dQ (Out0).
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t sBig0 = base, sBig1 = base + BIG_BYTES;
+  const uint32_t sSmall = base + 2 * BIG_BYTES;            // [buf][2 tiles]
+  const uint32_t sP = sSmall + 4 * SMALL_BYTES;            // P^T (dkv only)
+  const uint32_t sDS = sP + PS_BYTES;                      // dS^T / dS
+  constexpr int VEC_OFF = 2 * BIG_BYTES + 4 * SMALL_BYTES + 2 * PS_BYTES;
+  float* vec = reinterpret_cast<float*>(aligned + VEC_OFF);  // [2 buffers][lse 64 | D 64]
+  uint64_t* bar_mem = reinterpret_cast<uint64_t*>(aligned + VEC_OFF + 1024);
+  const uint32_t bars = smem_u32(bar_mem);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int blk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int big0 = blk * BIG;  // first key (dkv) or first query (dq) of this CTA
+  // inner blocks: dkv: queries from big0 on; dq: keys up to the last query of the block
+  const int n_small = (p.S + SMALL - 1) / SMALL;
+  const int it_beg = kDKV ? (big0 / SMALL) : 0;
+  const int it_end = kDKV ? n_small : min(n_small, (min(p.S, big0 + BIG) + SMALL - 1) / SMALL);
+  const int n_it = it_end - it_beg;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_at(bars, 0), 1);
+    mbar_init(bar_at(bars, 1), 1);
+    mbar_init(bar_at(bars, 2), 1);
+    mbar_init(bar_at(bars, 3), 1);
+    mbar_init(bar_at(bars, 4), 1);
+    mbar_init(bar_at(bars, 5), 1);
+    mbar_init(bar_at(bars, 6), 4);
+    mbar_init(bar_at(bars, 7), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  // TMEM columns: scores [0,64), dP [64,128), accumulator 0 [128,192), accumulator 1 [192,256)
+  const uint32_t tS = tmem, tDP = tmem + 64, tAcc0 = tmem + 128, tAcc1 = tmem + 192;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(bar_at(bars, 0), 2 * BIG_BYTES);
+      tma_load_4d(sBig0, &tmBig0, bar_at(bars, 0), 0, big0, h, b);
+      tma_load_4d(sBig1, &tmBig1, bar_at(bars, 0), 0, big0, h, b);
+      bool ok = true;
+      int last_buf_parity[2] = {-1, -1};
+      for (int it = 0; it < n_it && ok; ++it) {
+        const int buf = it & 1;
+        const uint32_t ph = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(bar_at(bars, 3 + buf), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        const int r0 = (it_beg + it) * SMALL;
+        mbar_expect_tx(bar_at(bars, 1 + buf), 2 * SMALL_BYTES);
+        last_buf_parity[buf] = (int)ph;
+        tma_load_4d(sSmall + (2 * buf) * SMALL_BYTES, &tmSmall0, bar_at(bars, 1 + buf), 0, r0, h, b);
+        tma_load_4d(sSmall + (2 * buf + 1) * SMALL_BYTES, &tmSmall1, bar_at(bars, 1 + buf), 0, r0, h, b);
+      }
+      if (!ok) {  // leave no copy of ours in flight
+        for (int buf = 0; buf < 2; ++buf)
+          if (last_buf_parity[buf] >= 0) {
+            const uint64_t t0 = global_ns();
+            while (!mbar_try_wait(bar_at(bars, 1 + buf), (uint32_t)last_buf_parity[buf]) &&
+                   global_ns() - t0 < 100000000ull) {
+            }
+          }
+        const uint64_t t0 = global_ns();
+        while (!mbar_try_wait(bar_at(bars, 0), 0) && global_ns() - t0 < 100000000ull) {
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      bool ok = mbar_wait(bar_at(bars, 0), 0, abort_flag, p.status);
+      tc_fence_after();
+      for (int it = 0; it < n_it && ok; ++it) {
+        const int buf = it & 1;
+        const uint32_t ph = (uint32_t)(it >> 1) & 1u, itp = (uint32_t)it & 1u;
+        if (!mbar_wait(bar_at(bars, 1 + buf), ph, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t s0 = sSmall + (2 * buf) * SMALL_BYTES, s1 = s0 + SMALL_BYTES;
+        // scores and dP: contraction over the head dimension, both operands K-major
+#pragma unroll
+        for (int k = 0; k < DH / 16; ++k)
+          tc_mma(tS, make_desc(sBig0 + 32 * k, 16, 1024), make_desc(s0 + 32 * k, 16, 1024), IDESC_KK, k != 0);
+#pragma unroll
+        for (int k = 0; k < DH / 16; ++k)
+          tc_mma(tDP, make_desc(sBig1 + 32 * k, 16, 1024), make_desc(s1 + 32 * k, 16, 1024), IDESC_KK, k != 0);
+        tc_commit(bar_at(bars, 5));
+        if (!mbar_wait(bar_at(bars, 6), itp, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        // accumulate: contraction over the 64 rows of the small tiles, which are MN-major B operands here
+        const uint32_t acc_on = it != 0 ? 1u : 0u;
+        if (kDKV) {
+#pragma unroll
+          for (int k = 0; k < SMALL / 16; ++k)  // dV += P^T dO
+            tc_mma(tAcc1, make_desc(sP + 32 * k, 16, 1024), make_desc(s1 + 2048 * k, 8192, 1024), IDESC_KMN,
+                   acc_on | (k != 0));
+#pragma unroll
+          for (int k = 0; k < SMALL / 16; ++k)  // dK += dS^T Q
+            tc_mma(tAcc0, make_desc(sDS + 32 * k, 16, 1024), make_desc(s0 + 2048 * k, 8192, 1024), IDESC_KMN,
+                   acc_on | (k != 0));
+        } else {
+#pragma unroll
+          for (int k = 0; k < SMALL / 16; ++k)  // dQ += dS K
+            tc_mma(tAcc0, make_desc(sDS + 32 * k, 16, 1024), make_desc(s0 + 2048 * k, 8192, 1024), IDESC_KMN,
+                   acc_on | (k != 0));
+        }
+        tc_commit(bar_at(bars, 3 + buf));
+      }
+      tc_commit(bar_at(bars, 7));
+      if (!ok) {
+        const uint64_t t0 = global_ns();
+        while (!mbar_try_wait(bar_at(bars, 7), 0) && global_ns() - t0 < 100000000ull) {
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax and epilogue (128 threads)
+    const int t = threadIdx.x - 64;             // 0..127
+    const int quarter = warp & 3;               // TMEM lane quarter this warp may read
+    const int row = quarter * 32 + lane;        // row of the big tile (key for dkv, query for dq)
+    const int grow = big0 + row;                // its index in the sequence
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const float scale2 = p.scale * LOG2E;
+    const int64_t stat_base = ((int64_t)b * p.H + h) * p.S;
+    float my_lse = 0.0f, my_d = 0.0f;
+    if (!kDKV) {  // one query per lane: its statistics are scalars
+      my_lse = grow < p.S ? p.lse[stat_base + grow] * LOG2E : INFINITY;
+      my_d = grow < p.S ? p.drow[stat_base + grow] : 0.0f;
+    }
+    bool ok = true;  // false after a wait gave up: keep pace with the named barriers, do no more work
+    for (int it = 0; it < n_it; ++it) {
+      const int c0 = (it_beg + it) * SMALL;  // first query (dkv) / key (dq) of the small block
+      float* vb = vec + (it & 1) * 128;
+      if (kDKV) {  // statistics of the 64 queries of this block, shared by all rows
+        const int q = c0 + (t & 63);
+        if (t < 64) vb[t] = q < p.S ? p.lse[stat_base + q] * LOG2E : INFINITY;
+        else vb[t] = q < p.S ? p.drow[stat_base + q] : 0.0f;
+        named_barrier_128();
+      }
+      if (!ok) continue;
+      if (!mbar_wait(bar_at(bars, 5), (uint32_t)it & 1u, abort_flag, p.status)) { ok = false; continue; }
+      tc_fence_after();
+#pragma unroll 1
+      for (int half = 0; half < 2; ++half) {
+        float s[32], dp[32];
+        tc_ld32(tS + lane_addr + half * 32, s);
+        tc_ld32(tDP + lane_addr + half * 32, dp);
+        float pv[32], ds[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const int col = c0 + half * 32 + c;
+          float lse2, dd;
+          bool vis;
+          if (kDKV) {  // row = key, column = query
+            lse2 = vb[half * 32 + c];
+            dd = vb[64 + half * 32 + c];
+            vis = (col >= grow) && (grow < p.S);
+          } else {     // row = query, column = key
+            lse2 = my_lse;
+            dd = my_d;
+            vis = (col <= grow) && (col < p.S);
+          }
+          const float pr = vis ? fast_exp2(fmaf(s[c], scale2, -lse2)) : 0.0f;
+          pv[c] = pr;
+          ds[c] = pr * (dp[c] - dd);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (kDKV) st_shared16(swz(sP, row, half * 4 + u), pack8(pv + 8 * u));
+          st_shared16(swz(sDS, row, half * 4 + u), pack8(ds + 8 * u));
+        }
+      }
+      fence_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_at(bars, 6));
+    }
+    // ---- epilogue: accumulators -> bf16 -> shared -> TMA store
+    ok = ok && mbar_wait(bar_at(bars, 7), 0, abort_flag, p.status);
+    if (ok) {
+      tc_fence_after();
+#pragma unroll 1
+      for (int o = 0; o < (kDKV ? 2 : 1); ++o) {
+        const uint32_t dst = o == 0 ? sDS : sP;          // staging: the probability tiles are free now
+        const float mul = o == 0 ? p.scale : 1.0f;       // dK and dQ carry the 1/sqrt(dh) factor, dV does not
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          float v[32];
+          tc_ld32((o == 0 ? tAcc0 : tAcc1) + lane_addr + half * 32, v);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) v[c] *= mul;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) st_shared16(swz(dst, row, half * 4 + u), pack8(v + 8 * u));
+        }
+      }
+      fence_async_smem();
+    }
+    named_barrier_128();
+    if (t == 0 && ok) {
+      tma_store_4d(&tmOut0, sDS, 0, big0, h, b);
+      if (kDKV) tma_store_4d(&tmOut1, sP, 0, big0, h, b);
+      tma_store_wait_all();
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+constexpr int SMEM_BYTES = 2 * BIG_BYTES + 4 * SMALL_BYTES + 2 * PS_BYTES + 1024 /*vectors*/ + 256 /*barriers*/ + 1024;
+
+// 4-D map {dh, sequence, head, batch} of one [tokens][ld] tensor's column block starting at `base`.
+bool make_map4(CUtensorMap* tm, const void* base, int S, int H, int B, int64_t ld, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)DH, (cuuint64_t)S, (cuuint64_t)H, (cuuint64_t)B};
+  cuuint64_t strides[3] = {(cuuint64_t)ld * 2, (cuuint64_t)DH * 2, (cuuint64_t)S * (cuuint64_t)ld * 2};
+  cuuint32_t box[4] = {(cuuint32_t)DH, (cuuint32_t)box_rows, 1, 1}, estr[4] = {1, 1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+// Runs dQ, dK, dV of attention_bwd on the tensor cores; delta_rows must already hold rowsum(dO * O).
+// Returns false (nothing launched) when the problem does not fit this kernel.
+bool attention_bwd_tc(Launcher& lc, const AttnArgs& a, int* status_word) {
+  if (a.dtype != HBP_BF16 || a.head_dim != DH || !status_word) return false;
+  const int d = a.heads * DH;
+  const int64_t ld3 = 3 * (int64_t)d;
+  if (((uintptr_t)a.qkv | (uintptr_t)a.d_o | (uintptr_t)a.d_qkv) & 15u) return false;
+  if (d % 8) return false;
+  const bf16* qkv = (const bf16*)a.qkv;
+  bf16* dqkv = (bf16*)a.d_qkv;
+  CUtensorMap qB, qS, kB, kS, vB, vS, oB, oS, dq, dk, dv;
+  bool ok = make_map4(&qB, qkv, a.seq, a.heads, a.batch, ld3, BIG) && make_map4(&qS, qkv, a.seq, a.heads, a.batch, ld3, SMALL) &&
+            make_map4(&kB, qkv + d, a.seq, a.heads, a.batch, ld3, BIG) && make_map4(&kS, qkv + d, a.seq, a.heads, a.batch, ld3, SMALL) &&
+            make_map4(&vB, qkv + 2 * d, a.seq, a.heads, a.batch, ld3, BIG) && make_map4(&vS, qkv + 2 * d, a.seq, a.heads, a.batch, ld3, SMALL) &&
+            make_map4(&oB, a.d_o, a.seq, a.heads, a.batch, d, BIG) && make_map4(&oS, a.d_o, a.seq, a.heads, a.batch, d, SMALL) &&
+            make_map4(&dq, dqkv, a.seq, a.heads, a.batch, ld3, BIG) && make_map4(&dk, dqkv + d, a.seq, a.heads, a.batch, ld3, BIG) &&
+            make_map4(&dv, dqkv + 2 * d, a.seq, a.heads, a.batch, ld3, BIG);
+  if (!ok) return false;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attn_bwd_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_bwd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    attr_set = true;
+  }
+  AttnTcParams p;
+  p.S = a.seq; p.H = a.heads; p.B = a.batch;
+  p.lse = a.lse; p.drow = a.delta_rows;
+  p.scale = 1.0f / sqrtf((float)DH);
+  p.status = status_word;
+  dim3 grid((a.seq + BIG - 1) / BIG, a.heads, a.batch);
+  // dK, dV: big tiles K, V; small tiles Q, dO
+  attn_bwd_tc_kernel<true><<<grid, THREADS, SMEM_BYTES, lc.stream>>>(kB, vB, qS, oS, dk, dv, p);
+  // dQ: big tiles Q, dO; small tiles K, V
+  attn_bwd_tc_kernel<false><<<grid, THREADS, SMEM_BYTES, lc.stream>>>(qB, oB, kS, vS, dq, dq, p);
+  lc.count(2);
+  lc.check();
+  return true;
+}
+
+}  // namespace hbp

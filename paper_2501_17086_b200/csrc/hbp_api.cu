@@ -273,6 +273,7 @@ struct Run {
     t.d_o = at(c->dO, (int64_t)b0 * state);
     t.d_qkv = at(c->dQKV, (int64_t)b0 * 3 * state);
     t.delta_rows = c->drow + (int64_t)b0 * f.batch * f.n_heads * f.seq;
+    t.status = c->status;
     attention_bwd(lc, t);
     if (!want_dy) return;
     GemmArgs b = base_args();  // dY = [dQ dK dV] [Wq; Wk; Wv]

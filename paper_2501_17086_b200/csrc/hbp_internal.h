@@ -137,9 +137,12 @@ struct AttnArgs {
   const void* d_o = nullptr;
   void* d_qkv = nullptr;        // [tokens][3d]
   float* delta_rows = nullptr;  // scratch [batch][heads][seq]: rowsum(dO * O)
+  int* status = nullptr;        // device status word for the bounded waits of the tensor-core kernels
 };
 void attention_fwd(Launcher& lc, const AttnArgs& a);
 void attention_bwd(Launcher& lc, const AttnArgs& a);
+// Tensor-core dQ/dK/dV (attention_tc.cu); false if the problem does not qualify (nothing launched).
+bool attention_bwd_tc(Launcher& lc, const AttnArgs& a, int* status_word);
 
 // ---------------------------------------------------------------- device math
 __device__ __forceinline__ float gelu_f(float z) { return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f)); }
