@@ -140,9 +140,9 @@ __global__ void reduce_splitk_kernel(const float* __restrict__ partial, float* _
                                      int64_t elems) {
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= elems) return;
-  float s = 0.0f;
-  for (int k = 0; k < splits; ++k) s += partial[(int64_t)k * elems + i];  // fixed order: deterministic
-  out[i] = s;
+  double s = 0.0;
+  for (int k = 0; k < splits; ++k) s += (double)partial[(int64_t)k * elems + i];  // fixed order: deterministic
+  out[i] = (float)s;
 }
 
 template <typename T>

@@ -36,6 +36,9 @@ struct TcParams {
   int M, N, K, batch;
   int m_tiles, n_tiles, num_tiles, k_blocks;
   int a_mn, b_mn;  // 1: the operand is MN-major
+  int tf32;        // operands are float, multiplied as tf32 (else bf16)
+  int segs;        // K segments, each with its own pair of operand maps (3 for the split-float product)
+  int splits, kb_per_split;  // split-K: tile z index = split * batch + b; each split covers kb_per_split k-blocks
   int epi, d_f32;
   void* D; int64_t ldd, d_sb;
   void* D2; int64_t ldd2, d2_sb;
@@ -99,6 +102,8 @@ __device__ __forceinline__ void residual_chunk(const TcParams& p, int b, int row
 // ------------------------------------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
+               const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
                const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmD2,
                const __grid_constant__ CUtensorMap tmE, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -146,6 +151,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int tiles_per_batch = p.m_tiles * p.n_tiles;
+  // per element size: elements per 128-byte row (= K elements per stage), bytes of one MN-major block
+  const int row_elems = p.tf32 ? 32 : 64;
+  const uint32_t mn_block = p.tf32 ? 4096u : 8192u;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -155,29 +163,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t issued_mask = 0, issued_parity = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
-        const int b = tile / tiles_per_batch, r = tile % tiles_per_batch;
+        const int zc = tile / tiles_per_batch, r = tile % tiles_per_batch;
+        const int b = zc % p.batch, split = zc / p.batch;
         const int m0 = (r % p.m_tiles) * BM, n0 = (r / p.m_tiles) * BN;
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
-          const uint32_t sA = base + stage * STAGE_BYTES, sB = sA + A_BYTES;
-          const uint32_t fb = full_bar(stage);
-          mbar_expect_tx(fb, STAGE_BYTES);
-          issued_mask |= 1u << stage;
-          issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
-          const int k0 = kb * BK;
-          if (p.a_mn) {
-#pragma unroll
-            for (int i = 0; i < BM / 64; ++i) tma_load_3d(sA + i * 8192, &tmA, fb, m0 + 64 * i, k0, b);
-          } else {
-            tma_load_3d(sA, &tmA, fb, k0, m0, b);
+        const int kb_lo = split * p.kb_per_split, kb_hi = min(p.k_blocks, kb_lo + p.kb_per_split);
+        for (int seg = 0; seg < p.segs && ok; ++seg) {
+          const CUtensorMap* mA = seg == 0 ? &tmA : (seg == 1 ? &tmA1 : &tmA2);
+          const CUtensorMap* mB = seg == 0 ? &tmB : (seg == 1 ? &tmB1 : &tmB2);
+          for (int kb = kb_lo; kb < kb_hi; ++kb) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+            const uint32_t sA = base + stage * STAGE_BYTES, sB = sA + A_BYTES;
+            const uint32_t fb = full_bar(stage);
+            mbar_expect_tx(fb, STAGE_BYTES);
+            issued_mask |= 1u << stage;
+            issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+            const int k0 = kb * row_elems;
+            if (p.a_mn) {
+              for (int i = 0; i < BM / row_elems; ++i) tma_load_3d(sA + i * mn_block, mA, fb, m0 + row_elems * i, k0, b);
+            } else {
+              tma_load_3d(sA, mA, fb, k0, m0, b);
+            }
+            if (p.b_mn) {
+              for (int i = 0; i < BN / row_elems; ++i) tma_load_3d(sB + i * mn_block, mB, fb, n0 + row_elems * i, k0, b);
+            } else {
+              tma_load_3d(sB, mB, fb, k0, n0, b);
+            }
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
           }
-          if (p.b_mn) {
-#pragma unroll
-            for (int i = 0; i < BN / 64; ++i) tma_load_3d(sB + i * 8192, &tmB, fb, n0 + 64 * i, k0, b);
-          } else {
-            tma_load_3d(sB, &tmB, fb, k0, n0, b);
-          }
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {
@@ -193,11 +205,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = (1u << 4) /*fp32 accumulate*/ | (1u << 7) /*A bf16*/ | (1u << 10) /*B bf16*/ |
-                             ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) | ((uint32_t)(BN >> 3) << 17) |
-                             ((uint32_t)(BM >> 4) << 24);
-      const uint32_t a_step = p.a_mn ? 2048u : 32u, b_step = p.b_mn ? 2048u : 32u;  // bytes per 16 of K
-      const uint32_t a_lead = p.a_mn ? 8192u : 16u, b_lead = p.b_mn ? 8192u : 16u;
+      const uint32_t fmt = p.tf32 ? 2u : 1u;  // operand format: tf32 or bf16
+      const uint32_t idesc = (1u << 4) /*fp32 accumulate*/ | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn << 15) |
+                             ((uint32_t)p.b_mn << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      // one instruction consumes 32 bytes of K: 32 bytes along a K-major row, or 16 rows of an MN-major bf16 block
+      const uint32_t a_step = p.a_mn ? 2048u : 32u, b_step = p.b_mn ? 2048u : 32u;
+      const uint32_t a_lead = p.a_mn ? mn_block : 16u, b_lead = p.b_mn ? mn_block : 16u;
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
@@ -205,16 +218,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)acc * BN;
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        const int split = (tile / tiles_per_batch) / p.batch;
+        const int kb_lo = split * p.kb_per_split, kb_hi = min(p.k_blocks, kb_lo + p.kb_per_split);
+        uint32_t first = 1;
+        for (int it = (kb_hi - kb_lo) * p.segs; it > 0; --it) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sA = base + stage * STAGE_BYTES, sB = sA + A_BYTES;
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
+          for (int k = 0; k < 4; ++k) {
             const uint64_t ad = make_desc(sA + k * a_step, a_lead, 1024u);
             const uint64_t bd = make_desc(sB + k * b_step, b_lead, 1024u);
-            tc_mma(tmem_d, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+            if (p.tf32) tc_mma_tf32(tmem_d, ad, bd, idesc, (first && k == 0) ? 0u : 1u);
+            else tc_mma(tmem_d, ad, bd, idesc, (first && k == 0) ? 0u : 1u);
           }
+          first = 0;
           tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -243,6 +261,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int cw = p.d_f32 ? 32 : 64;      // accumulator columns per staged chunk (128 bytes of output per row)
     const int nchunks = 128 / cw;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+      // b indexes the outputs: with split-K it is split * batch + batch entry (partial sums [split][batch][M][N])
       const int b = tile / tiles_per_batch, r = tile % tiles_per_batch;
       const int m0 = (r % p.m_tiles) * BM, n0 = (r / p.m_tiles) * BN;
       const int row0 = m0 + quarter * 32, colw = n0 + half * 128;
@@ -368,7 +387,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // ------------------------------------------------------------------------------------------- host
 // Tensor map of one operand: element (mn, k, b) at base + b*sb + mn*s_mn + k*s_k (element strides).
 bool make_map(CUtensorMap* tm, const void* base, int extent_mn, int K, int batch, int64_t s_mn, int64_t s_k,
-              int64_t s_b, bool mn_major, int box_mn) {
+              int64_t s_b, bool mn_major, int box_mn, bool f32) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[3], strides[2];
@@ -377,12 +396,14 @@ bool make_map(CUtensorMap* tm, const void* base, int extent_mn, int K, int batch
   dims[0] = mn_major ? (cuuint64_t)extent_mn : (cuuint64_t)K;
   dims[1] = mn_major ? (cuuint64_t)K : (cuuint64_t)extent_mn;
   dims[2] = (cuuint64_t)batch;
-  strides[0] = (cuuint64_t)row_stride * 2;
-  strides[1] = batch > 1 ? (cuuint64_t)s_b * 2 : (cuuint64_t)row_stride * 2 * dims[1];
-  box[0] = 64;
-  box[1] = mn_major ? 64 : (cuuint32_t)box_mn;
+  const cuuint64_t es = f32 ? 4 : 2;
+  const cuuint32_t row_elems = f32 ? 32 : 64;  // 128 bytes
+  strides[0] = (cuuint64_t)row_stride * es;
+  strides[1] = batch > 1 ? (cuuint64_t)s_b * es : (cuuint64_t)row_stride * es * dims[1];
+  box[0] = row_elems;
+  box[1] = mn_major ? row_elems : (cuuint32_t)box_mn;
   box[2] = 1;
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(tm, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -404,11 +425,11 @@ bool make_map_epi(CUtensorMap* tm, const void* base, bool f32, int M, int N, int
 bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 // An operand qualifies if one of its two strides is 1 and the others keep every row 16-byte aligned.
-bool operand_ok(const void* base, int64_t s_mn, int64_t s_k, int64_t s_b, int batch, bool* mn_major) {
+bool operand_ok(const void* base, int64_t s_mn, int64_t s_k, int64_t s_b, int batch, bool* mn_major, int vec) {
   if (!aligned16(base)) return false;
-  if (batch > 1 && (s_b % 8 != 0 || s_b <= 0)) return false;
-  if (s_k == 1 && s_mn % 8 == 0 && s_mn > 0) { *mn_major = false; return true; }
-  if (s_mn == 1 && s_k % 8 == 0 && s_k > 0) { *mn_major = true; return true; }
+  if (batch > 1 && (s_b % vec != 0 || s_b <= 0)) return false;
+  if (s_k == 1 && s_mn % vec == 0 && s_mn > 0) { *mn_major = false; return true; }
+  if (s_mn == 1 && s_k % vec == 0 && s_k > 0) { *mn_major = true; return true; }
   return false;
 }
 
@@ -445,19 +466,35 @@ int sm_count() {
 int gemm_tc_stats_slots(int N) { return 2 * ((N + BN - 1) / BN); }
 
 bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
-  if (g.in_dtype != HBP_BF16 || g.A2 || g.splitk > 1 || !status_word) return false;
+  if (!status_word) return false;
+  const bool f32 = g.in_dtype == HBP_F32;
+  if (f32 && (!g.A_hi || !g.A_lo || !g.B_hi || !g.B_lo)) return false;  // float needs the split operands
+  if (!f32 && g.A2) return false;
   if (g.M <= 0 || g.N <= 0 || g.K <= 0 || g.batch <= 0) return false;
-  if (g.N % 8 || g.K % 8) return false;
+  const int vec = f32 ? 4 : 8;  // elements per 16 bytes
+  if (g.N % vec || g.K % vec) return false;
   if (g.epi != EPI_STORE && g.epi != EPI_GELU_FWD && g.epi != EPI_MUL && g.epi != EPI_RESID && g.epi != EPI_STORE_LN)
     return false;
   if (g.epi == EPI_STORE_LN && (!g.stats || !g.E)) return false;
-  if (g.d_f32 && g.epi != EPI_STORE) return false;
+  const bool out_f32 = g.d_f32 || f32;
+  if (out_f32 && g.epi != EPI_STORE) return false;
+  if (g.splitk > 1 && (g.epi != EPI_STORE || !out_f32 || !g.partial || g.ldd != g.N || (g.batch > 1 && g.d_sb != (int64_t)g.M * g.N)))
+    return false;
+  const void* A0 = f32 ? (const void*)g.A_hi : g.A;
+  const void* B0 = f32 ? (const void*)g.B_hi : g.B;
+  // strides of the operands the kernel reads (the split float copies have their own layout)
+  const int64_t a_sm = f32 && g.hl_a_sm ? g.hl_a_sm : g.a_sm, a_sk = f32 && g.hl_a_sk ? g.hl_a_sk : g.a_sk;
+  const int64_t b_sn = f32 && g.hl_b_sn ? g.hl_b_sn : g.b_sn, b_sk = f32 && g.hl_b_sk ? g.hl_b_sk : g.b_sk;
   bool a_mn = false, b_mn = false;
-  if (!operand_ok(g.A, g.a_sm, g.a_sk, g.a_sb, g.batch, &a_mn)) return false;
-  if (!operand_ok(g.B, g.b_sn, g.b_sk, g.b_sb, g.batch, &b_mn)) return false;
-  if (a_mn && g.M % 8) return false;
+  if (!operand_ok(A0, a_sm, a_sk, g.a_sb, g.batch, &a_mn, vec)) return false;
+  if (!operand_ok(B0, b_sn, b_sk, g.b_sb, g.batch, &b_mn, vec)) return false;
+  if (f32 && (!aligned16(g.A_lo) || !aligned16(g.B_lo))) return false;
+  // 32-bit MN-major operands need a shared-memory layout of their own that this kernel does not build:
+  // float operands must be K-major (the callers write the split copies that way)
+  if (f32 && (a_mn || b_mn || g.batch != 1)) return false;
+  if (a_mn && g.M % vec) return false;
   // epilogue operands: 16-byte vectors
-  const int dv = g.d_f32 ? 4 : 8;
+  const int dv = out_f32 ? 4 : 8;
   if (!aligned16(g.D) || g.ldd % dv || g.d_sb % dv) return false;
   if (g.D2 && (!aligned16(g.D2) || g.ldd2 % 8 || g.d2_sb % 8)) return false;
   if (g.E && (!aligned16(g.E) || g.lde % 8 || g.e_sb % 8)) return false;
@@ -468,13 +505,32 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   if (g.epi == EPI_RESID && !g.R && !g.E) return false;
 
   CUtensorMap tmA, tmB;
-  if (!make_map(&tmA, g.A, g.M, g.K, g.batch, g.a_sm, g.a_sk, g.a_sb, a_mn, BM)) return false;
-  if (!make_map(&tmB, g.B, g.N, g.K, g.batch, g.b_sn, g.b_sk, g.b_sb, b_mn, BN)) return false;
+  if (!make_map(&tmA, A0, g.M, g.K, g.batch, a_sm, a_sk, g.a_sb, a_mn, BM, f32)) return false;
+  if (!make_map(&tmB, B0, g.N, g.K, g.batch, b_sn, b_sk, g.b_sb, b_mn, BN, f32)) return false;
+  // float: segments A_hi B_lo, A_lo B_hi, A_hi B_hi - the small terms first, so that only the last segment adds
+  // to an accumulator of full magnitude (the tensor core's fp32 accumulation does not round to nearest)
+  CUtensorMap tmA1 = tmA, tmB1 = tmB, tmA2 = tmA, tmB2 = tmB;
+  if (f32) {
+    CUtensorMap a_lo, b_lo;
+    if (!make_map(&b_lo, g.B_lo, g.N, g.K, g.batch, b_sn, b_sk, g.b_sb, b_mn, BN, true)) return false;
+    if (!make_map(&a_lo, g.A_lo, g.M, g.K, g.batch, a_sm, a_sk, g.a_sb, a_mn, BM, true)) return false;
+    tmA2 = tmA; tmB2 = tmB;      // segment 2: hi x hi
+    tmA1 = a_lo; tmB1 = tmB;     // segment 1: lo x hi
+    tmB = b_lo;                  // segment 0: hi x lo (tmA stays A_hi)
+  }
+  const int row_elems = f32 ? 32 : 64;
+  const int k_blocks = (g.K + row_elems - 1) / row_elems;
+  int splits = g.splitk > 1 ? g.splitk : 1;
+  if (splits > k_blocks) splits = k_blocks;
+  const int kb_per_split = (k_blocks + splits - 1) / splits;
+  splits = (k_blocks + kb_per_split - 1) / kb_per_split;  // no empty split
   // epilogue operands that are staged through shared memory (everything but the forward residual update)
   CUtensorMap tmD = tmA, tmD2 = tmA, tmE = tmA;  // placeholders when unused
   if (g.epi != EPI_RESID) {
     if (g.batch > 1 && g.d_sb <= 0) return false;
-    if (!make_map_epi(&tmD, g.D, g.d_f32, g.M, g.N, g.batch, g.ldd, g.d_sb)) return false;
+    if (splits > 1) {
+      if (!make_map_epi(&tmD, g.partial, true, g.M, g.N, g.batch * splits, g.N, (int64_t)g.M * g.N)) return false;
+    } else if (!make_map_epi(&tmD, g.D, out_f32, g.M, g.N, g.batch, g.ldd, g.d_sb)) return false;
     if (g.epi == EPI_GELU_FWD && !make_map_epi(&tmD2, g.D2, false, g.M, g.N, g.batch, g.ldd2, g.d2_sb)) return false;
     if ((g.epi == EPI_MUL || g.epi == EPI_STORE_LN) && !make_map_epi(&tmE, g.E, false, g.M, g.N, g.batch, g.lde, g.e_sb))
       return false;
@@ -492,10 +548,12 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   p.M = g.M; p.N = g.N; p.K = g.K; p.batch = g.batch;
   p.m_tiles = (g.M + BM - 1) / BM;
   p.n_tiles = (g.N + BN - 1) / BN;
-  p.num_tiles = p.m_tiles * p.n_tiles * g.batch;
-  p.k_blocks = (g.K + BK - 1) / BK;
+  p.num_tiles = p.m_tiles * p.n_tiles * g.batch * splits;
+  p.k_blocks = k_blocks;
   p.a_mn = a_mn; p.b_mn = b_mn;
-  p.epi = g.epi; p.d_f32 = g.d_f32;
+  p.tf32 = f32; p.segs = f32 ? 3 : 1;
+  p.splits = splits; p.kb_per_split = kb_per_split;
+  p.epi = g.epi; p.d_f32 = out_f32;
   p.D = g.D; p.ldd = g.ldd; p.d_sb = g.d_sb;
   p.D2 = g.D2; p.ldd2 = g.ldd2; p.d2_sb = g.d2_sb;
   p.E = g.E; p.lde = g.lde; p.e_sb = g.e_sb;
@@ -504,9 +562,10 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   p.stats = g.stats; p.stats_sb = g.stats_sb;
   p.status = status_word;
   const int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
-  gemm_tc_kernel<<<grid, THREADS, SMEM_BYTES, lc.stream>>>(tmA, tmB, tmD, tmD2, tmE, p);
+  gemm_tc_kernel<<<grid, THREADS, SMEM_BYTES, lc.stream>>>(tmA, tmB, tmA1, tmB1, tmA2, tmB2, tmD, tmD2, tmE, p);
   lc.count();
   lc.check();
+  if (splits > 1) reduce_splitk(lc, g.partial, (float*)g.D, splits, (int64_t)g.batch * g.M * g.N);
   return true;
 }
 

@@ -12,7 +12,7 @@ namespace hbp {
 bool g_force_simt = false;
 
 bool gemm(Launcher& lc, const GemmArgs& g, int* status_word) {
-  if (!g_force_simt && g.in_dtype == HBP_BF16 && gemm_tc(lc, g, status_word)) return true;
+  if (!g_force_simt && gemm_tc(lc, g, status_word)) return true;
   gemm_simt(lc, g);
   return false;
 }
@@ -48,6 +48,11 @@ struct hbp_ctx {
   char* DACT = nullptr;    // [layers][N][h] gelu'(Z)
   float* xres = nullptr;   // [N][d] float master of the residual stream (bf16 only)
   double* hres = nullptr;  // RNN: 2 x [B][d] double master of the recurrent state (ping-pong)
+  // RNN, float: tf32 high/low splits of the GEMM operands, each written with the contraction index
+  // contiguous: A* is g * tanh' as [T*B][d] for the VJP or [d][T*B] for the weight gradients, H* the states
+  // h_0..h_{T-1} as [d][T*B], X* the inputs as [in][T*B], W* the recurrent matrix transposed
+  float *Ahi = nullptr, *Alo = nullptr, *Hhi = nullptr, *Hlo = nullptr, *Xhi = nullptr, *Xlo = nullptr;
+  float *Whi = nullptr, *Wlo = nullptr;
   char* U = nullptr;       // [steps][N][d] block VJP outputs (dY before the LayerNorm finish)
   char* H1 = nullptr;      // [group][N][h] dZ
   float2* lnpart = nullptr;  // [steps][N][slots] partial row sums of dY and dY * xhat from the GEMM epilogue
@@ -71,7 +76,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kGateBlocks = 256;
-constexpr int kMaxSplit = 64;
+constexpr int kMaxSplit = 256;
 
 inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
@@ -123,6 +128,12 @@ size_t carve(hbp_ctx* c, char* base) {
   if (f.block == HBP_BLOCK_RNN_TANH) {
     c->C = take(steps * N * d * es);
     c->hres = (double*)take(2 * N * d * 8);
+    if (f.dtype == HBP_F32) {
+      c->Ahi = (float*)take(steps * N * d * 4); c->Alo = (float*)take(steps * N * d * 4);
+      c->Hhi = (float*)take(steps * N * d * 4); c->Hlo = (float*)take(steps * N * d * 4);
+      c->Xhi = (float*)take(steps * N * (size_t)f.in_dim * 4); c->Xlo = (float*)take(steps * N * (size_t)f.in_dim * 4);
+      c->Whi = (float*)take(d * d * 4); c->Wlo = (float*)take(d * d * 4);
+    }
     c->scan_scratch_bytes = scan_scratch_bytes(f.dtype, f.L, f.tokens, f.d);
     c->scan_scratch = take(c->scan_scratch_bytes);
     const size_t wmax = d * (d > (size_t)f.in_dim ? d : (size_t)f.in_dim);
@@ -316,12 +327,19 @@ struct Run {
     a.A = at(g, state); a.A2 = c->C; a.a_sm = d; a.a_sk = 1;
     a.B = p->W; a.b_sn = 1; a.b_sk = d;
     a.epi = EPI_STORE; a.D = c->U; a.ldd = d;
+    if (c->Ahi) {  // float: g * tanh' split for the tf32 tensor-core product; B(n, k) = W[k][n] = W^T[n][k]
+      split_tf32(lc, (const float*)at(g, state), (const float*)c->C, c->Ahi, c->Alo, (int64_t)T * state);
+      a.A_hi = c->Ahi; a.A_lo = c->Alo;
+      a.B_hi = c->Whi; a.B_lo = c->Wlo; a.hl_b_sn = d; a.hl_b_sk = 1;
+    }
     run_gemm(a);
   }
   void rnn_wgrad(const hbp_grads* gr) {
     const int T = c->cfg.L;
     const int64_t rows = (int64_t)T * N, in = c->cfg.in_dim;
-    int split = (int)(rows / 2048);
+    // float on the tensor cores: at most 512 rows (16 k-blocks) per split keeps each fp32 accumulation chain
+    // short; the partial sums are then added in double in a fixed order
+    int split = (int)(rows / (c->Ahi ? 512 : 2048));
     if (split < 1) split = 1;
     if (split > kMaxSplit) split = kMaxSplit;
     for (int w = 0; w < 2; ++w) {
@@ -329,6 +347,12 @@ struct Run {
       a.M = (int)d; a.N = w == 0 ? (int)d : (int)in; a.K = (int)rows;
       a.A = at(g, state); a.A2 = c->C; a.a_sm = 1; a.a_sk = d;
       a.B = w == 0 ? x_all : inputs; a.b_sn = 1; a.b_sk = a.N;
+      if (c->Ahi) {  // tf32 path: transposed splits, so that the row index (the contraction) is contiguous
+        if (w == 0)
+          split_tf32_transposed(lc, (const float*)at(g, state), (const float*)c->C, c->Ahi, c->Alo, rows, (int)d);
+        a.A_hi = c->Ahi; a.A_lo = c->Alo; a.hl_a_sm = rows; a.hl_a_sk = 1;
+        a.B_hi = w == 0 ? c->Hhi : c->Xhi; a.B_lo = w == 0 ? c->Hlo : c->Xlo; a.hl_b_sn = rows; a.hl_b_sk = 1;
+      }
       a.epi = EPI_STORE; a.d_f32 = true;
       a.D = w == 0 ? gr->dW : gr->dU; a.ldd = a.N;
       if (split > 1) { a.splitk = split; a.partial = c->partial; }
@@ -555,6 +579,11 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
       rnn_forward_step(r.lc, f.dtype, params->W, params->U, r.at(inputs, (int64_t)t * N * f.in_dim), r.gate_ptr(t), hin,
                        hout, r.at(ctx->C, (int64_t)t * state), r.at(xa, (int64_t)(t + 1) * state), (int)N, (int)d,
                        f.in_dim);
+    }
+    if (ctx->Ahi) {  // operand splits that do not change between backward calls
+      split_tf32_transposed(r.lc, (const float*)xa, nullptr, ctx->Hhi, ctx->Hlo, (int64_t)T * N, (int)d);
+      split_tf32_transposed(r.lc, (const float*)inputs, nullptr, ctx->Xhi, ctx->Xlo, (int64_t)T * N, f.in_dim);
+      split_tf32_transposed(r.lc, (const float*)params->W, nullptr, ctx->Whi, ctx->Wlo, d, (int)d);
     }
   } else {
     const bool tr = f.block == HBP_BLOCK_PRELN_TRANSFORMER;

@@ -46,6 +46,12 @@ struct GemmArgs {
   float* R = nullptr;  // fp32 master copy of the residual stream [M][N], leading dim N
   float2* stats = nullptr;  // EPI_STORE_LN: [batch][M][stats_slots] partial sums; batch stride stats_sb (in float2)
   int64_t stats_sb = 0;
+  // float operands for the tensor cores: each of A (after the A2 product) and B split into a tf32-exact
+  // high part and a tf32-rounded remainder, written with the contraction index contiguous (their own
+  // strides below).  The tensor-core kernel forms A_hi B_lo + A_lo B_hi + A_hi B_hi (three tf32 products,
+  // fp32 accumulation, the small terms first).
+  const float *A_hi = nullptr, *A_lo = nullptr, *B_hi = nullptr, *B_lo = nullptr;
+  int64_t hl_a_sm = 0, hl_a_sk = 0, hl_b_sn = 0, hl_b_sk = 0;
   int splitk = 1;      // > 1: partial sums to `partial` [splitk][batch][M][N], reduced in fixed order
   float* partial = nullptr;
 };
@@ -115,6 +121,10 @@ void convert_to_f32(Launcher& lc, int dtype, const void* src, float* dst, int64_
 void gate_grad(Launcher& lc, int dtype, const void* g, const void* x, int64_t rows_total, int d, float* da,
                float* partial, int blocks);
 void reduce_splitk(Launcher& lc, const float* partial, float* out, int splits, int64_t elems);
+// hi = tf32-exact part of v, lo = tf32 rounding of (v - hi), with v = a[i] * (b ? b[i] : 1).
+void split_tf32(Launcher& lc, const float* a, const float* b, float* hi, float* lo, int64_t elems);
+// The same for a [rows][cols] matrix, written transposed: hiT, loT are [cols][rows].
+void split_tf32_transposed(Launcher& lc, const float* a, const float* b, float* hiT, float* loT, int64_t rows, int cols);
 
 // ---------------------------------------------------------------- RNN forward step (rnn.cu)
 // z = W h + U x_t in double from the double master state h_in; writes h_out (double), the cached

@@ -430,6 +430,58 @@ __global__ void __launch_bounds__(256) gate_grad_kernel(const T* __restrict__ g,
   }
 }
 
+// v = a * b (b optional); hi = v rounded to tf32 precision (13 low mantissa bits cleared), lo = the same
+// rounding of v - hi.  hi + lo carries 21+ bits of v, and both are exact tf32 operands.
+__device__ __forceinline__ float round_tf32(float v) {
+  uint32_t u = __float_as_uint(v);
+  u += 0x00000fffu + ((u >> 13) & 1u);  // round to nearest even at bit 13
+  return __uint_as_float(u & 0xffffe000u);
+}
+__global__ void split_tf32_kernel(const float4* __restrict__ a, const float4* __restrict__ b, float4* __restrict__ hi,
+                                  float4* __restrict__ lo, int64_t nvec) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= nvec) return;
+  float4 v = a[i];
+  if (b) {
+    const float4 w = b[i];
+    v.x *= w.x; v.y *= w.y; v.z *= w.z; v.w *= w.w;
+  }
+  float4 h, l;
+  h.x = round_tf32(v.x); h.y = round_tf32(v.y); h.z = round_tf32(v.z); h.w = round_tf32(v.w);
+  l.x = round_tf32(v.x - h.x); l.y = round_tf32(v.y - h.y); l.z = round_tf32(v.z - h.z); l.w = round_tf32(v.w - h.w);
+  hi[i] = h;
+  lo[i] = l;
+}
+__global__ void __launch_bounds__(256) split_tf32_transposed_kernel(const float* __restrict__ a, const float* __restrict__ b,
+                                                                    float* __restrict__ hiT, float* __restrict__ loT,
+                                                                    int64_t rows, int cols) {
+  __shared__ float th[32][33], tl[32][33];
+  const int64_t r0 = (int64_t)blockIdx.x * 32;
+  const int c0 = blockIdx.y * 32;
+  const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;  // ty in 0..7
+  for (int i = ty; i < 32; i += 8) {
+    const int64_t r = r0 + i;
+    const int c = c0 + tx;
+    float v = 0.0f;
+    if (r < rows && c < cols) {
+      v = a[r * cols + c];
+      if (b) v *= b[r * cols + c];
+    }
+    const float h = round_tf32(v);
+    th[i][tx] = h;
+    tl[i][tx] = round_tf32(v - h);
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int c = c0 + i;
+    const int64_t r = r0 + tx;
+    if (c < cols && r < rows) {
+      hiT[(int64_t)c * rows + r] = th[tx][i];
+      loT[(int64_t)c * rows + r] = tl[tx][i];
+    }
+  }
+}
+
 inline int row_block_threads(int d, int V) {
   int t = (d / V + 31) / 32 * 32;
   return t < 32 ? 32 : t;
@@ -530,6 +582,21 @@ void layernorm_fwd(Launcher& lc, int dtype, const void* x, bool x_is_f32, void* 
     layernorm_fwd_kernel<bf16, float><<<(unsigned)rows, threads, 0, lc.stream>>>((const float*)x, (bf16*)xhat, rstd, d, eps);
   else
     layernorm_fwd_kernel<bf16, bf16><<<(unsigned)rows, threads, 0, lc.stream>>>((const bf16*)x, (bf16*)xhat, rstd, d, eps);
+  lc.count();
+  lc.check();
+}
+
+void split_tf32(Launcher& lc, const float* a, const float* b, float* hi, float* lo, int64_t elems) {
+  const int64_t nvec = elems / 4;
+  split_tf32_kernel<<<(unsigned)((nvec + 255) / 256), 256, 0, lc.stream>>>((const float4*)a, (const float4*)b, (float4*)hi,
+                                                                          (float4*)lo, nvec);
+  lc.count();
+  lc.check();
+}
+
+void split_tf32_transposed(Launcher& lc, const float* a, const float* b, float* hiT, float* loT, int64_t rows, int cols) {
+  dim3 grid((unsigned)((rows + 31) / 32), (unsigned)((cols + 31) / 32));
+  split_tf32_transposed_kernel<<<grid, 256, 0, lc.stream>>>(a, b, hiT, loT, rows, cols);
   lc.count();
   lc.check();
 }
