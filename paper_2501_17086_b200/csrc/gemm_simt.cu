@@ -34,6 +34,11 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int b, int m, 
       if (g.R) g.R[(int64_t)m * g.N + n] = v;
       ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(v);
     } break;
+    case EPI_ADD: {
+      float e = to_f(((const T*)g.E)[b * g.e_sb + (int64_t)m * g.lde + n]);
+      if (g.d_f32) ((float*)g.D)[b * g.d_sb + dn] = acc + e;
+      else ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(acc + e);
+    } break;
     case EPI_MUL: {
       float e = to_f(((const T*)g.E)[b * g.e_sb + (int64_t)m * g.lde + n]);
       ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(acc * e);

@@ -257,7 +257,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     int acc = 0;
     uint32_t acc_phase = 0;
     const bool staged = p.epi != EPI_RESID;
-    const bool has_e = p.epi == EPI_MUL || p.epi == EPI_STORE_LN;
+    const bool has_e = p.epi == EPI_MUL || p.epi == EPI_STORE_LN || p.epi == EPI_ADD;
     const int cw = p.d_f32 ? 32 : 64;      // accumulator columns per staged chunk (128 bytes of output per row)
     const int nchunks = 128 / cw;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
@@ -301,6 +301,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!mbar_wait(ebar, e_phase, abort_flag, p.status)) { ok = false; break; }
             e_phase ^= 1u;
             e_pending = false;
+            if (p.epi == EPI_ADD) {  // float tile: 32 columns
+#pragma unroll
+              for (int u = 0; u < 8; ++u) {
+                const uint4 raw = ld_shared16(swz(buf, lane, u));
+                v[4 * u] += __uint_as_float(raw.x);
+                v[4 * u + 1] += __uint_as_float(raw.y);
+                v[4 * u + 2] += __uint_as_float(raw.z);
+                v[4 * u + 3] += __uint_as_float(raw.w);
+              }
+            } else
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
               float e[8];
@@ -473,11 +483,13 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   if (g.M <= 0 || g.N <= 0 || g.K <= 0 || g.batch <= 0) return false;
   const int vec = f32 ? 4 : 8;  // elements per 16 bytes
   if (g.N % vec || g.K % vec) return false;
-  if (g.epi != EPI_STORE && g.epi != EPI_GELU_FWD && g.epi != EPI_MUL && g.epi != EPI_RESID && g.epi != EPI_STORE_LN)
+  if (g.epi != EPI_STORE && g.epi != EPI_GELU_FWD && g.epi != EPI_MUL && g.epi != EPI_RESID && g.epi != EPI_STORE_LN &&
+      g.epi != EPI_ADD)
     return false;
+  if (g.epi == EPI_ADD && (!g.E || !(g.d_f32 || g.in_dtype == HBP_F32) || g.splitk > 1)) return false;  // float outputs only
   if (g.epi == EPI_STORE_LN && (!g.stats || !g.E)) return false;
   const bool out_f32 = g.d_f32 || f32;
-  if (out_f32 && g.epi != EPI_STORE) return false;
+  if (out_f32 && g.epi != EPI_STORE && g.epi != EPI_ADD) return false;
   if (g.splitk > 1 && (g.epi != EPI_STORE || !out_f32 || !g.partial || g.ldd != g.N || (g.batch > 1 && g.d_sb != (int64_t)g.M * g.N)))
     return false;
   const void* A0 = f32 ? (const void*)g.A_hi : g.A;
@@ -497,7 +509,7 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   const int dv = out_f32 ? 4 : 8;
   if (!aligned16(g.D) || g.ldd % dv || g.d_sb % dv) return false;
   if (g.D2 && (!aligned16(g.D2) || g.ldd2 % 8 || g.d2_sb % 8)) return false;
-  if (g.E && (!aligned16(g.E) || g.lde % 8 || g.e_sb % 8)) return false;
+  if (g.E && (!aligned16(g.E) || g.lde % (g.epi == EPI_ADD ? 4 : 8) || g.e_sb % (g.epi == EPI_ADD ? 4 : 8))) return false;
   if (g.gate && (!aligned16(g.gate) || g.gate_sb % 8)) return false;
   if (g.R && (!aligned16(g.R) || g.N % 4)) return false;
   if (g.epi == EPI_GELU_FWD && !g.D2) return false;
@@ -534,6 +546,7 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
     if (g.epi == EPI_GELU_FWD && !make_map_epi(&tmD2, g.D2, false, g.M, g.N, g.batch, g.ldd2, g.d2_sb)) return false;
     if ((g.epi == EPI_MUL || g.epi == EPI_STORE_LN) && !make_map_epi(&tmE, g.E, false, g.M, g.N, g.batch, g.lde, g.e_sb))
       return false;
+    if (g.epi == EPI_ADD && !make_map_epi(&tmE, g.E, true, g.M, g.N, g.batch, g.lde, g.e_sb)) return false;
   }
 
   static bool attr_set = false;

@@ -202,6 +202,7 @@ struct Run {
     a.in_dtype = c->cfg.dtype;
     return a;
   }
+  bool u_has_delta = false;  // the VJP GEMM already added delta_l to u_l
   bool stats_ok = true;  // every dY GEMM since the last reset also produced the LayerNorm row sums
   bool run_gemm(const GemmArgs& a) { return gemm(lc, a, c->status); }
   hbp_status result() const { return lc.err == cudaSuccess ? HBP_OK : HBP_ERR_CUDA; }
@@ -327,6 +328,10 @@ struct Run {
     a.A = at(g, state); a.A2 = c->C; a.a_sm = d; a.a_sk = 1;
     a.B = p->W; a.b_sn = 1; a.b_sk = d;
     a.epi = EPI_STORE; a.D = c->U; a.ldd = d;
+    if (c->cfg.loss == HBP_LOSS_EVERY_STEP) {  // u_t + delta_t in the epilogue: one tensor less for the scan
+      a.epi = EPI_ADD; a.E = delta; a.lde = d;
+      u_has_delta = true;
+    }
     if (c->Ahi) {  // float: g * tanh' split for the tf32 tensor-core product; B(n, k) = W[k][n] = W^T[n][k]
       split_tf32(lc, (const float*)at(g, state), (const float*)c->C, c->Ahi, c->Alo, (int64_t)T * state);
       a.A_hi = c->Ahi; a.A_lo = c->Alo;
@@ -383,6 +388,7 @@ struct Run {
     ScanArgs s;
     s.dtype = c->cfg.dtype; s.L = c->steps; s.l_lo = lo; s.l_hi = hi; s.rows = N; s.d = (int)d;
     s.u = with_u ? c->U : nullptr;
+    s.u_has_delta = with_u && u_has_delta;
     s.delta = delta; s.loss = c->cfg.loss;
     s.a = p->a; s.gate = c->cfg.gate;
     s.g = g;

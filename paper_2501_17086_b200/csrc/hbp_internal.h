@@ -20,6 +20,7 @@ enum Epilogue {
   EPI_MUL = 3,       // D = acc * E[m,n]   (dZ = dA * gelu'(Z) with the cached derivative)
   EPI_AFFINE = 4,    // D = (E ? E[m,n] : 0) + gate[n] * E2[m,n] + acc
   EPI_STORE_LN = 6,  // D = acc, plus per-row partial sums (sum acc, sum acc * E[m,n]) per 128 columns -> stats
+  EPI_ADD = 7,       // D = acc + E[m,n]   (u_t + delta_t: the scan then reads one tensor less)
   EPI_RNN_FWD = 5,   // c = tanh(acc + E[m,n]);  D2 = 1 - c^2;  D = gate[n] * E2[m,n] + c
 };
 
@@ -92,6 +93,7 @@ struct ScanArgs {
   int64_t rows = 0;
   int d = 0;
   const void* u = nullptr;      // [L][rows][d] or nullptr (zeros)
+  bool u_has_delta = false;     // u[l] already contains delta_l for l < L (added by the producing GEMM)
   const void* delta = nullptr;  // per hbp_loss
   int loss = HBP_LOSS_FINAL;
   const void* a = nullptr;  // gate

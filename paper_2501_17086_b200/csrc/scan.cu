@@ -72,7 +72,7 @@ __device__ __forceinline__ void stv(T* p, const Vec<T>& v) {
 template <typename T>
 __device__ __forceinline__ const T* delta_at(const ScanArgs& s, int l, int64_t state_elems) {
   if (!s.delta) return nullptr;
-  if (s.loss == HBP_LOSS_EVERY_STEP) return (const T*)s.delta + (int64_t)l * state_elems;
+  if (s.loss == HBP_LOSS_EVERY_STEP) return (s.u_has_delta && l < s.L) ? nullptr : (const T*)s.delta + (int64_t)l * state_elems;
   return (l == s.L) ? (const T*)s.delta : nullptr;
 }
 template <typename T>
