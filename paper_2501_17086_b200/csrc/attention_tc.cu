@@ -31,7 +31,8 @@ constexpr float LOG2E = 1.4426950408889634f;
 struct AttnTcParams {
   int S, H, B;
   const float* lse;   // [B][H][S]
-  const float* drow;  // [B][H][S]
+  const float* drow;  // rowsum(dO * O) of (batch b, head h, query q) at drow[b * d_sb + h * d_sh + q * d_sq]
+  int64_t d_sb, d_sh, d_sq;
   float scale;
   int* status;
 };
@@ -199,7 +200,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
     float my_lse = 0.0f, my_d = 0.0f;
     if (!kDKV) {  // one query per lane: its statistics are scalars
       my_lse = grow < p.S ? p.lse[stat_base + grow] * LOG2E : INFINITY;
-      my_d = grow < p.S ? p.drow[stat_base + grow] : 0.0f;
+      my_d = grow < p.S ? p.drow[(int64_t)b * p.d_sb + (int64_t)h * p.d_sh + (int64_t)grow * p.d_sq] : 0.0f;
     }
     bool ok = true;  // false after a wait gave up: keep pace with the named barriers, do no more work
     for (int it = 0; it < n_it; ++it) {
@@ -208,35 +209,41 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
       if (kDKV) {  // statistics of the 64 queries of this block, shared by all rows
         const int q = c0 + (t & 63);
         if (t < 64) vb[t] = q < p.S ? p.lse[stat_base + q] * LOG2E : INFINITY;
-        else vb[t] = q < p.S ? p.drow[stat_base + q] : 0.0f;
+        else vb[t] = q < p.S ? p.drow[(int64_t)b * p.d_sb + (int64_t)h * p.d_sh + (int64_t)q * p.d_sq] : 0.0f;
         named_barrier_128();
       }
       if (!ok) continue;
       if (!mbar_wait(bar_at(bars, 5), (uint32_t)it & 1u, abort_flag, p.status)) { ok = false; continue; }
       tc_fence_after();
+      // only blocks that touch the diagonal (or the end of the sequence) need the per-element mask
+      const bool full = kDKV ? (c0 >= big0 + BIG - 1 && big0 + BIG <= p.S) : (c0 + SMALL - 1 <= big0 && c0 + SMALL <= p.S);
 #pragma unroll 1
       for (int half = 0; half < 2; ++half) {
         float s[32], dp[32];
         tc_ld32(tS + lane_addr + half * 32, s);
         tc_ld32(tDP + lane_addr + half * 32, dp);
         float pv[32], ds[32];
+        if (full) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const int col = c0 + half * 32 + c;
-          float lse2, dd;
-          bool vis;
-          if (kDKV) {  // row = key, column = query
-            lse2 = vb[half * 32 + c];
-            dd = vb[64 + half * 32 + c];
-            vis = (col >= grow) && (grow < p.S);
-          } else {     // row = query, column = key
-            lse2 = my_lse;
-            dd = my_d;
-            vis = (col <= grow) && (col < p.S);
+          for (int c = 0; c < 32; ++c) {
+            const float lse2 = kDKV ? vb[half * 32 + c] : my_lse;
+            const float dd = kDKV ? vb[64 + half * 32 + c] : my_d;
+            const float pr = fast_exp2(fmaf(s[c], scale2, -lse2));
+            pv[c] = pr;
+            ds[c] = pr * (dp[c] - dd);
           }
-          const float pr = vis ? fast_exp2(fmaf(s[c], scale2, -lse2)) : 0.0f;
-          pv[c] = pr;
-          ds[c] = pr * (dp[c] - dd);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            const int col = c0 + half * 32 + c;
+            const float lse2 = kDKV ? vb[half * 32 + c] : my_lse;
+            const float dd = kDKV ? vb[64 + half * 32 + c] : my_d;
+            // dkv: row = key, column = query; dq: row = query, column = key
+            const bool vis = kDKV ? ((col >= grow) && (grow < p.S)) : ((col <= grow) && (col < p.S));
+            const float pr = vis ? fast_exp2(fmaf(s[c], scale2, -lse2)) : 0.0f;
+            pv[c] = pr;
+            ds[c] = pr * (dp[c] - dd);
+          }
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -330,7 +337,14 @@ bool attention_bwd_tc(Launcher& lc, const AttnArgs& a, int* status_word) {
   }
   AttnTcParams p;
   p.S = a.seq; p.H = a.heads; p.B = a.batch;
-  p.lse = a.lse; p.drow = a.delta_rows;
+  p.lse = a.lse;
+  if (a.d_stats) {  // float2 {sum dO, sum dO * O} per token and 64-column slot: the .y of slot `head`
+    p.drow = reinterpret_cast<const float*>(a.d_stats) + 1;
+    p.d_sb = (int64_t)a.seq * a.d_slots * 2; p.d_sh = 2; p.d_sq = (int64_t)a.d_slots * 2;
+  } else {
+    p.drow = a.delta_rows;
+    p.d_sb = (int64_t)a.heads * a.seq; p.d_sh = a.seq; p.d_sq = 1;
+  }
   p.scale = 1.0f / sqrtf((float)DH);
   p.status = status_word;
   dim3 grid((a.seq + BIG - 1) / BIG, a.heads, a.batch);

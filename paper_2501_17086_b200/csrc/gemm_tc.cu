@@ -285,7 +285,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) mbar_arrive(acce_bar(acc));
       } else {
         bool ok = true;
-        float s1 = 0.0f, s2 = 0.0f;  // EPI_STORE_LN: row sums of acc and acc * E over this warp's 128 columns
+        float s1 = 0.0f, s2 = 0.0f;  // EPI_STORE_LN: row sums of acc and acc * E over the current 64 columns
 #pragma unroll 1
         for (int c = 0; c < nchunks; ++c) {
           float v[64];
@@ -326,6 +326,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
               }
             }
+          }
+          if (p.epi == EPI_STORE_LN) {  // one slot of row sums per 64 columns
+            if (row0 + lane < p.M)
+              p.stats[(int64_t)b * p.stats_sb + (int64_t)(row0 + lane) * (4 * p.n_tiles) + 4 * (n0 / BN) + 2 * half + c] =
+                  make_float2(s1, s2);
+            s1 = s2 = 0.0f;
           }
           if (p.d_f32) {
 #pragma unroll
@@ -370,9 +376,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           __syncwarp();
         }
         if (!ok) break;
-        if (p.epi == EPI_STORE_LN && row0 + lane < p.M)
-          p.stats[(int64_t)b * p.stats_sb + (int64_t)(row0 + lane) * (2 * p.n_tiles) + 2 * (n0 / BN) + half] =
-              make_float2(s1, s2);
       }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
@@ -473,7 +476,7 @@ int sm_count() {
 
 }  // namespace tc
 
-int gemm_tc_stats_slots(int N) { return 2 * ((N + BN - 1) / BN); }
+int gemm_tc_stats_slots(int N) { return 4 * ((N + BN - 1) / BN); }
 
 bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   if (!status_word) return false;

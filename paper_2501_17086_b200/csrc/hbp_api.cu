@@ -70,6 +70,8 @@ struct hbp_ctx {
   char* dO = nullptr;      // [Lb][N][d]
   char* dQKV = nullptr;    // [Lb][N][3d]
   float* drow = nullptr;   // [Lb][B][H][S]
+  float2* dopart = nullptr;  // [Lb][N][do_slots] row sums of dO and dO * O per 64 columns (= per head)
+  int do_slots = 0;
 };
 
 namespace {
@@ -166,6 +168,10 @@ size_t carve(hbp_ctx* c, char* base) {
     c->dO = take(Lb * N * d * es);
     c->dQKV = take(Lb * N * 3 * d * es);
     c->drow = (float*)take(Lb * (size_t)f.batch * f.n_heads * f.seq * 4);
+    if (f.dtype == HBP_BF16 && f.head_dim == 64) {
+      c->do_slots = gemm_tc_stats_slots(f.d);
+      c->dopart = (float2*)take(Lb * N * c->do_slots * sizeof(float2));
+    }
   }
   c->partial = (float*)take(c->partial_floats * 4);
   return off;
@@ -276,7 +282,12 @@ struct Run {
     a.B = at(p->Wo, (int64_t)b0 * d * d); a.b_sn = 1; a.b_sk = d; a.b_sb = d * d;
     a.epi = EPI_STORE;
     a.D = at(c->dO, (int64_t)b0 * state); a.ldd = d; a.d_sb = state;
-    run_gemm(a);
+    if (c->dopart) {  // also the per-head row sums of dO * O that the attention backward needs
+      a.epi = EPI_STORE_LN;
+      a.E = at(c->O, (int64_t)b0 * state); a.lde = d; a.e_sb = state;
+      a.stats = c->dopart + (int64_t)b0 * N * c->do_slots; a.stats_sb = N * c->do_slots;
+    }
+    const bool do_tc = run_gemm(a);
     AttnArgs t;
     t.dtype = f.dtype; t.batch = nb * f.batch; t.seq = f.seq; t.heads = f.n_heads; t.head_dim = f.head_dim;
     t.qkv = at(c->QKV, (int64_t)b0 * 3 * state);
@@ -286,6 +297,7 @@ struct Run {
     t.d_qkv = at(c->dQKV, (int64_t)b0 * 3 * state);
     t.delta_rows = c->drow + (int64_t)b0 * f.batch * f.n_heads * f.seq;
     t.status = c->status;
+    if (c->dopart && do_tc) { t.d_stats = c->dopart + (int64_t)b0 * N * c->do_slots; t.d_slots = c->do_slots; }
     attention_bwd(lc, t);
     if (!want_dy) return;
     GemmArgs b = base_args();  // dY = [dQ dK dV] [Wq; Wk; Wv]

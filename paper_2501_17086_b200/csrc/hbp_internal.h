@@ -19,7 +19,7 @@ enum Epilogue {
   EPI_RESID = 2,     // v = gate[n] * r + acc with r = R ? R[m,n] : E[m,n];  R = v (if R);  D = v
   EPI_MUL = 3,       // D = acc * E[m,n]   (dZ = dA * gelu'(Z) with the cached derivative)
   EPI_AFFINE = 4,    // D = (E ? E[m,n] : 0) + gate[n] * E2[m,n] + acc
-  EPI_STORE_LN = 6,  // D = acc, plus per-row partial sums (sum acc, sum acc * E[m,n]) per 128 columns -> stats
+  EPI_STORE_LN = 6,  // D = acc, plus per-row partial sums (sum acc, sum acc * E[m,n]) per 64 columns -> stats
   EPI_ADD = 7,       // D = acc + E[m,n]   (u_t + delta_t: the scan then reads one tensor less)
   EPI_RNN_FWD = 5,   // c = tanh(acc + E[m,n]);  D2 = 1 - c^2;  D = gate[n] * E2[m,n] + c
 };
@@ -79,7 +79,7 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word);
 // Picks gemm_tc when it applies, else gemm_simt (EPI_STORE_LN then degrades to EPI_STORE); returns
 // whether the tensor-core kernel ran.
 bool gemm(Launcher& lc, const GemmArgs& g, int* status_word);
-// Number of 128-column slots of partial sums the tensor-core kernel writes per row for N columns.
+// Number of 64-column slots of partial sums the tensor-core kernel writes per row for N columns.
 int gemm_tc_stats_slots(int N);
 // Set from the environment variable HBP_FORCE_SIMT=1 when a context is created: keeps every GEMM
 // on the CUDA-core kernel (used to cross-check the tensor-core kernel).
@@ -149,6 +149,10 @@ struct AttnArgs {
   const void* d_o = nullptr;
   void* d_qkv = nullptr;        // [tokens][3d]
   float* delta_rows = nullptr;  // scratch [batch][heads][seq]: rowsum(dO * O)
+  // If set (head dimension 64 only): rowsum(dO * O) already sits in the .y of d_stats[token][d_slots + head],
+  // written by the epilogue of the GEMM that produced dO; the row-dot pass is then skipped.
+  const float2* d_stats = nullptr;
+  int d_slots = 0;
   int* status = nullptr;        // device status word for the bounded waits of the tensor-core kernels
 };
 void attention_fwd(Launcher& lc, const AttnArgs& a);
