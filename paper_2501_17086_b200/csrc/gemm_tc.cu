@@ -165,7 +165,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
         const int zc = tile / tiles_per_batch, r = tile % tiles_per_batch;
         const int b = zc % p.batch, split = zc / p.batch;
-        const int m0 = (r % p.m_tiles) * BM, n0 = (r / p.m_tiles) * BN;
+        const int m0 = (r / p.n_tiles) * BM, n0 = (r % p.n_tiles) * BN;  // n fastest: a wave shares few A row-panels
         const int kb_lo = split * p.kb_per_split, kb_hi = min(p.k_blocks, kb_lo + p.kb_per_split);
         for (int seg = 0; seg < p.segs && ok; ++seg) {
           const CUtensorMap* mA = seg == 0 ? &tmA : (seg == 1 ? &tmA1 : &tmA2);
@@ -263,7 +263,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
       // b indexes the outputs: with split-K it is split * batch + batch entry (partial sums [split][batch][M][N])
       const int b = tile / tiles_per_batch, r = tile % tiles_per_batch;
-      const int m0 = (r % p.m_tiles) * BM, n0 = (r / p.m_tiles) * BN;
+      const int m0 = (r / p.n_tiles) * BM, n0 = (r % p.n_tiles) * BN;  // n fastest: a wave shares few A row-panels
       const int row0 = m0 + quarter * 32, colw = n0 + half * 128;
       if (has_e && lane == 0) {  // the buffer is free here: fetch the first chunk of E while the MMAs still run
         mbar_expect_tx(ebar, EPI_BUF_BYTES);
