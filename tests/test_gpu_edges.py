@@ -1,0 +1,136 @@
+"""Edge cases of the CUDA path through the C ABI: the scan on its own against the oracle's recurrence, gated
+MLP stacks (shared and per-step gates, loss on every state), degenerate sizes, and the error statuses."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import hbp_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+def rel(a, b):
+    nb = np.linalg.norm(b)
+    return float(np.linalg.norm(np.asarray(a, dtype=np.float64).reshape(b.shape) - b) / nb) if nb else float(np.linalg.norm(a))
+
+
+def np64(t):
+    return t.detach().float().cpu().double().numpy()
+
+
+@pytest.mark.parametrize("dtype,L,rows,d,gate,every", [
+    (torch.float32, 1, 1, 4, None, False),            # a single step, a single row
+    (torch.float32, 7, 3, 12, "shared", True),
+    (torch.float32, 300, 5, 64, "shared", True),      # time-chunked, ragged last chunk
+    (torch.float32, 257, 2, 32, "per_step", True),    # time-chunked with a gate per step
+    (torch.float32, 40, 700, 256, None, False),       # depth scan, many channels
+    (torch.bfloat16, 33, 130, 128, "per_step", False),
+    (torch.bfloat16, 200, 4, 64, "shared", True),     # time-chunked in bf16
+])
+def test_cumsumprod_matches_the_recurrence(dtype, L, rows, d, gate, every):
+    from paper_2501_17086_b200 import binding as B
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(L * 1000 + rows)
+    u = torch.randn((L, rows, d), generator=gen, device="cuda").to(dtype)
+    delta = torch.randn((L + 1, rows, d) if every else (rows, d), generator=gen, device="cuda").to(dtype)
+    a = None
+    if gate == "shared":
+        a = (0.8 + 0.25 * torch.rand((d,), generator=gen, device="cuda")).to(dtype)
+    elif gate == "per_step":
+        a = (0.8 + 0.25 * torch.rand((L, d), generator=gen, device="cuda")).to(dtype)
+    g = B.cumsumprod(u, delta, a, loss=B.LOSS_EVERY_STEP if every else B.LOSS_FINAL)
+    torch.cuda.synchronize()
+    # oracle: Eq. 9 solved in order on v_l = u_l + delta_l, with the carry delta_L beyond the last step
+    dl = np64(delta)
+    v = [np64(u[l]) + (dl[l] if every else 0.0) for l in range(L)] + [dl[L] if every else dl]
+    gates = [(1.0 if a is None else np64(a if a.dim() == 1 else a[l])) for l in range(L)] + [1.0]
+    ref = O.cumsumprod_sequential(v, gates)
+    tol = 1e-6 if dtype == torch.float32 else 6e-3      # bf16: one rounding of the stored g_l
+    for l in range(L + 1):
+        assert rel(np64(g[l]), ref[l]) < tol, l
+
+
+@pytest.mark.parametrize("dtype,gate", [("f32", "shared"), ("f32", "per_step"), ("bf16", "per_step")])
+def test_gated_mlp_stack_with_losses_on_every_state(dtype, gate):
+    from paper_2501_17086_b200 import binding as B
+    L, d, h, N = 4, 64, 96, 40
+    dt = torch.float32 if dtype == "f32" else torch.bfloat16
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(77)
+    W1 = (torch.randn((L, h, d), generator=gen, device="cuda") / d ** 0.5).to(dt)
+    W2 = (torch.randn((L, d, h), generator=gen, device="cuda") / h ** 0.5 * 0.5).to(dt)
+    a = (0.7 + 0.3 * torch.rand((d,) if gate == "shared" else (L, d), generator=gen, device="cuda")).to(dt)
+    x0 = torch.randn((N, d), generator=gen, device="cuda").to(dt)
+    delta = torch.randn((L + 1, N, d), generator=gen, device="cuda").to(dt)
+    cfg = B.make_config("preln_mlp", dtype, L, d, N, hidden=h,
+                        gate=B.GATE_CHANNEL_SHARED if gate == "shared" else B.GATE_CHANNEL_PER_STEP, loss=B.LOSS_EVERY_STEP)
+    ctx = B.Context(cfg)
+    params = {"W1": W1, "W2": W2, "a": a}
+    x_all = ctx.forward(params, x0)
+    got, grads = {}, {}
+    for k in (0, 1, 2, 9):
+        grads[k] = ctx.new_grads(with_gate=True)
+        got[k] = ctx.backward(params, k, delta, x_all, grads=grads[k]).clone()
+    ge = ctx.exact(params, delta, x_all)
+    ctx.sync_status()
+    gates = [np64(a) if gate == "shared" else np64(a[l]) for l in range(L)]
+    steps = [O.MLPStep(np64(W1[l]), np64(W2[l]), True) for l in range(L)]
+    stack = O.Stack(steps, gates, gate_shared=(gate == "shared"))
+    xs, caches = O.forward(stack, np64(x0))
+    deltas = [np64(delta[l]) for l in range(L + 1)]
+    tol = 1e-5 if dtype == "f32" else 2e-2
+    exact = O.exact_bp(stack, caches, deltas)
+    for l in range(L + 1):
+        assert rel(np64(x_all[l]), xs[l]) < tol
+        assert rel(np64(ge[l]), exact[l]) < tol
+    for k in (0, 1, 2, 9):
+        ref = O.highway_bp(stack, caches, deltas, k)
+        assert max(rel(np64(got[k][l]), ref[l]) for l in range(L + 1)) < tol, k
+    ref = O.highway_bp(stack, caches, deltas, 2)
+    pg = O.param_grads(stack, caches, xs, ref, [("", l) for l in range(L)])
+    assert rel(np64(grads[2]["dW1"]), pg["W1"]) < tol and rel(np64(grads[2]["dW2"]), pg["W2"]) < tol
+    if gate == "shared":
+        assert rel(np64(grads[2]["da"]), pg["a"]) < tol
+    else:
+        da = np.stack([(ref[l + 1] * xs[l]).sum(axis=0) for l in range(L)])
+        assert rel(np64(grads[2]["da"]), da) < tol
+
+
+def test_error_statuses_on_the_device():
+    from paper_2501_17086_b200 import binding as B
+    cfg = B.make_config("mlp", "f32", 3, 16, 8, hidden=32)
+    ctx = B.Context(cfg)
+    W1 = torch.zeros((3, 32, 16), device="cuda")
+    W2 = torch.zeros((3, 16, 32), device="cuda")
+    params = {"W1": W1, "W2": W2}
+    x0 = torch.zeros((8, 16), device="cuda")
+    x_all = ctx.new_states()
+    with pytest.raises(B.HbpError) as e:          # backward before any forward
+        ctx.backward(params, 1, x0, x_all)
+    assert e.value.code == 4
+    ctx.forward(params, x0, x_all=x_all)
+    with pytest.raises(B.HbpError) as e:          # negative k
+        ctx.backward(params, -1, x0, x_all)
+    assert e.value.code == 1
+    with pytest.raises(B.HbpError) as e:          # no delta
+        ctx.backward(params, 1, None, x_all)
+    assert e.value.code == 1
+    mis = torch.zeros(8 * 16 + 1, device="cuda")[1:].view(8, 16)   # 4-byte aligned only
+    with pytest.raises(B.HbpError) as e:
+        ctx.backward(params, 1, mis, x_all)
+    assert e.value.code == 2
+    with pytest.raises(B.HbpError) as e:          # parameter gradients asked for but a buffer is missing
+        ctx.backward(params, 1, x0, x_all, grads={"dW1": torch.zeros_like(W1)})
+    assert e.value.code == 1
+    need = B.workspace_bytes(cfg)                 # workspace too small / misaligned
+    ws = torch.empty(need + 512, dtype=torch.uint8, device="cuda")
+    base = (ws.data_ptr() + 255) // 256 * 256
+    h = C.c_void_p()
+    assert B.lib.hbp_create(C.byref(cfg), C.c_void_p(base), need - 1, C.byref(h)) == 5
+    assert B.lib.hbp_create(C.byref(cfg), C.c_void_p(base + 8), need, C.byref(h)) == 5
+    ctx.sync_status()                             # the context is still usable and clean
+    g = ctx.backward(params, 5, x0, x_all)        # zero weights: every g_l is delta_L (Eq. 5 with a = 1)
+    torch.cuda.synchronize()
+    assert torch.equal(g, x0.expand_as(g))
