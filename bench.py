@@ -77,7 +77,11 @@ def oracle_timing(w, k, sample, steps, warmup):
         threads = len(os.sched_getaffinity(0))
     inp = make_inputs(w, "cpu")
     # full float64 copies of the weights once, so that a step times the method and not dtype conversion
-    inp64 = {n: (t.double() if n in ("W1", "W2", "Wq", "Wk", "Wv", "Wo", "W", "U", "a") else t) for n, t in inp.items()}
+    weights = ("W1", "W2", "Wq", "Wk", "Wv", "Wo", "W", "U", "a")
+    if sum(t.numel() for n, t in inp.items() if n in weights) < 1.5e9:
+        inp64 = {n: (t.double() if n in weights else t) for n, t in inp.items()}
+    else:  # too large to hold in float64 at once: converted layer by layer inside the timed calls
+        inp64 = inp
     units = {"preln_transformer": w.batch, "rnn_tanh": w.batch}.get(w.block, w.tokens)
     sample = min(sample, units)
     times = []
