@@ -5,7 +5,7 @@
 // are bitwise reproducible):
 //   attn_dkv_kernel  one CTA per 128 keys; loops over blocks of 64 queries that can see them:
 //                       S^T = K Q^T, dP^T = V dO^T            (tcgen05.mma 128x64x16, accumulators in TMEM)
-//                       P^T = exp(S^T/sqrt(dh) - lse), dS^T = P^T * (dP^T - D)   (4 warps, one key row per lane)
+//                       P^T = exp(S^T/sqrt(dh) - lse), dS^T = P^T * (dP^T - D)   (8 warps, one key row per lane, 32 query columns per thread)
 //                       dV += P^T dO,  dK += dS^T Q           (P^T, dS^T go back through shared memory as bf16)
 //   attn_dq_kernel   one CTA per 128 queries; loops over blocks of 64 keys up to the diagonal:
 //                       S = Q K^T, dP = dO V^T, dS = P * (dP - D),  dQ += dS K
@@ -24,7 +24,8 @@ namespace {
 constexpr int DH = 64;
 constexpr int BIG = 128, SMALL = 64;
 constexpr int BIG_BYTES = BIG * DH * 2, SMALL_BYTES = SMALL * DH * 2, PS_BYTES = BIG * SMALL * 2;
-constexpr int THREADS = 192;  // warp 0 TMA, warp 1 MMA, warps 2..5 softmax / epilogue
+constexpr int THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2..9 softmax / epilogue (two warps per TMEM lane quarter)
+constexpr int SOFTMAX_WARPS = 8;
 constexpr uint32_t TMEM_COLS = 256;
 constexpr float LOG2E = 1.4426950408889634f;
 
@@ -42,7 +43,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ void named_barrier_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void named_barrier_softmax() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 64, A K-major, B K-major or MN-major
 constexpr uint32_t make_idesc(int b_mn) {
@@ -52,7 +53,8 @@ constexpr uint32_t make_idesc(int b_mn) {
 constexpr uint32_t IDESC_KK = make_idesc(0), IDESC_KMN = make_idesc(1);
 
 // Barrier slots (8 bytes each):
-// 0 big tiles loaded, 1-2 full[2], 3-4 empty[2], 5 scores ready, 6 probabilities ready, 7 all MMAs done.
+// 0 big tiles loaded, 1-2 full[2], 3-4 empty[2], 5 scores ready, 6 probabilities ready, 7 all MMAs done,
+// 8 scores copied out of tensor memory (the next block's score MMAs may overwrite them).
 __device__ __forceinline__ uint32_t bar_at(uint32_t bars, int i) { return bars + 8u * i; }
 
 template <bool kDKV>
@@ -74,7 +76,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
   float* vec = reinterpret_cast<float*>(aligned + VEC_OFF);  // [2 buffers][lse 64 | D 64]
   uint64_t* bar_mem = reinterpret_cast<uint64_t*>(aligned + VEC_OFF + 1024);
   const uint32_t bars = smem_u32(bar_mem);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 10);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -93,8 +95,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
     mbar_init(bar_at(bars, 3), 1);
     mbar_init(bar_at(bars, 4), 1);
     mbar_init(bar_at(bars, 5), 1);
-    mbar_init(bar_at(bars, 6), 4);
+    mbar_init(bar_at(bars, 6), SOFTMAX_WARPS);
     mbar_init(bar_at(bars, 7), 1);
+    mbar_init(bar_at(bars, 8), SOFTMAX_WARPS);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -144,13 +147,11 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      bool ok = mbar_wait(bar_at(bars, 0), 0, abort_flag, p.status);
-      tc_fence_after();
-      for (int it = 0; it < n_it && ok; ++it) {
+      // Software pipeline: the score MMAs of block it+1 are issued as soon as the softmax warps have copied the
+      // scores of block it out of tensor memory, so they run under the exp / pack work of block it; the
+      // accumulating MMAs of block it follow once its probabilities are in shared memory.
+      auto issue_scores = [&](int it) {
         const int buf = it & 1;
-        const uint32_t ph = (uint32_t)(it >> 1) & 1u, itp = (uint32_t)it & 1u;
-        if (!mbar_wait(bar_at(bars, 1 + buf), ph, abort_flag, p.status)) { ok = false; break; }
-        tc_fence_after();
         const uint32_t s0 = sSmall + (2 * buf) * SMALL_BYTES, s1 = s0 + SMALL_BYTES;
         // scores and dP: contraction over the head dimension, both operands K-major
 #pragma unroll
@@ -160,6 +161,22 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
         for (int k = 0; k < DH / 16; ++k)
           tc_mma(tDP, make_desc(sBig1 + 32 * k, 16, 1024), make_desc(s1 + 32 * k, 16, 1024), IDESC_KK, k != 0);
         tc_commit(bar_at(bars, 5));
+      };
+      bool ok = mbar_wait(bar_at(bars, 0), 0, abort_flag, p.status);
+      ok = ok && mbar_wait(bar_at(bars, 1), 0, abort_flag, p.status);
+      tc_fence_after();
+      if (ok) issue_scores(0);
+      for (int it = 0; it < n_it && ok; ++it) {
+        const int buf = it & 1;
+        const uint32_t itp = (uint32_t)it & 1u;
+        if (it + 1 < n_it) {
+          const int nb = (it + 1) & 1;
+          if (!mbar_wait(bar_at(bars, 1 + nb), (uint32_t)((it + 1) >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+          if (!mbar_wait(bar_at(bars, 8), itp, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          issue_scores(it + 1);
+        }
+        const uint32_t s0 = sSmall + (2 * buf) * SMALL_BYTES, s1 = s0 + SMALL_BYTES;
         if (!mbar_wait(bar_at(bars, 6), itp, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         // accumulate: contraction over the 64 rows of the small tiles, which are MN-major B operands here
@@ -190,7 +207,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
     }
   } else {
     // ------------------------------------------------------------------ softmax and epilogue (128 threads)
-    const int t = threadIdx.x - 64;             // 0..127
+    const int t = threadIdx.x - 64;             // 0..255
+    const int ch = (warp - 2) >> 2;             // which 32 of the block's 64 columns this warp handles
     const int quarter = warp & 3;               // TMEM lane quarter this warp may read
     const int row = quarter * 32 + lane;        // row of the big tile (key for dkv, query for dq)
     const int grow = big0 + row;                // its index in the sequence
@@ -209,47 +227,53 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
       if (kDKV) {  // statistics of the 64 queries of this block, shared by all rows
         const int q = c0 + (t & 63);
         if (t < 64) vb[t] = q < p.S ? p.lse[stat_base + q] * LOG2E : INFINITY;
-        else vb[t] = q < p.S ? p.drow[(int64_t)b * p.d_sb + (int64_t)h * p.d_sh + (int64_t)q * p.d_sq] : 0.0f;
-        named_barrier_128();
+        else if (t < 128) vb[t] = q < p.S ? p.drow[(int64_t)b * p.d_sb + (int64_t)h * p.d_sh + (int64_t)q * p.d_sq] : 0.0f;
+        named_barrier_softmax();
       }
       if (!ok) continue;
       if (!mbar_wait(bar_at(bars, 5), (uint32_t)it & 1u, abort_flag, p.status)) { ok = false; continue; }
       tc_fence_after();
+      // copy this warp's 32 score columns out of tensor memory and release it for the next block's score MMAs
+      float sc[32], dp[32];
+      tc_ld32_async(tS + lane_addr + ch * 32, sc);
+      tc_ld32_async(tDP + lane_addr + ch * 32, dp);
+      tc_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_at(bars, 8));
       // only blocks that touch the diagonal (or the end of the sequence) need the per-element mask
       const bool full = kDKV ? (c0 >= big0 + BIG - 1 && big0 + BIG <= p.S) : (c0 + SMALL - 1 <= big0 && c0 + SMALL <= p.S);
-#pragma unroll 1
-      for (int half = 0; half < 2; ++half) {
-        float s[32], dp[32];
-        tc_ld32(tS + lane_addr + half * 32, s);
-        tc_ld32(tDP + lane_addr + half * 32, dp);
-        float pv[32], ds[32];
-        if (full) {
+      if (full) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const float lse2 = kDKV ? vb[half * 32 + c] : my_lse;
-            const float dd = kDKV ? vb[64 + half * 32 + c] : my_d;
-            const float pr = fast_exp2(fmaf(s[c], scale2, -lse2));
-            pv[c] = pr;
-            ds[c] = pr * (dp[c] - dd);
-          }
-        } else {
-#pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const int col = c0 + half * 32 + c;
-            const float lse2 = kDKV ? vb[half * 32 + c] : my_lse;
-            const float dd = kDKV ? vb[64 + half * 32 + c] : my_d;
-            // dkv: row = key, column = query; dq: row = query, column = key
-            const bool vis = kDKV ? ((col >= grow) && (grow < p.S)) : ((col <= grow) && (col < p.S));
-            const float pr = vis ? fast_exp2(fmaf(s[c], scale2, -lse2)) : 0.0f;
-            pv[c] = pr;
-            ds[c] = pr * (dp[c] - dd);
-          }
+        for (int c = 0; c < 32; ++c) {
+          const float lse2 = kDKV ? vb[ch * 32 + c] : my_lse;
+          const float dd = kDKV ? vb[64 + ch * 32 + c] : my_d;
+          const float pr = fast_exp2(fmaf(sc[c], scale2, -lse2));
+          sc[c] = pr;
+          dp[c] = pr * (dp[c] - dd);
         }
+      } else {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (kDKV) st_shared16(swz(sP, row, half * 4 + u), pack8(pv + 8 * u));
-          st_shared16(swz(sDS, row, half * 4 + u), pack8(ds + 8 * u));
+        for (int c = 0; c < 32; ++c) {
+          const int col = c0 + ch * 32 + c;
+          const float lse2 = kDKV ? vb[ch * 32 + c] : my_lse;
+          const float dd = kDKV ? vb[64 + ch * 32 + c] : my_d;
+          // dkv: row = key, column = query; dq: row = query, column = key
+          const bool vis = kDKV ? ((col >= grow) && (grow < p.S)) : ((col <= grow) && (col < p.S));
+          const float pr = vis ? fast_exp2(fmaf(sc[c], scale2, -lse2)) : 0.0f;
+          sc[c] = pr;
+          dp[c] = pr * (dp[c] - dd);
         }
+      }
+      // the accumulating MMAs of the previous block read the probability tiles: wait until they are done
+      if (it > 0 && !mbar_wait(bar_at(bars, 3 + ((it - 1) & 1)), (uint32_t)((it - 1) >> 1) & 1u, abort_flag, p.status)) {
+        ok = false;
+        continue;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (kDKV) st_shared16(swz(sP, row, ch * 4 + u), pack8(sc + 8 * u));
+        st_shared16(swz(sDS, row, ch * 4 + u), pack8(dp + 8 * u));
       }
       fence_async_smem();
       tc_fence_before();
@@ -264,19 +288,16 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
       for (int o = 0; o < (kDKV ? 2 : 1); ++o) {
         const uint32_t dst = o == 0 ? sDS : sP;          // staging: the probability tiles are free now
         const float mul = o == 0 ? p.scale : 1.0f;       // dK and dQ carry the 1/sqrt(dh) factor, dV does not
-#pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-          float v[32];
-          tc_ld32((o == 0 ? tAcc0 : tAcc1) + lane_addr + half * 32, v);
+        float v[32];
+        tc_ld32((o == 0 ? tAcc0 : tAcc1) + lane_addr + ch * 32, v);
 #pragma unroll
-          for (int c = 0; c < 32; ++c) v[c] *= mul;
+        for (int c = 0; c < 32; ++c) v[c] *= mul;
 #pragma unroll
-          for (int u = 0; u < 4; ++u) st_shared16(swz(dst, row, half * 4 + u), pack8(v + 8 * u));
-        }
+        for (int u = 0; u < 4; ++u) st_shared16(swz(dst, row, ch * 4 + u), pack8(v + 8 * u));
       }
       fence_async_smem();
     }
-    named_barrier_128();
+    named_barrier_softmax();
     if (t == 0 && ok) {
       tma_store_4d(&tmOut0, sDS, 0, big0, h, b);
       if (kDKV) tma_store_4d(&tmOut1, sP, 0, big0, h, b);

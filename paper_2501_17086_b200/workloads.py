@@ -59,6 +59,9 @@ WORKLOADS = {
     "c5": Workload("c5", "preln_mlp", "bf16", L=128, d=2048, hidden=8192, batch=32, seq=512, tokens=16384, seed=1005),
     # c2 with 8 layers: same per-launch tile shapes, small enough for multi-pass profiler captures
     "c2_small": Workload("c2_small", "preln_mlp", "bf16", L=8, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1012),
+    # c4 with 4 decoder blocks: same per-launch shapes, small enough for multi-pass profiler captures
+    "c4_small": Workload("c4_small", "preln_transformer", "bf16", L=4, d=768, hidden=3072, n_heads=12, head_dim=64,
+                         seq=1024, batch=16, tokens=16384, seed=1014),
     # reduced twins: same structure, sizes the fp64 oracle runs in full; they
     # span several tiles and leave ragged tails against 128/256-wide tiles.
     "c2_twin": Workload("c2_twin", "preln_mlp", "bf16", L=5, d=256, hidden=1024, batch=1, seq=328, tokens=328, seed=2002),
