@@ -15,6 +15,12 @@
  * blocks; it is the exact gradient for l >= L-k, and everywhere once k >= L.
  * Parameter gradients use the final estimate (last sentence of Section 4.2).
  *
+ * Shifted split (Appendix C.3, Eq. 17): with cfg.gamma > 0 (plain residual connections only, cfg.gate ==
+ * HBP_GATE_ONE) a layer x + Block(x) is split as r(x, z) = (1 - gamma) x + z around g(x) = Block(x) + gamma x: the
+ * forward pass and exact backpropagation are unchanged, while every Highway-BP iteration uses K = (1 - gamma) I and
+ * adds gamma g_{l+1} (from the previous iterate) to each block VJP.  gamma = 1 is the fixed-point iteration of
+ * Section 5.2.1.
+ *
  * Conventions
  *  - Every pointer named below is a DEVICE pointer unless it says "host".
  *    All device buffers are allocated and owned by the caller and are only
@@ -82,7 +88,7 @@ typedef struct {
   int32_t batch;    /* Transformer: sequences; RNN: rows (== tokens) */
   int64_t tokens;   /* N: rows of one state */
   float ln_eps;
-  int32_t reserved;
+  float gamma;      /* shift of the residual split, 0 <= gamma <= 1 (Appendix C.3, Eq. 17); 0 = the plain split */
 } hbp_config;
 
 /* Borrowed parameter pointers; those the block kind does not use are ignored.

@@ -185,6 +185,32 @@ class RNNStep:
         return {"W": dz.T @ cache["h"], "U": dz.T @ _f64(self.x_t)}
 
 
+class ShiftedStep:
+    """The gamma-shifted split of a residual layer x + Block(x) (Appendix C.3, Eq. 17): the block becomes
+    g(x) = Block(x) + gamma x and the residual function r(x, z) = (1 - gamma) x + z, so the layer itself is
+    unchanged while J gains gamma I and K becomes (1 - gamma) I."""
+
+    def __init__(self, step, gamma):
+        self.step, self.gamma = step, float(gamma)
+
+    def forward(self, x):
+        f, cache = self.step.forward(x)
+        return f + self.gamma * x, cache
+
+    def vjp(self, cache, g):
+        return self.step.vjp(cache, g) + self.gamma * g
+
+    def param_vjp(self, cache, g):
+        return self.step.param_vjp(cache, g)
+
+
+def shifted_stack(stack, gamma):
+    """Same network as ``stack`` (all gates 1), split with the shift gamma."""
+    if any(a is not None for a in stack.gates):
+        raise ValueError("the shift is defined for plain residual connections")
+    return Stack([ShiftedStep(st, gamma) for st in stack.steps], [1.0 - float(gamma)] * stack.L)
+
+
 class Stack:
     """L residual steps x_{l+1} = a_l * x_l + f_l(x_l).
 

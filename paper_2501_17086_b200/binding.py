@@ -35,7 +35,7 @@ class hbp_config(C.Structure):
     _fields_ = [("block", C.c_int32), ("dtype", C.c_int32), ("gate", C.c_int32), ("loss", C.c_int32),
                 ("L", C.c_int32), ("d", C.c_int32), ("hidden", C.c_int32), ("in_dim", C.c_int32),
                 ("n_heads", C.c_int32), ("head_dim", C.c_int32), ("seq", C.c_int32), ("batch", C.c_int32),
-                ("tokens", C.c_int64), ("ln_eps", C.c_float), ("reserved", C.c_int32)]
+                ("tokens", C.c_int64), ("ln_eps", C.c_float), ("gamma", C.c_float)]
 
 
 class hbp_params(C.Structure):
@@ -107,9 +107,9 @@ def _dtype_code(dt):
 
 
 def make_config(block, dtype, L, d, tokens, hidden=0, in_dim=0, n_heads=0, head_dim=0, seq=0, batch=0,
-                gate=GATE_ONE, loss=LOSS_FINAL, ln_eps=1e-5) -> hbp_config:
+                gate=GATE_ONE, loss=LOSS_FINAL, ln_eps=1e-5, gamma=0.0) -> hbp_config:
     return hbp_config(BLOCKS[block], HBP_F32 if dtype in ("f32", torch.float32) else HBP_BF16, gate, loss, L, d,
-                      hidden, in_dim, n_heads, head_dim, seq, batch, tokens, ln_eps, 0)
+                      hidden, in_dim, n_heads, head_dim, seq, batch, tokens, ln_eps, gamma)
 
 
 def config_from_workload(w) -> hbp_config:

@@ -90,6 +90,8 @@ hbp_status check_config(const hbp_config* c) {
   if (c->loss != HBP_LOSS_FINAL && c->loss != HBP_LOSS_EVERY_STEP) return HBP_ERR_UNSUPPORTED;
   const int v = c->dtype == HBP_F32 ? 4 : 8;
   if (c->L <= 0 || c->d <= 0 || c->tokens <= 0) return HBP_ERR_SHAPE;
+  if (!(c->gamma >= 0.0f && c->gamma <= 1.0f)) return HBP_ERR_INVALID_ARG;
+  if (c->gamma != 0.0f && (c->gate != HBP_GATE_ONE || c->block == HBP_BLOCK_RNN_TANH)) return HBP_ERR_UNSUPPORTED;
   if (c->d % v) return HBP_ERR_SHAPE;
   if (c->d / v > 1024) return HBP_ERR_SHAPE;  // one block per row in the LayerNorm kernels
   if (c->block == HBP_BLOCK_RNN_TANH) {
@@ -209,6 +211,7 @@ struct Run {
     return a;
   }
   bool u_has_delta = false;  // the VJP GEMM already added delta_l to u_l
+  bool shifted = false;      // Highway-BP call on a config with gamma > 0 (exact BP ignores the shift)
   bool stats_ok = true;  // every dY GEMM since the last reset also produced the LayerNorm row sums
   bool run_gemm(const GemmArgs& a) { return gemm(lc, a, c->status); }
   hbp_status result() const { return lc.err == cudaSuccess ? HBP_OK : HBP_ERR_CUDA; }
@@ -401,6 +404,10 @@ struct Run {
     s.dtype = c->cfg.dtype; s.L = c->steps; s.l_lo = lo; s.l_hi = hi; s.rows = N; s.d = (int)d;
     s.u = with_u ? c->U : nullptr;
     s.u_has_delta = with_u && u_has_delta;
+    if (shifted) {
+      s.keep = 1.0f - c->cfg.gamma;
+      s.gamma = with_u ? c->cfg.gamma : 0.0f;
+    }
     s.delta = delta; s.loss = c->cfg.loss;
     s.a = p->a; s.gate = c->cfg.gate;
     s.g = g;
@@ -696,6 +703,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
   }
 
   if (!exact) {
+    r.shifted = f.gamma != 0.0f;
     // g^0 = CumSumProd(delta, K) (Eq. 10), then k iterations of {all-step VJP (Eq. 8); reverse scan (Eq. 9, 11)}
     {
       PhaseScope ph(r, HBP_PHASE_OTHER);  // g^0: a scan without VJPs (a broadcast of delta_L when a = 1)

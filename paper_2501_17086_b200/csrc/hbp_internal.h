@@ -93,6 +93,9 @@ struct ScanArgs {
   int64_t rows = 0;
   int d = 0;
   const void* u = nullptr;      // [L][rows][d] or nullptr (zeros)
+  // Shifted split: g_l = delta_l + keep * a_l * g_{l+1} + u_l + gamma * (g_{l+1} of the previous iterate, read from
+  // the g buffer before it is overwritten).  keep = 1 - gamma during Highway-BP, 1 otherwise.
+  float keep = 1.0f, gamma = 0.0f;
   bool u_has_delta = false;     // u[l] already contains delta_l for l < L (added by the producing GEMM)
   const void* delta = nullptr;  // per hbp_loss
   int loss = HBP_LOSS_FINAL;

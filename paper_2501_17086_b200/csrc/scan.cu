@@ -94,7 +94,7 @@ __device__ __forceinline__ void scan_step(const ScanArgs& s, int l, int64_t stat
     for (int i = 0; i < V; ++i) val[i] = a[i] * carry[i];
   } else {
 #pragma unroll
-    for (int i = 0; i < V; ++i) val[i] = carry[i];
+    for (int i = 0; i < V; ++i) val[i] = s.keep * carry[i];
   }
   if (s.u) {
     float u[V];
@@ -125,9 +125,17 @@ __global__ void __launch_bounds__(256) scan_depth_kernel(const ScanArgs s) {
   typedef typename Acc<T>::type A;
   A carry[V];
   ldv<T>(g + (int64_t)s.l_hi * state_elems + off).get(carry);
+  float old_next[V];  // shifted split: g_{l+1} of the previous iterate
+#pragma unroll
+  for (int i = 0; i < V; ++i) old_next[i] = (float)carry[i];
   for (int l = s.l_hi - 1; l >= s.l_lo; --l) {
     A val[V];
     scan_step<T>(s, l, state_elems, off, ch, carry, val);
+    if (s.gamma != 0.0f) {
+#pragma unroll
+      for (int i = 0; i < V; ++i) val[i] += s.gamma * old_next[i];
+      ldv<T>(g + (int64_t)l * state_elems + off).get(old_next);  // before it is overwritten below
+    }
     Vec<T> out;
     out.set(val);
     stv<T>(g + (int64_t)l * state_elems + off, out);
@@ -150,8 +158,10 @@ __global__ void __launch_bounds__(256) scan_depth_lnstat_kernel(const ScanArgs s
   const int64_t row = off / s.d;
   const int ch = (int)(off - row * s.d);
   T* g = (T*)s.g;
-  float carry[V];
+  float carry[V], old_next[V];
   ldv<T>(g + (int64_t)s.l_hi * state_elems + off).get(carry);
+#pragma unroll
+  for (int i = 0; i < V; ++i) old_next[i] = carry[i];
   for (int l = s.l_hi - 1; l >= s.l_lo; --l) {
     float dy[V], xh[V], val[V];
     ldv_stream<T>((const T*)s.u + (int64_t)l * state_elems + off).get(dy);
@@ -165,10 +175,15 @@ __global__ void __launch_bounds__(256) scan_depth_lnstat_kernel(const ScanArgs s
       for (int i = 0; i < V; ++i) val[i] = a[i] * carry[i];
     } else {
 #pragma unroll
-      for (int i = 0; i < V; ++i) val[i] = carry[i];
+      for (int i = 0; i < V; ++i) val[i] = s.keep * carry[i];
     }
 #pragma unroll
     for (int i = 0; i < V; ++i) val[i] += st.x * (dy[i] - st.y - xh[i] * st.z);
+    if (s.gamma != 0.0f) {
+#pragma unroll
+      for (int i = 0; i < V; ++i) val[i] += s.gamma * old_next[i];
+      ldv<T>(g + (int64_t)l * state_elems + off).get(old_next);
+    }
     const T* dp = delta_at<T>(s, l, state_elems);
     if (dp) {
       float dl[V];
@@ -210,11 +225,12 @@ __global__ void __launch_bounds__(1024) scan_depth_ln_kernel(const ScanArgs s) {
   const int64_t state_elems = s.rows * s.d;
   const int64_t off = row * s.d + (int64_t)threadIdx.x * V;
   T* g = (T*)s.g;
-  float carry[V], dy[V], xh[V];
+  float carry[V], dy[V], xh[V], old_next[V];
 #pragma unroll
-  for (int i = 0; i < V; ++i) carry[i] = dy[i] = xh[i] = 0.0f;
+  for (int i = 0; i < V; ++i) carry[i] = dy[i] = xh[i] = old_next[i] = 0.0f;
   if (active) {
     ldv<T>(g + (int64_t)s.l_hi * state_elems + off).get(carry);
+    ldv<T>(g + (int64_t)s.l_hi * state_elems + off).get(old_next);
     ldv_stream<T>((const T*)s.u + (int64_t)(s.l_hi - 1) * state_elems + off).get(dy);
     ldv_stream<T>((const T*)s.xhat + (int64_t)(s.l_hi - 1) * state_elems + off).get(xh);
   }
@@ -262,10 +278,15 @@ __global__ void __launch_bounds__(1024) scan_depth_ln_kernel(const ScanArgs s) {
         for (int i = 0; i < V; ++i) val[i] = a[i] * carry[i];
       } else {
 #pragma unroll
-        for (int i = 0; i < V; ++i) val[i] = carry[i];
+        for (int i = 0; i < V; ++i) val[i] = s.keep * carry[i];
       }
 #pragma unroll
       for (int i = 0; i < V; ++i) val[i] += r * (dy[i] - m1 - xh[i] * m2);
+      if (s.gamma != 0.0f) {
+#pragma unroll
+        for (int i = 0; i < V; ++i) val[i] += s.gamma * old_next[i];
+        ldv<T>(g + (int64_t)l * state_elems + off).get(old_next);
+      }
       const T* dp = delta_at<T>(s, l, state_elems);
       if (dp) {
         float dl[V];
@@ -519,7 +540,7 @@ void scan_reverse(Launcher& lc, const ScanArgs& s) {
   }
   const int steps = s.l_hi - s.l_lo;
   const size_t need = scan_scratch_bytes(s.dtype, steps, s.rows, s.d);
-  if (need > 0 && s.scratch && s.scratch_bytes >= need) {
+  if (need > 0 && s.scratch && s.scratch_bytes >= need && s.keep == 1.0f && s.gamma == 0.0f) {
     const int nchunks = (steps + kChunk - 1) / kChunk;
     dim3 grid((unsigned)((nvec + 127) / 128), nchunks);
     const unsigned cgrid = (unsigned)((s.rows * s.d + 127) / 128);

@@ -134,3 +134,40 @@ def test_error_statuses_on_the_device():
     g = ctx.backward(params, 5, x0, x_all)        # zero weights: every g_l is delta_L (Eq. 5 with a = 1)
     torch.cuda.synchronize()
     assert torch.equal(g, x0.expand_as(g))
+
+
+@pytest.mark.parametrize("name,gamma", [("c2_twin_f32", 0.2), ("c2_twin", 0.2), ("c2_twin_f32", 1.0), ("c4_twin", 0.2), ("c1", 0.5)])
+def test_gamma_shifted_split_matches_oracle(name, gamma):
+    """Appendix C.3, Eq. 17: K = (1 - gamma) I, each VJP gains gamma g_{l+1}; exact BP does not depend on gamma."""
+    from oracle import run as orun
+    from paper_2501_17086_b200 import binding as B, harness
+    from paper_2501_17086_b200.workloads import WORKLOADS, make_inputs
+    w = WORKLOADS[name]
+    inp = make_inputs(w, "cuda")
+    cfg = B.config_from_workload(w)
+    cfg.gamma = gamma
+    ctx = B.Context(cfg)
+    params = harness.params_for(w, inp)
+    x_all = ctx.forward(params, inp["x0"])
+    delta = harness.loss_delta(w, x_all, inp)
+    ks = (0, 1, 2, w.steps)
+    got = {k: ctx.backward(params, k, delta, x_all).clone() for k in ks}
+    grads = ctx.new_grads()
+    ctx.backward(params, 2, delta, x_all, grads=grads)
+    ge = ctx.exact(params, delta, x_all)
+    ctx.sync_status()
+    base, x0, groups = orun.build_stack(w, inp)
+    st = O.shifted_stack(base, gamma)
+    xs, caches = O.forward(st, x0)
+    deltas = orun.loss_deltas(w, xs, inp)
+    tol = 1e-5 if w.dtype == "f32" else 2e-2
+    exact = O.exact_bp(st, caches, deltas)
+    shape = xs[0].shape
+    for k in ks:
+        ref = O.highway_bp(st, caches, deltas, k)
+        worst = max(rel(np64(got[k][l]), ref[l]) for l in range(w.steps + 1))
+        assert worst < tol, (k, worst)
+    assert max(rel(np64(ge[l]), exact[l]) for l in range(w.steps + 1)) < tol
+    pg = O.param_grads(st, caches, xs, O.highway_bp(st, caches, deltas, 2), groups)
+    for n, v in pg.items():
+        assert rel(np64(grads["d" + n]), v) < tol, n

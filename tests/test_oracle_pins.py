@@ -431,3 +431,61 @@ def test_gelu_and_layernorm_pieces():
     xhat, rstd = O.layernorm(x, 1e-5)
     np.testing.assert_allclose(xhat.mean(-1), 0, atol=1e-14)
     np.testing.assert_allclose((xhat ** 2).mean(-1), 1 - 1e-5 * rstd[:, 0] ** 2, rtol=1e-12)
+
+
+# ---------------------------------------------- 10. gamma-shifted split (Appendix C.3)
+def test_gamma_shift_leaves_the_network_and_exact_bp_unchanged():
+    rng = np.random.default_rng(31)
+    L, d = 5, 4
+    base = tiny_stack("preln_mlp", L=L, d=d, gate="one", rng=rng)
+    x0 = rng.normal(size=(2, d))
+    xs0, c0 = O.forward(base, x0)
+    deltas = random_deltas(xs0, every=False, rng=rng)
+    g0 = O.exact_bp(base, c0, deltas)
+    for gamma in (0.0, 0.2, 0.8, 1.0):
+        st = O.shifted_stack(base, gamma)
+        xs, c = O.forward(st, x0)
+        for a, b in zip(xs, xs0):
+            np.testing.assert_allclose(a, b, rtol=1e-13, atol=1e-14)
+        for a, b in zip(O.exact_bp(st, c, deltas), g0):       # Eq. 16 and Eq. 17 agree under backpropagation
+            np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
+        w = O.highway_bp(st, c, deltas, L)                     # and Highway-BP still ends at the exact gradient
+        for a, b in zip(w, g0):
+            np.testing.assert_allclose(a, b, rtol=1e-11, atol=1e-12)
+    for k in (0, 1, 3):                                        # gamma = 0 is the plain split
+        for a, b in zip(O.highway_bp(O.shifted_stack(base, 0.0), c0, deltas, k), O.highway_bp(base, c0, deltas, k)):
+            np.testing.assert_allclose(a, b, rtol=1e-13, atol=1e-14)
+
+
+def test_gamma_one_is_fixed_point_iteration_and_path_sums_hold():
+    rng = np.random.default_rng(32)
+    L, d = 4, 3
+    base = tiny_stack("mlp", L=L, d=d, gate="one", rng=rng)
+    x0 = rng.normal(size=(1, d))
+    xs, _ = O.forward(base, x0)
+    deltas = random_deltas(xs, every=True, rng=rng)
+    J, _ = dense_jacobians(base, xs)                            # block Jacobians by finite differences
+    flat = [x.reshape(-1) for x in deltas]
+    for gamma in (0.3, 1.0):
+        st = O.shifted_stack(base, gamma)
+        _, caches = O.forward(st, x0)
+        Jg = [None] + [J[m] + gamma * np.eye(d) for m in range(1, L + 1)]
+        Kg = [None] + [(1.0 - gamma) * np.eye(d)] * L
+        for k in range(L + 1):
+            w = O.highway_bp(st, caches, deltas, k)
+            for i in range(L + 1):
+                np.testing.assert_allclose(w[i].reshape(-1), O.path_sum(flat, Jg, Kg, i, k), rtol=1e-6, atol=1e-8)
+    # gamma = 1: K = 0, every iteration is one more step of plain backpropagation from each loss (Section 5.2.1)
+    st = O.shifted_stack(base, 1.0)
+    _, caches = O.forward(st, x0)
+    full = [None] + [J[m] + np.eye(d) for m in range(1, L + 1)]
+    for k in range(L + 1):
+        w = O.highway_bp(st, caches, deltas, k)
+        for l in range(L + 1):
+            ref = np.zeros(d)
+            for j in range(l, min(l + k, L) + 1):
+                vec = flat[j]
+                for m in range(j, l, -1):
+                    vec = vec @ full[m]
+                ref = ref + vec
+            np.testing.assert_allclose(w[l].reshape(-1), ref, rtol=1e-6, atol=1e-8)
