@@ -185,6 +185,50 @@ class RNNStep:
         return {"W": dz.T @ cache["h"], "U": dz.T @ _f64(self.x_t)}
 
 
+def _sigmoid(v):
+    return 1.0 / (1.0 + np.exp(-v))
+
+
+class GRUStep:
+    """One GRU cell as a layer with a data-dependent gate (Table 1, row "GRU": f(x) = a(x) * x + b(x),
+    g = [a, b], r(x, z) = z1 * x + z2).  With r = sigmoid(U_r x_t + W_r h), z = sigmoid(U_z x_t + W_z h),
+    n = tanh(U_n x_t + r * (W_n h)):  h' = z * h + (1 - z) * n, so a(h) = z, b(h) = (1 - z) * n,
+    K = diag(z) and J = diag(h) da/dh + db/dh.  W [3d, d] and U [3d, in] stack the r, z, n rows."""
+
+    def __init__(self, W, U, x_t):
+        self.W, self.U, self.x_t = W, U, x_t
+
+    def forward(self, h):
+        W, U = _f64(self.W), _f64(self.U)
+        d = h.shape[-1]
+        pre = _f64(self.x_t) @ U.T
+        rec = h @ W.T
+        r = _sigmoid(pre[..., :d] + rec[..., :d])
+        z = _sigmoid(pre[..., d:2 * d] + rec[..., d:2 * d])
+        rec_n = rec[..., 2 * d:]
+        n = np.tanh(pre[..., 2 * d:] + r * rec_n)
+        return (1.0 - z) * n, dict(h=h, r=r, z=z, n=n, rec_n=rec_n)
+
+    def gate(self, cache):
+        return cache["z"]
+
+    def _pre_grads(self, c, g):
+        dn_pre = g * (1.0 - c["z"]) * (1.0 - c["n"] ** 2)
+        dz_pre = g * (c["h"] - c["n"]) * c["z"] * (1.0 - c["z"])      # through a = z (times h) and through b
+        dr_pre = dn_pre * c["rec_n"] * c["r"] * (1.0 - c["r"])
+        return dr_pre, dz_pre, dn_pre
+
+    def vjp(self, c, g):
+        dr_pre, dz_pre, dn_pre = self._pre_grads(c, g)
+        return np.concatenate([dr_pre, dz_pre, dn_pre * c["r"]], axis=-1) @ _f64(self.W)
+
+    def param_vjp(self, c, g):
+        dr_pre, dz_pre, dn_pre = self._pre_grads(c, g)
+        rec = np.concatenate([dr_pre, dz_pre, dn_pre * c["r"]], axis=-1)
+        pre = np.concatenate([dr_pre, dz_pre, dn_pre], axis=-1)
+        return {"W": rec.T @ c["h"], "U": pre.T @ _f64(self.x_t)}
+
+
 class ShiftedStep:
     """The gamma-shifted split of a residual layer x + Block(x) (Appendix C.3, Eq. 17): the block becomes
     g(x) = Block(x) + gamma x and the residual function r(x, z) = (1 - gamma) x + z, so the layer itself is
@@ -226,7 +270,14 @@ class Stack:
         self.names = names
         self.gate_shared = gate_shared
 
-    def gate(self, l):
+    def gate(self, l, caches=None):
+        """Diagonal of K_{l+1}: a constant, or - for blocks with a data-dependent gate (GRU) - the value the
+        forward pass produced at x_l, taken from its cache."""
+        step = self.steps[l]
+        if hasattr(step, "gate"):
+            if caches is None:
+                raise ValueError("this stack's gates depend on the states: pass the forward caches")
+            return step.gate(caches[l])
         a = self.gates[l]
         return 1.0 if a is None else _f64(a)
 
@@ -235,6 +286,12 @@ def mlp_stack(W1, W2, pre_ln, eps=1e-5, gate=None):
     L = len(W1)
     steps = [MLPStep(_Lazy(W1, l), _Lazy(W2, l), pre_ln, eps) for l in range(L)]
     return Stack(steps, [gate] * L)
+
+
+def gru_stack(W, U, X):
+    """GRU over time; X is [T, B, in]."""
+    T = len(X)
+    return Stack([GRUStep(W, U, _Lazy(X, t)) for t in range(T)])
 
 
 def rnn_stack(W, U, a, X):
@@ -274,7 +331,7 @@ def forward(stack, x0):
     for l, step in enumerate(stack.steps):
         f, cache = step.forward(xs[l])
         caches.append(cache)
-        xs.append(stack.gate(l) * xs[l] + f)
+        xs.append(stack.gate(l, caches) * xs[l] + f)
     return xs, caches
 
 
@@ -285,7 +342,7 @@ def exact_bp(stack, caches, deltas):
     g = [None] * (L + 1)
     g[L] = _f64(deltas[L])
     for l in range(L - 1, -1, -1):
-        g[l] = _f64(deltas[l]) + stack.gate(l) * g[l + 1] + stack.steps[l].vjp(caches[l], g[l + 1])
+        g[l] = _f64(deltas[l]) + stack.gate(l, caches) * g[l + 1] + stack.steps[l].vjp(caches[l], g[l + 1])
     return g
 
 
@@ -354,13 +411,13 @@ def cumsumprod_parallel(v, K):
     return u
 
 
-def initial_estimate(stack, deltas):
+def initial_estimate(stack, deltas, caches=None):
     """Eq. 5 / Eq. 10: w^0 = CumSumProd(delta, K), the pure residual-path term."""
     L = stack.L
     w0 = [None] * (L + 1)
     w0[L] = _f64(deltas[L])
     for l in range(L - 1, -1, -1):
-        w0[l] = _f64(deltas[l]) + stack.gate(l) * w0[l + 1]
+        w0[l] = _f64(deltas[l]) + stack.gate(l, caches) * w0[l + 1]
     return w0
 
 
@@ -372,12 +429,12 @@ def highway_bp(stack, caches, deltas, k, return_all=False):
     if k < 0:
         raise ValueError("k must be >= 0")
     L = stack.L
-    w0 = initial_estimate(stack, deltas)
+    w0 = initial_estimate(stack, deltas, caches)
     w = list(w0)
     history = [list(w)]
     for _ in range(k):
         v = [stack.steps[l].vjp(caches[l], w[l + 1]) for l in range(L)]
-        u = cumsumprod_sequential(v, [stack.gate(l) for l in range(L)])
+        u = cumsumprod_sequential(v, [stack.gate(l, caches) for l in range(L)])
         w = [w0[l] + u[l] for l in range(L)] + [w0[L]]
         history.append(list(w))
     return history if return_all else w
@@ -388,13 +445,13 @@ def highway_bp_folded(stack, caches, deltas, k):
     g_l = delta_l + a_l g_{l+1} + u_l; equal to the literal form by linearity
     of the recurrence."""
     L = stack.L
-    g = initial_estimate(stack, deltas)
+    g = initial_estimate(stack, deltas, caches)
     for _ in range(k):
         v = [stack.steps[l].vjp(caches[l], g[l + 1]) for l in range(L)]
         new = [None] * (L + 1)
         new[L] = _f64(deltas[L])
         for l in range(L - 1, -1, -1):
-            new[l] = _f64(deltas[l]) + stack.gate(l) * new[l + 1] + v[l]
+            new[l] = _f64(deltas[l]) + stack.gate(l, caches) * new[l + 1] + v[l]
         g = new
     return g
 

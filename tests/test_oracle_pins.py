@@ -489,3 +489,69 @@ def test_gamma_one_is_fixed_point_iteration_and_path_sums_hold():
                     vec = vec @ full[m]
                 ref = ref + vec
             np.testing.assert_allclose(w[l].reshape(-1), ref, rtol=1e-6, atol=1e-8)
+
+
+# ---------------------------------------------- 11. GRU: a data-dependent gate (Table 1)
+def _gru_setup(rng, T=4, d=3, nin=2, B=1):
+    W = rng.normal(size=(3 * d, d)) * 0.7
+    U = rng.normal(size=(3 * d, nin)) * 0.7
+    X = rng.normal(size=(T, B, nin))
+    return W, U, X, O.gru_stack(W, U, X)
+
+
+def test_gru_matches_the_textbook_cell_and_torch():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(41)
+    T, d, nin, B = 5, 4, 3, 2
+    W, U, X, st = _gru_setup(rng, T, d, nin, B)
+    h0 = rng.normal(size=(B, d))
+    xs, caches = O.forward(st, h0)
+    cell = torch.nn.GRUCell(nin, d, bias=False).double()
+    with torch.no_grad():
+        cell.weight_ih.copy_(torch.tensor(U))
+        cell.weight_hh.copy_(torch.tensor(W))
+    h = torch.tensor(h0, requires_grad=True)
+    hs = [h]
+    for t in range(T):
+        hs.append(cell(torch.tensor(X[t]), hs[-1]))
+        hs[-1].retain_grad()
+    # torch: h' = (1 - z) * n + z * h with the same r, z, n: the library cell is the pin for the forward map
+    for t in range(T + 1):
+        np.testing.assert_allclose(xs[t], hs[t].detach().numpy(), rtol=1e-12, atol=1e-13)
+    Y = rng.normal(size=(T, B, d))
+    loss = sum(0.5 * ((hs[t] - torch.tensor(Y[t - 1])) ** 2).sum() for t in range(1, T + 1))
+    loss.backward()
+    deltas = [np.zeros_like(h0)] + [xs[t] - Y[t - 1] for t in range(1, T + 1)]
+    g = O.exact_bp(st, caches, deltas)
+    np.testing.assert_allclose(g[0], h.grad.numpy(), rtol=1e-10, atol=1e-12)
+    grads = O.param_grads(st, caches, xs, g, [("", None)] * T)
+    np.testing.assert_allclose(grads["W"], cell.weight_hh.grad.numpy(), rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(grads["U"], cell.weight_ih.grad.numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_gru_path_sums_with_state_dependent_gate():
+    rng = np.random.default_rng(42)
+    T, d = 4, 3
+    W, U, X, st = _gru_setup(rng, T, d)
+    xs, caches = O.forward(st, rng.normal(size=(1, d)))
+    deltas = random_deltas(xs, every=True, rng=rng)
+    # K_m = diag(z) from the forward pass; J_m = (Jacobian of the whole cell, by finite differences) - K_m
+    J, K = [None], [None]
+    for l in range(T):
+        def cell(hflat, l=l):
+            f, c = st.steps[l].forward(hflat.reshape(1, d))
+            return (c["z"] * hflat.reshape(1, d) + f).reshape(-1)
+        full = O.finite_difference_jacobian(cell, xs[l].reshape(-1), h=1e-5)
+        Km = np.diag(caches[l]["z"].reshape(-1))
+        K.append(Km)
+        J.append(full - Km)
+    flat = [x.reshape(-1) for x in deltas]
+    for k in range(T + 1):
+        w = O.highway_bp(st, caches, deltas, k)
+        for i in range(T + 1):
+            np.testing.assert_allclose(w[i].reshape(-1), O.path_sum(flat, J, K, i, k), rtol=1e-6, atol=1e-8)
+    g = O.exact_bp(st, caches, deltas)
+    for a, b in zip(O.highway_bp(st, caches, deltas, T), g):
+        np.testing.assert_allclose(a, b, rtol=1e-11, atol=1e-12)
+    for a, b in zip(O.highway_bp_folded(st, caches, deltas, 2), O.highway_bp(st, caches, deltas, 2)):
+        np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
