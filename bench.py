@@ -52,6 +52,9 @@ def algorithmic_flops(w, k):
     if w.block == "rnn_tanh":
         rows = w.L * w.batch
         return 2 * w.d * w.d * rows, 2 * w.d * (w.d + w.in_dim) * rows
+    if w.block == "gru":
+        rows = w.L * w.batch
+        return 6 * w.d * w.d * rows, 6 * w.d * (w.d + w.in_dim) * rows
     if w.block == "preln_transformer":
         n, d, s = w.tokens, w.d, w.seq
         blk = 8 * d * d * n + 5 * s * d * n + 16 * d * d * n
@@ -82,7 +85,7 @@ def oracle_timing(w, k, sample, steps, warmup):
         inp64 = {n: (t.double() if n in weights else t) for n, t in inp.items()}
     else:  # too large to hold in float64 at once: converted layer by layer inside the timed calls
         inp64 = inp
-    units = {"preln_transformer": w.batch, "rnn_tanh": w.batch}.get(w.block, w.tokens)
+    units = {"preln_transformer": w.batch, "rnn_tanh": w.batch, "gru": w.batch}.get(w.block, w.tokens)
     sample = min(sample, units)
     times = []
     for it in range(warmup + steps):
@@ -289,7 +292,7 @@ def run_ours(args):
             "phases_ms_per_step": {"vjp": vjp_ms / args.steps, "scan": scan_ms / args.steps, "wgrad": wg_ms / args.steps},
             "tflops": {"vjp": vjp_flops * kk / (vjp_ms / args.steps * 1e-3) / 1e12 if vjp_ms else None,
                        "wgrad": wgrad_flops / (wg_ms / args.steps * 1e-3) / 1e12 if wg_ms else None},
-            "replicas_tokens_per_s": world * w.tokens * (w.L if w.block == "rnn_tanh" else 1) / (ms_step * 1e-3)}
+            "replicas_tokens_per_s": world * w.tokens * (w.L if w.block in ("rnn_tanh", "gru") else 1) / (ms_step * 1e-3)}
 
     if not args.no_detail and rank == 0:
         detail = {}

@@ -64,8 +64,15 @@ typedef enum {
  *  MLP               f(x) = W2 gelu(W1 x)                     (exact erf GELU, no biases)
  *  PRELN_MLP         f(x) = W2 gelu(W1 LN(x))                 (LN without affine, biased variance)
  *  RNN_TANH          f_t(h) = tanh(W h + U x_t), weights shared over t; L is the sequence length
- *  PRELN_TRANSFORMER L decoder blocks = 2L residual steps: causal softmax MHA(LN(x)) Wo, then PRELN_MLP */
-typedef enum { HBP_BLOCK_MLP = 0, HBP_BLOCK_PRELN_MLP = 1, HBP_BLOCK_RNN_TANH = 2, HBP_BLOCK_PRELN_TRANSFORMER = 3 } hbp_block;
+ *  PRELN_TRANSFORMER L decoder blocks = 2L residual steps: causal softmax MHA(LN(x)) Wo, then PRELN_MLP
+ *  GRU               Table 1, row "GRU": h' = z (.) h + (1 - z) (.) n with r = sigmoid(U_r x_t + W_r h),
+ *                    z = sigmoid(U_z x_t + W_z h), n = tanh(U_n x_t + r (.) W_n h), no biases, weights shared over
+ *                    t.  The residual gate is the update gate z_t itself, K = diag(z_t): it depends on the state,
+ *                    is produced by hbp_forward and kept in the workspace; cfg.gate must be HBP_GATE_ONE (there is
+ *                    no further constant gate) and cfg.gamma 0. */
+typedef enum {
+  HBP_BLOCK_MLP = 0, HBP_BLOCK_PRELN_MLP = 1, HBP_BLOCK_RNN_TANH = 2, HBP_BLOCK_PRELN_TRANSFORMER = 3, HBP_BLOCK_GRU = 4
+} hbp_block;
 typedef enum { HBP_F32 = 0, HBP_BF16 = 1 } hbp_dtype;
 /* Residual gate a_l, the diagonal of K (Eq. 2): all ones, one vector a[d] for every step, or a[steps][d]. */
 typedef enum { HBP_GATE_ONE = 0, HBP_GATE_CHANNEL_SHARED = 1, HBP_GATE_CHANNEL_PER_STEP = 2 } hbp_gate;
@@ -81,11 +88,11 @@ typedef struct {
   int32_t L;        /* residual steps (MLP kinds), time steps (RNN), decoder blocks (Transformer) */
   int32_t d;        /* state width */
   int32_t hidden;   /* MLP hidden width (MLP kinds, Transformer) */
-  int32_t in_dim;   /* RNN input width */
+  int32_t in_dim;   /* RNN / GRU input width */
   int32_t n_heads;  /* Transformer: n_heads * head_dim == d */
   int32_t head_dim;
   int32_t seq;      /* Transformer: tokens == batch * seq */
-  int32_t batch;    /* Transformer: sequences; RNN: rows (== tokens) */
+  int32_t batch;    /* Transformer: sequences; RNN / GRU: rows (== tokens) */
   int64_t tokens;   /* N: rows of one state */
   float ln_eps;
   float gamma;      /* shift of the residual split, 0 <= gamma <= 1 (Appendix C.3, Eq. 17); 0 = the plain split */
@@ -94,6 +101,7 @@ typedef struct {
 /* Borrowed parameter pointers; those the block kind does not use are ignored.
  *  MLP kinds:    W1 [L][hidden][d], W2 [L][d][hidden]
  *  RNN:          W [d][d], U [d][in_dim]
+ *  GRU:          W [3d][d], U [3d][in_dim]: the rows of the r, z and n parts stacked in that order
  *  Transformer:  Wq, Wk, Wv, Wo [L][d][d], W1 [L][hidden][d], W2 [L][d][hidden]
  *  gate:         a [d] or [steps][d] when cfg.gate != HBP_GATE_ONE (steps = 2L for the Transformer) */
 typedef struct {
@@ -123,7 +131,7 @@ hbp_status hbp_create(const hbp_config* cfg, void* workspace, size_t workspace_b
 
 /* Section 3, h_i = f_i(h_{i-1}): runs the steps from x0 [N][d] and stores every state in
  * x_all [steps+1][N][d] (x_all[0] = x0) plus, in the workspace, what the block VJPs need.
- * `inputs` is the RNN's x [L][batch][in_dim] (NULL otherwise). */
+ * `inputs` is the RNN's or GRU's x [L][batch][in_dim] (NULL otherwise). */
 hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, const void* inputs,
                        void* x_all, void* cuda_stream);
 

@@ -1,0 +1,257 @@
+// GRU cell as a residual step with a state-dependent gate (Table 1, row "GRU"):
+//     r = sigmoid(U_r x_t + W_r h),  z = sigmoid(U_z x_t + W_z h),  n = tanh(U_n x_t + r * (W_n h)),
+//     h' = z * h + (1 - z) * n,
+// so K = diag(z) is the cheap Jacobian and J^T g = (g * [c_r | c_z | c_nr]) W is the block VJP, with the
+// per-element coefficients
+//     c_n  = (1 - z)(1 - n^2)        (dLoss/d(pre-activation of n) per unit of g)
+//     c_z  = (h - n) z (1 - z)
+//     c_r  = c_n * (W_n h) * r (1 - r)
+//     c_nr = c_n * r
+// which the forward step computes once, in double, from the pre-activations (no cancellation near saturated
+// gates) and stores as C4 = [c_r | c_z | c_nr | c_n] per row.  The input-weight gradient uses
+// [c_r | c_z | c_n] instead of the first three.  Like the tanh RNN, the recurrence itself and exact
+// backpropagation through time are carried in double beside the stored values.
+#include "hbp_internal.h"
+
+namespace hbp {
+
+namespace {
+
+constexpr int kTile = 32;
+
+// acc[gate][j] += sum_k src[m_j][k] * Wm[gate * d + n][k] over k in [0, kdim)
+template <typename T, bool kSrcDouble>
+__device__ __forceinline__ void gru_accumulate(const void* __restrict__ src, const T* __restrict__ Wm, int kdim, int B,
+                                               int d, int m0, int n0, double (*Hs)[kTile + 1],
+                                               float (*Ws)[kTile][kTile + 1], double acc[3][4]) {
+  const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
+  for (int k0 = 0; k0 < kdim; k0 += kTile) {
+    for (int i = ty; i < kTile; i += 8) {
+      const int k = k0 + tx, m = m0 + i, n = n0 + i;
+      double hv = 0.0;
+      if (k < kdim && m < B)
+        hv = kSrcDouble ? ((const double*)src)[(int64_t)m * kdim + k] : (double)to_f(((const T*)src)[(int64_t)m * kdim + k]);
+      Hs[i][tx] = hv;
+#pragma unroll
+      for (int q = 0; q < 3; ++q)
+        Ws[q][i][tx] = (k < kdim && n < d) ? to_f(Wm[((int64_t)q * d + n) * kdim + k]) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int kk = 0; kk < kTile; ++kk) {
+      double w[3];
+#pragma unroll
+      for (int q = 0; q < 3; ++q) w[q] = (double)Ws[q][tx][kk];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const double hv = Hs[ty + 8 * j][kk];
+#pragma unroll
+        for (int q = 0; q < 3; ++q) acc[q][j] = fma(hv, w[q], acc[q][j]);
+      }
+    }
+    __syncthreads();
+  }
+}
+
+__device__ __forceinline__ double sigmoid_d(double v) { return 1.0 / (1.0 + exp(-v)); }
+
+template <typename T>
+__global__ void __launch_bounds__(256) gru_step_kernel(const T* __restrict__ W, const T* __restrict__ U,
+                                                       const T* __restrict__ x_t, const double* __restrict__ h_in,
+                                                       double* __restrict__ h_out, T* __restrict__ zc,
+                                                       T* __restrict__ c4, T* __restrict__ state_out, int B, int d,
+                                                       int in_dim) {
+  __shared__ double Hs[kTile][kTile + 1];
+  __shared__ float Ws[3][kTile][kTile + 1];
+  const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
+  const int n0 = blockIdx.x * kTile, m0 = blockIdx.y * kTile;
+  double rec[3][4], pre[3][4];
+#pragma unroll
+  for (int q = 0; q < 3; ++q)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) rec[q][j] = pre[q][j] = 0.0;
+  gru_accumulate<T, true>(h_in, W, d, B, d, m0, n0, Hs, Ws, rec);
+  gru_accumulate<T, false>(x_t, U, in_dim, B, d, m0, n0, Hs, Ws, pre);
+  const int n = n0 + tx;
+  if (n >= d) return;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int m = m0 + ty + 8 * j;
+    if (m >= B) continue;
+    const int64_t idx = (int64_t)m * d + n;
+    const double ar = pre[0][j] + rec[0][j], az = pre[1][j] + rec[1][j];
+    const double r = sigmoid_d(ar), r1 = sigmoid_d(-ar);  // r and 1 - r
+    const double z = sigmoid_d(az), z1 = sigmoid_d(-az);
+    const double an = pre[2][j] + r * rec[2][j];
+    const double e = exp(-2.0 * fabs(an));
+    const double nn = copysign((1.0 - e) / (1.0 + e), an);
+    const double dn = 4.0 * e / ((1.0 + e) * (1.0 + e));  // 1 - tanh(an)^2
+    const double h = h_in[idx];
+    const double hn = z * h + z1 * nn;
+    const double cn = z1 * dn;
+    h_out[idx] = hn;
+    state_out[idx] = from_f<T>((float)hn);
+    zc[idx] = from_f<T>((float)z);
+    T* c = c4 + (int64_t)m * 4 * d + n;
+    c[0] = from_f<T>((float)(cn * rec[2][j] * r * r1));
+    c[d] = from_f<T>((float)((h - nn) * z * z1));
+    c[2 * d] = from_f<T>((float)(cn * r));
+    c[3 * d] = from_f<T>((float)cn);
+  }
+}
+
+// Exact backpropagation through one GRU step in double:
+//     g_t = delta_t + z_t * g_{t+1} + (g_{t+1} * [c_r | c_z | c_nr]) W.
+template <typename T>
+__global__ void __launch_bounds__(256) gru_bwd_step_kernel(const T* __restrict__ W, const T* __restrict__ zc,
+                                                           const T* __restrict__ c4, const T* __restrict__ delta,
+                                                           const double* __restrict__ g_in, double* __restrict__ g_out,
+                                                           T* __restrict__ g_store, int B, int d) {
+  __shared__ double Hs[kTile][kTile + 1];
+  __shared__ float Ws[kTile][kTile + 1];
+  const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
+  const int n0 = blockIdx.x * kTile, m0 = blockIdx.y * kTile;
+  double acc[4] = {0.0, 0.0, 0.0, 0.0};
+  for (int q = 0; q < 3; ++q) {
+    for (int k0 = 0; k0 < d; k0 += kTile) {
+      for (int i = ty; i < kTile; i += 8) {
+        const int m = m0 + i, k = k0 + tx;
+        Hs[i][tx] = (m < B && k < d) ? g_in[(int64_t)m * d + k] * (double)to_f(c4[(int64_t)m * 4 * d + (int64_t)q * d + k]) : 0.0;
+        const int kk = k0 + i, n = n0 + tx;  // W[q*d + k][n]: contiguous in n
+        Ws[tx][i] = (kk < d && n < d) ? to_f(W[((int64_t)q * d + kk) * d + n]) : 0.0f;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int kk = 0; kk < kTile; ++kk) {
+        const double w = (double)Ws[tx][kk];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[j] = fma(Hs[ty + 8 * j][kk], w, acc[j]);
+      }
+      __syncthreads();
+    }
+  }
+  const int n = n0 + tx;
+  if (n >= d) return;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int m = m0 + ty + 8 * j;
+    if (m >= B) continue;
+    const int64_t idx = (int64_t)m * d + n;
+    const double v = (delta ? (double)to_f(delta[idx]) : 0.0) + (double)to_f(zc[idx]) * g_in[idx] + acc[j];
+    g_out[idx] = v;
+    g_store[idx] = from_f<T>((float)v);
+  }
+}
+
+// a4[row][q*d + c] = g[row][c] * c4[row][q*d + c] for q = 0..3 (the operand of the CUDA-core GEMMs).
+template <typename T>
+__global__ void gru_operand_kernel(const T* __restrict__ g, const T* __restrict__ c4, T* __restrict__ a4, int64_t rows,
+                                   int d) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= rows * 4 * d) return;
+  const int64_t row = i / (4 * d);
+  const int c = (int)(i % d);
+  a4[i] = from_f<T>(to_f(g[row * d + c]) * to_f(c4[i]));
+}
+
+// tf32 split of g * [c_r | c_z | c_nr] as [rows][3d] (the VJP's A operand, contraction index contiguous)
+__global__ void gru_split_kernel(const float* __restrict__ g, const float* __restrict__ c4, float4* __restrict__ hi,
+                                 float4* __restrict__ lo, int64_t rows, int d) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;  // one float4 of the [rows][3d] output
+  const int vrow = 3 * d / 4;
+  if (i >= rows * vrow) return;
+  const int64_t row = i / vrow;
+  const int col = (int)(i % vrow) * 4;  // column in [0, 3d); never straddles a block since d % 4 == 0
+  const float4 gv = *reinterpret_cast<const float4*>(g + row * d + col % d);
+  const float4 cv = *reinterpret_cast<const float4*>(c4 + row * 4 * d + col);
+  const float v[4] = {gv.x * cv.x, gv.y * cv.y, gv.z * cv.z, gv.w * cv.w};
+  float h[4], l[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    h[k] = round_tf32(v[k]);
+    l[k] = round_tf32(v[k] - h[k]);
+  }
+  hi[i] = make_float4(h[0], h[1], h[2], h[3]);
+  lo[i] = make_float4(l[0], l[1], l[2], l[3]);
+}
+
+// tf32 split of g * C4 written transposed, [4d][rows] (the weight-gradient GEMMs contract over rows)
+__global__ void __launch_bounds__(256) gru_split_transposed_kernel(const float* __restrict__ g,
+                                                                   const float* __restrict__ c4, float* __restrict__ hiT,
+                                                                   float* __restrict__ loT, int64_t rows, int d) {
+  __shared__ float th[32][33], tl[32][33];
+  const int64_t r0 = (int64_t)blockIdx.x * 32;
+  const int c0 = blockIdx.y * 32;  // column of C4 in [0, 4d)
+  const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
+  for (int i = ty; i < 32; i += 8) {
+    const int64_t r = r0 + i;
+    const int c = c0 + tx;
+    float v = 0.0f;
+    if (r < rows && c < 4 * d) v = g[r * d + c % d] * c4[r * 4 * d + c];
+    const float h = round_tf32(v);
+    th[i][tx] = h;
+    tl[i][tx] = round_tf32(v - h);
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int c = c0 + i;
+    const int64_t r = r0 + tx;
+    if (c < 4 * d && r < rows) {
+      hiT[(int64_t)c * rows + r] = th[tx][i];
+      loT[(int64_t)c * rows + r] = tl[tx][i];
+    }
+  }
+}
+
+}  // namespace
+
+void gru_forward_step(Launcher& lc, int dtype, const void* W, const void* U, const void* x_t, const double* h_in,
+                      double* h_out, void* zc, void* c4, void* state_out, int B, int d, int in_dim) {
+  dim3 grid((d + kTile - 1) / kTile, (B + kTile - 1) / kTile);
+  if (dtype == HBP_F32)
+    gru_step_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)U, (const float*)x_t, h_in, h_out,
+                                                        (float*)zc, (float*)c4, (float*)state_out, B, d, in_dim);
+  else
+    gru_step_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)U, (const bf16*)x_t, h_in, h_out,
+                                                       (bf16*)zc, (bf16*)c4, (bf16*)state_out, B, d, in_dim);
+  lc.count();
+  lc.check();
+}
+
+void gru_backward_step(Launcher& lc, int dtype, const void* W, const void* zc, const void* c4, const void* delta,
+                       const double* g_in, double* g_out, void* g_store, int B, int d) {
+  dim3 grid((d + kTile - 1) / kTile, (B + kTile - 1) / kTile);
+  if (dtype == HBP_F32)
+    gru_bwd_step_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)zc, (const float*)c4,
+                                                            (const float*)delta, g_in, g_out, (float*)g_store, B, d);
+  else
+    gru_bwd_step_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)zc, (const bf16*)c4,
+                                                           (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, d);
+  lc.count();
+  lc.check();
+}
+
+void gru_operand(Launcher& lc, int dtype, const void* g, const void* c4, void* a4, int64_t rows, int d) {
+  const int64_t n = rows * 4 * d;
+  const unsigned grid = (unsigned)((n + 255) / 256);
+  if (dtype == HBP_F32) gru_operand_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)g, (const float*)c4, (float*)a4, rows, d);
+  else gru_operand_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)g, (const bf16*)c4, (bf16*)a4, rows, d);
+  lc.count();
+  lc.check();
+}
+
+void gru_split(Launcher& lc, const float* g, const float* c4, float* hi, float* lo, int64_t rows, int d) {
+  const int64_t nvec = rows * (3 * d / 4);
+  gru_split_kernel<<<(unsigned)((nvec + 255) / 256), 256, 0, lc.stream>>>(g, c4, (float4*)hi, (float4*)lo, rows, d);
+  lc.count();
+  lc.check();
+}
+
+void gru_split_transposed(Launcher& lc, const float* g, const float* c4, float* hiT, float* loT, int64_t rows, int d) {
+  dim3 grid((unsigned)((rows + 31) / 32), (unsigned)((4 * d + 31) / 32));
+  gru_split_transposed_kernel<<<grid, 256, 0, lc.stream>>>(g, c4, hiT, loT, rows, d);
+  lc.count();
+  lc.check();
+}
+
+}  // namespace hbp

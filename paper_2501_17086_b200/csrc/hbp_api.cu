@@ -59,6 +59,9 @@ struct hbp_ctx {
   float4* lnstat = nullptr;  // [steps][N] {rstd, mean dY, mean dY * xhat, 0}
   int ln_slots = 0;
   char* C = nullptr;       // RNN: [T][B][d] tanh'(z_t) = 1 - tanh(z_t)^2
+  // GRU: the update gate z_t [T][B][d] (the diagonal of K), the VJP coefficients [T*B][4d] = [c_r|c_z|c_nr|c_n]
+  // and, for the GEMMs that do not take the tf32 splits, g times those coefficients [T*B][4d]
+  char *Zc = nullptr, *C4 = nullptr, *A4 = nullptr;
   char* scan_scratch = nullptr;
   size_t scan_scratch_bytes = 0;
   float* partial = nullptr;  // split-K / gate-gradient partial sums
@@ -85,7 +88,7 @@ inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 hbp_status check_config(const hbp_config* c) {
   if (!c) return HBP_ERR_INVALID_ARG;
   if (c->dtype != HBP_F32 && c->dtype != HBP_BF16) return HBP_ERR_DTYPE;
-  if (c->block < 0 || c->block > HBP_BLOCK_PRELN_TRANSFORMER) return HBP_ERR_UNSUPPORTED;
+  if (c->block < 0 || c->block > HBP_BLOCK_GRU) return HBP_ERR_UNSUPPORTED;
   if (c->gate < 0 || c->gate > HBP_GATE_CHANNEL_PER_STEP) return HBP_ERR_UNSUPPORTED;
   if (c->loss != HBP_LOSS_FINAL && c->loss != HBP_LOSS_EVERY_STEP) return HBP_ERR_UNSUPPORTED;
   const int v = c->dtype == HBP_F32 ? 4 : 8;
@@ -94,7 +97,8 @@ hbp_status check_config(const hbp_config* c) {
   if (c->gamma != 0.0f && (c->gate != HBP_GATE_ONE || c->block == HBP_BLOCK_RNN_TANH)) return HBP_ERR_UNSUPPORTED;
   if (c->d % v) return HBP_ERR_SHAPE;
   if (c->d / v > 1024) return HBP_ERR_SHAPE;  // one block per row in the LayerNorm kernels
-  if (c->block == HBP_BLOCK_RNN_TANH) {
+  if (c->block == HBP_BLOCK_GRU && (c->gate != HBP_GATE_ONE || c->gamma != 0.0f)) return HBP_ERR_UNSUPPORTED;
+  if (c->block == HBP_BLOCK_RNN_TANH || c->block == HBP_BLOCK_GRU) {
     if (c->in_dim <= 0 || c->in_dim % v) return HBP_ERR_SHAPE;
     if (c->batch != c->tokens) return HBP_ERR_SHAPE;
   } else {
@@ -127,9 +131,26 @@ size_t carve(hbp_ctx* c, char* base) {
   const size_t steps = (size_t)c->steps;
   c->status = (int*)take(256);
   c->U = take(steps * N * d * es);
-  if (f.dtype == HBP_BF16 && f.block != HBP_BLOCK_RNN_TANH) c->xres = (float*)take(N * d * 4);
+  const bool recurrent = f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU;
+  if (f.dtype == HBP_BF16 && !recurrent) c->xres = (float*)take(N * d * 4);
   c->partial_floats = (size_t)kGateBlocks * d;
-  if (f.block == HBP_BLOCK_RNN_TANH) {
+  if (f.block == HBP_BLOCK_GRU) {
+    const size_t in = (size_t)f.in_dim;
+    c->Zc = take(steps * N * d * es);
+    c->C4 = take(steps * N * 4 * d * es);
+    c->A4 = take(steps * N * 4 * d * es);
+    c->hres = (double*)take(2 * N * d * 8);
+    if (f.dtype == HBP_F32) {
+      c->Ahi = (float*)take(steps * N * 4 * d * 4); c->Alo = (float*)take(steps * N * 4 * d * 4);
+      c->Hhi = (float*)take(steps * N * d * 4); c->Hlo = (float*)take(steps * N * d * 4);
+      c->Xhi = (float*)take(steps * N * in * 4); c->Xlo = (float*)take(steps * N * in * 4);
+      c->Whi = (float*)take(3 * d * d * 4); c->Wlo = (float*)take(3 * d * d * 4);
+    }
+    c->scan_scratch_bytes = scan_scratch_bytes(f.dtype, f.L, f.tokens, f.d);
+    c->scan_scratch = take(c->scan_scratch_bytes);
+    const size_t wmax = 3 * d * (d > in ? d : in);
+    if ((size_t)kMaxSplit * wmax > c->partial_floats) c->partial_floats = (size_t)kMaxSplit * wmax;
+  } else if (f.block == HBP_BLOCK_RNN_TANH) {
     c->C = take(steps * N * d * es);
     c->hres = (double*)take(2 * N * d * 8);
     if (f.dtype == HBP_F32) {
@@ -380,6 +401,71 @@ struct Run {
     }
   }
 
+  // ---- GRU ---------------------------------------------------------------------------------------
+  // u_t = (g_{t+1} * [c_r | c_z | c_nr]_t) W for every t at once: one GEMM over T*B rows with K = 3d
+  void gru_vjp_all() {
+    const int T = c->cfg.L;
+    const int64_t rows = (int64_t)T * N;
+    GemmArgs a = base_args();
+    a.M = (int)rows; a.N = (int)d; a.K = (int)(3 * d);
+    a.A = c->A4; a.a_sm = 4 * d; a.a_sk = 1;
+    a.B = p->W; a.b_sn = 1; a.b_sk = d;
+    a.epi = EPI_STORE; a.D = c->U; a.ldd = d;
+    if (c->cfg.loss == HBP_LOSS_EVERY_STEP) {
+      a.epi = EPI_ADD; a.E = delta; a.lde = d;
+      u_has_delta = true;
+    }
+    bool tc = false;
+    if (c->Ahi && !g_force_simt) {
+      gru_split(lc, (const float*)at(g, state), (const float*)c->C4, c->Ahi, c->Alo, rows, (int)d);
+      a.A_hi = c->Ahi; a.A_lo = c->Alo; a.hl_a_sm = 3 * d; a.hl_a_sk = 1;
+      a.B_hi = c->Whi; a.B_lo = c->Wlo; a.hl_b_sn = 3 * d; a.hl_b_sk = 1;
+      tc = gemm_tc(lc, a, c->status);
+    }
+    if (!tc) {
+      gru_operand(lc, c->cfg.dtype, at(g, state), c->C4, c->A4, rows, (int)d);
+      a.A_hi = a.A_lo = a.B_hi = a.B_lo = nullptr;
+      run_gemm(a);
+    }
+  }
+  // dW = [dr|dz|d(W_n h)]^T H (H = states 0..T-1),  dU = [dr|dz|dn]^T X, with the pre-activation gradients
+  // g * coefficients; dU is two products because its third row block uses another coefficient than dW's
+  void gru_wgrad(const hbp_grads* gr) {
+    const int T = c->cfg.L;
+    const int64_t rows = (int64_t)T * N, in = c->cfg.in_dim;
+    int split = (int)(rows / (c->Ahi ? 512 : 2048));
+    if (split < 1) split = 1;
+    if (split > kMaxSplit) split = kMaxSplit;
+    const bool try_tc = c->Ahi && !g_force_simt;
+    if (try_tc) gru_split_transposed(lc, (const float*)at(g, state), (const float*)c->C4, c->Ahi, c->Alo, rows, (int)d);
+    bool have_a4 = false;
+    // {first row of the [4d] operand, rows, output, output row, against the states or the inputs}
+    struct Part { int64_t a_row, m; float* out; int64_t out_row; bool states; };
+    const Part parts[3] = {{0, 3 * d, gr->dW, 0, true}, {0, 2 * d, gr->dU, 0, false}, {3 * d, d, gr->dU, 2 * d, false}};
+    for (const Part& pt : parts) {
+      const int64_t n = pt.states ? d : in;
+      GemmArgs a = base_args();
+      a.M = (int)pt.m; a.N = (int)n; a.K = (int)rows;
+      a.A = at(c->A4, pt.a_row); a.a_sm = 1; a.a_sk = 4 * d;
+      a.B = pt.states ? x_all : inputs; a.b_sn = 1; a.b_sk = n;
+      a.epi = EPI_STORE; a.d_f32 = true;
+      a.D = pt.out + pt.out_row * n; a.ldd = n;
+      if (split > 1) { a.splitk = split; a.partial = c->partial; }
+      bool tc = false;
+      if (try_tc) {
+        a.A_hi = c->Ahi + pt.a_row * rows; a.A_lo = c->Alo + pt.a_row * rows; a.hl_a_sm = rows; a.hl_a_sk = 1;
+        a.B_hi = pt.states ? c->Hhi : c->Xhi; a.B_lo = pt.states ? c->Hlo : c->Xlo; a.hl_b_sn = rows; a.hl_b_sk = 1;
+        tc = gemm_tc(lc, a, c->status);
+      }
+      if (!tc) {
+        if (!have_a4) gru_operand(lc, c->cfg.dtype, at(g, state), c->C4, c->A4, rows, (int)d);
+        have_a4 = true;
+        a.A_hi = a.A_lo = a.B_hi = a.B_lo = nullptr;
+        run_gemm(a);
+      }
+    }
+  }
+
   void gate_grads(const hbp_grads* gr) {
     if (!gr->da || c->cfg.gate == HBP_GATE_ONE) return;
     if (c->cfg.gate == HBP_GATE_CHANNEL_SHARED) {
@@ -410,6 +496,7 @@ struct Run {
     }
     s.delta = delta; s.loss = c->cfg.loss;
     s.a = p->a; s.gate = c->cfg.gate;
+    if (c->cfg.block == HBP_BLOCK_GRU) { s.a = c->Zc; s.gate = kGateElement; }
     s.g = g;
     if (with_u && c->preln) {
       s.xhat = c->Y; s.rstd = c->rstd;
@@ -455,7 +542,7 @@ hbp_status check_call(hbp_ctx* ctx, const hbp_params* p, bool need_forward) {
   if (!ctx || !p) return HBP_ERR_INVALID_ARG;
   if (need_forward && !ctx->forward_done) return HBP_ERR_STATE;
   const hbp_config& f = ctx->cfg;
-  if (f.block == HBP_BLOCK_RNN_TANH) {
+  if (f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU) {
     if (!p->W || !p->U) return HBP_ERR_INVALID_ARG;
   } else {
     if (!p->W1 || !p->W2) return HBP_ERR_INVALID_ARG;
@@ -468,7 +555,7 @@ hbp_status check_call(hbp_ctx* ctx, const hbp_params* p, bool need_forward) {
 hbp_status check_grads(const hbp_ctx* ctx, const hbp_grads* g) {
   if (!g) return HBP_OK;
   const hbp_config& f = ctx->cfg;
-  if (f.block == HBP_BLOCK_RNN_TANH) return (g->dW && g->dU) ? HBP_OK : HBP_ERR_INVALID_ARG;
+  if (f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU) return (g->dW && g->dU) ? HBP_OK : HBP_ERR_INVALID_ARG;
   if (!g->dW1 || !g->dW2) return HBP_ERR_INVALID_ARG;
   if (f.block == HBP_BLOCK_PRELN_TRANSFORMER && (!g->dWq || !g->dWk || !g->dWv || !g->dWo)) return HBP_ERR_INVALID_ARG;
   return HBP_OK;
@@ -587,7 +674,7 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
   if (!x0 || !x_all) return HBP_ERR_INVALID_ARG;
   if (misaligned(x0) || misaligned(x_all)) return HBP_ERR_SHAPE;
   const hbp_config& f = ctx->cfg;
-  if (f.block == HBP_BLOCK_RNN_TANH && !inputs) return HBP_ERR_INVALID_ARG;
+  if ((f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU) && !inputs) return HBP_ERR_INVALID_ARG;
   Run r(ctx, params, cuda_stream);
   r.x_all = (const char*)x_all;
   char* xa = (char*)x_all;
@@ -595,7 +682,22 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
   copy_state(r.lc, f.dtype, xa, x0, state);
   if (ctx->xres) convert_to_f32(r.lc, f.dtype, x0, ctx->xres, state);
 
-  if (f.block == HBP_BLOCK_RNN_TANH) {
+  if (f.block == HBP_BLOCK_GRU) {
+    const int T = f.L;
+    convert_to_f64(r.lc, f.dtype, x0, ctx->hres, state);
+    for (int t = 0; t < T; ++t) {
+      const double* hin = ctx->hres + (int64_t)(t & 1) * state;
+      double* hout = ctx->hres + (int64_t)((t + 1) & 1) * state;
+      gru_forward_step(r.lc, f.dtype, params->W, params->U, r.at(inputs, (int64_t)t * N * f.in_dim), hin, hout,
+                       r.at(ctx->Zc, (int64_t)t * state), r.at(ctx->C4, (int64_t)t * 4 * state),
+                       r.at(xa, (int64_t)(t + 1) * state), (int)N, (int)d, f.in_dim);
+    }
+    if (ctx->Ahi) {
+      split_tf32_transposed(r.lc, (const float*)xa, nullptr, ctx->Hhi, ctx->Hlo, (int64_t)T * N, (int)d);
+      split_tf32_transposed(r.lc, (const float*)inputs, nullptr, ctx->Xhi, ctx->Xlo, (int64_t)T * N, f.in_dim);
+      split_tf32_transposed(r.lc, (const float*)params->W, nullptr, ctx->Whi, ctx->Wlo, 3 * d, (int)d);  // -> [d][3d]
+    }
+  } else if (f.block == HBP_BLOCK_RNN_TANH) {
     const int T = f.L;
     convert_to_f64(r.lc, f.dtype, x0, ctx->hres, state);
     for (int t = 0; t < T; ++t) {
@@ -689,7 +791,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
   st = check_grads(ctx, grads);
   if (st != HBP_OK) return st;
   const hbp_config& f = ctx->cfg;
-  if (f.block == HBP_BLOCK_RNN_TANH && grads && !inputs) return HBP_ERR_INVALID_ARG;
+  if ((f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU) && grads && !inputs) return HBP_ERR_INVALID_ARG;
   Run r(ctx, params, cuda_stream);
   r.x_all = (const char*)x_all;
   r.inputs = (const char*)inputs;
@@ -697,6 +799,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
   r.delta = (const char*)delta;
   const int steps = ctx->steps, layers = ctx->layers, grp = ctx->group;
   const bool tr = f.block == HBP_BLOCK_PRELN_TRANSFORMER, rnn = f.block == HBP_BLOCK_RNN_TANH;
+  const bool gru = f.block == HBP_BLOCK_GRU;
   {
     PhaseScope ph(r, HBP_PHASE_OTHER);
     r.set_last_state();
@@ -715,6 +818,8 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
         PhaseScope ph(r, HBP_PHASE_VJP);
         if (rnn) {
           r.rnn_vjp_all();
+        } else if (gru) {
+          r.gru_vjp_all();
         } else {
           for (int b0 = 0; b0 < layers; b0 += grp) r.mlp_vjp(b0, b0 + grp < layers ? b0 + grp : layers, true);
           if (tr) r.attn_vjp(0, layers, true);
@@ -727,6 +832,8 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
       PhaseScope ph(r, HBP_PHASE_WGRAD);
       if (rnn) {
         r.rnn_wgrad(grads);
+      } else if (gru) {
+        r.gru_wgrad(grads);
       } else {
         for (int b0 = 0; b0 < layers; b0 += grp) {
           const int b1 = b0 + grp < layers ? b0 + grp : layers;
@@ -754,6 +861,17 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
                           gin, gout, r.at(r.g, (int64_t)t * r.state), (int)r.N, (int)r.d);
       }
       if (grads) r.rnn_wgrad(grads);
+    } else if (gru) {
+      convert_to_f64(r.lc, f.dtype, r.at(r.g, (int64_t)steps * r.state), ctx->hres, r.state);
+      for (int t = steps - 1; t >= 0; --t) {
+        const double* gin = ctx->hres + (int64_t)((steps - 1 - t) & 1) * r.state;
+        double* gout = ctx->hres + (int64_t)((steps - t) & 1) * r.state;
+        gru_backward_step(r.lc, f.dtype, params->W, r.at(ctx->Zc, (int64_t)t * r.state),
+                          r.at(ctx->C4, (int64_t)t * 4 * r.state),
+                          f.loss == HBP_LOSS_EVERY_STEP ? r.at(r.delta, (int64_t)t * r.state) : nullptr, gin, gout,
+                          r.at(r.g, (int64_t)t * r.state), (int)r.N, (int)r.d);
+      }
+      if (grads) r.gru_wgrad(grads);
     } else {
       for (int l = steps - 1; l >= 0; --l) {
         const int b = tr ? l / 2 : l;

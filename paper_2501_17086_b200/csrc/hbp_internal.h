@@ -86,6 +86,9 @@ int gemm_tc_stats_slots(int N);
 extern bool g_force_simt;
 
 // ---------------------------------------------------------------- scans and elementwise (scan.cu)
+// Internal gate kind beside the public hbp_gate values: a[L][rows][d], one gate per element and step (the
+// state-dependent gate of a GRU, produced by its forward pass).
+constexpr int kGateElement = 3;
 struct ScanArgs {
   int dtype = HBP_F32;
   int L = 0;               // number of steps in the buffers
@@ -100,7 +103,7 @@ struct ScanArgs {
   const void* delta = nullptr;  // per hbp_loss
   int loss = HBP_LOSS_FINAL;
   const void* a = nullptr;  // gate
-  int gate = HBP_GATE_ONE;
+  int gate = HBP_GATE_ONE;  // an hbp_gate value, or kGateElement
   void* g = nullptr;  // [L+1][rows][d]
   // LayerNorm-backward finish: u is dY; the kernel forms rstd * (dy - mean(dy) - xhat * mean(dy*xhat)).
   // xhat [L][rows][d] in dtype, rstd [L][rows] float.
@@ -141,6 +144,20 @@ void rnn_backward_step(Launcher& lc, int dtype, const void* W, const void* deriv
                        const double* g_in, double* g_out, void* g_store, int B, int d);
 void convert_to_f64(Launcher& lc, int dtype, const void* src, double* dst, int64_t elems);
 
+// ---------------------------------------------------------------- GRU (gru.cu)
+// One forward step in double from the double master state; writes the new master, the stored state, the
+// gate z [B][d] and the VJP coefficients c4 [B][4d] = [c_r | c_z | c_nr | c_n].
+void gru_forward_step(Launcher& lc, int dtype, const void* W, const void* U, const void* x_t, const double* h_in,
+                      double* h_out, void* zc, void* c4, void* state_out, int B, int d, int in_dim);
+// g_t = delta_t + z_t * g_{t+1} + (g_{t+1} * [c_r | c_z | c_nr]) W in double from the double master g_in.
+void gru_backward_step(Launcher& lc, int dtype, const void* W, const void* zc, const void* c4, const void* delta,
+                       const double* g_in, double* g_out, void* g_store, int B, int d);
+// a4[row][q*d + c] = g[row][c] * c4[row][q*d + c], in dtype.
+void gru_operand(Launcher& lc, int dtype, const void* g, const void* c4, void* a4, int64_t rows, int d);
+// tf32 high/low split of g * c4: columns [0, 3d) as [rows][3d], or all of it transposed as [4d][rows].
+void gru_split(Launcher& lc, const float* g, const float* c4, float* hi, float* lo, int64_t rows, int d);
+void gru_split_transposed(Launcher& lc, const float* g, const float* c4, float* hiT, float* loT, int64_t rows, int d);
+
 // ---------------------------------------------------------------- attention (attention.cu)
 struct AttnArgs {
   int dtype = HBP_BF16;
@@ -167,6 +184,12 @@ bool attention_bwd_tc(Launcher& lc, const AttnArgs& a, int* status_word);
 __device__ __forceinline__ float gelu_f(float z) { return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f)); }
 __device__ __forceinline__ float gelu_prime_f(float z) {
   return 0.5f * (1.0f + erff(z * 0.70710678118654752440f)) + z * expf(-0.5f * z * z) * 0.39894228040143267794f;
+}
+// v rounded to tf32 precision (13 low mantissa bits cleared, round to nearest even)
+__device__ __forceinline__ float round_tf32(float v) {
+  uint32_t u = __float_as_uint(v);
+  u += 0x00000fffu + ((u >> 13) & 1u);
+  return __uint_as_float(u & 0xffffe000u);
 }
 __device__ __forceinline__ float to_f(float v) { return v; }
 __device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }

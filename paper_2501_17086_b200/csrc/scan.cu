@@ -75,10 +75,12 @@ __device__ __forceinline__ const T* delta_at(const ScanArgs& s, int l, int64_t s
   if (s.loss == HBP_LOSS_EVERY_STEP) return (s.u_has_delta && l < s.L) ? nullptr : (const T*)s.delta + (int64_t)l * state_elems;
   return (l == s.L) ? (const T*)s.delta : nullptr;
 }
+// gate vector of step l for the 16-byte group at element `off` of the state, channel `ch` (nullptr = ones)
 template <typename T>
-__device__ __forceinline__ const T* gate_at(const ScanArgs& s, int l) {
+__device__ __forceinline__ const T* gate_at(const ScanArgs& s, int l, int64_t state_elems, int64_t off, int ch) {
   if (s.gate == HBP_GATE_ONE || !s.a) return nullptr;
-  return (const T*)s.a + (s.gate == HBP_GATE_CHANNEL_PER_STEP ? (int64_t)l * s.d : 0);
+  if (s.gate == kGateElement) return (const T*)s.a + (int64_t)l * state_elems + off;
+  return (const T*)s.a + (s.gate == HBP_GATE_CHANNEL_PER_STEP ? (int64_t)l * s.d : 0) + ch;
 }
 
 // One step of the recurrence for a 16-byte channel group: val = a * carry + u + delta.
@@ -86,10 +88,10 @@ template <typename T>
 __device__ __forceinline__ void scan_step(const ScanArgs& s, int l, int64_t state_elems, int64_t off, int ch,
                                           const typename Acc<T>::type* carry, typename Acc<T>::type* val) {
   constexpr int V = Vec<T>::N;
-  const T* gp = gate_at<T>(s, l);
+  const T* gp = gate_at<T>(s, l, state_elems, off, ch);
   if (gp) {
     float a[V];
-    ldv<T>(gp + ch).get(a);
+    ldv<T>(gp).get(a);
 #pragma unroll
     for (int i = 0; i < V; ++i) val[i] = a[i] * carry[i];
   } else {
@@ -167,10 +169,10 @@ __global__ void __launch_bounds__(256) scan_depth_lnstat_kernel(const ScanArgs s
     ldv_stream<T>((const T*)s.u + (int64_t)l * state_elems + off).get(dy);
     ldv_stream<T>((const T*)s.xhat + (int64_t)l * state_elems + off).get(xh);
     const float4 st = __ldg(s.lnstat + (int64_t)l * s.rows + row);
-    const T* gp = gate_at<T>(s, l);
+    const T* gp = gate_at<T>(s, l, state_elems, off, ch);
     if (gp) {
       float a[V];
-      ldv<T>(gp + ch).get(a);
+      ldv<T>(gp).get(a);
 #pragma unroll
       for (int i = 0; i < V; ++i) val[i] = a[i] * carry[i];
     } else {
@@ -270,10 +272,10 @@ __global__ void __launch_bounds__(1024) scan_depth_ln_kernel(const ScanArgs s) {
     const float r = s.rstd[(int64_t)l * s.rows + row];
     if (active) {
       float val[V];
-      const T* gp = gate_at<T>(s, l);
+      const T* gp = gate_at<T>(s, l, state_elems, off, (int)threadIdx.x * V);
       if (gp) {
         float a[V];
-        ldv<T>(gp + threadIdx.x * V).get(a);
+        ldv<T>(gp).get(a);
 #pragma unroll
         for (int i = 0; i < V; ++i) val[i] = a[i] * carry[i];
       } else {
@@ -344,10 +346,10 @@ __global__ void __launch_bounds__(128) scan_chunk_kernel(const ScanArgs s, typen
       out.set(val);
       stv<T>(g + (int64_t)l * state_elems + off, out);
     } else {
-      const T* gp = gate_at<T>(s, l);
+      const T* gp = gate_at<T>(s, l, state_elems, off, ch);
       if (gp) {
         float a[V];
-        ldv<T>(gp + ch).get(a);
+        ldv<T>(gp).get(a);
 #pragma unroll
         for (int i = 0; i < V; ++i) prod[i] *= a[i];
       }
@@ -451,13 +453,8 @@ __global__ void __launch_bounds__(256) gate_grad_kernel(const T* __restrict__ g,
   }
 }
 
-// v = a * b (b optional); hi = v rounded to tf32 precision (13 low mantissa bits cleared), lo = the same
-// rounding of v - hi.  hi + lo carries 21+ bits of v, and both are exact tf32 operands.
-__device__ __forceinline__ float round_tf32(float v) {
-  uint32_t u = __float_as_uint(v);
-  u += 0x00000fffu + ((u >> 13) & 1u);  // round to nearest even at bit 13
-  return __uint_as_float(u & 0xffffe000u);
-}
+// v = a * b (b optional); hi = v rounded to tf32 precision, lo = the same rounding of v - hi.  hi + lo carries
+// 21+ bits of v, and both are exact tf32 operands.
 __global__ void split_tf32_kernel(const float4* __restrict__ a, const float4* __restrict__ b, float4* __restrict__ hi,
                                   float4* __restrict__ lo, int64_t nvec) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;

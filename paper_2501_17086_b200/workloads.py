@@ -24,7 +24,7 @@ import torch
 @dataclasses.dataclass(frozen=True)
 class Workload:
     name: str
-    block: str            # "mlp" | "preln_mlp" | "rnn_tanh" | "preln_transformer"
+    block: str            # "mlp" | "preln_mlp" | "rnn_tanh" | "preln_transformer" | "gru"
     dtype: str            # "f32" | "bf16"
     L: int                # residual steps (mlp), time steps (rnn), decoder blocks (transformer)
     d: int
@@ -57,6 +57,11 @@ WORKLOADS = {
     "c4": Workload("c4", "preln_transformer", "bf16", L=24, d=768, hidden=3072, n_heads=12, head_dim=64,
                    seq=1024, batch=16, tokens=16384, seed=1004),
     "c5": Workload("c5", "preln_mlp", "bf16", L=128, d=2048, hidden=8192, batch=32, seq=512, tokens=16384, seed=1005),
+    # GRU cells with the update gate as the residual gate, in the shapes of the paper's recurrent experiments
+    # (Table of RNN hyperparameters: batch 128; 256 steps x 512 units on characters, 1024 steps x 64 units on
+    # pixels); the input widths 210 and 3 are rounded up to multiples of 4 for 128-bit access
+    "g1": Workload("g1", "gru", "f32", L=256, d=512, in_dim=212, batch=128, tokens=128, seed=1006, loss="every_mse"),
+    "g2": Workload("g2", "gru", "f32", L=1024, d=64, in_dim=4, batch=128, tokens=128, seed=1007, loss="every_mse"),
     # c2 with 8 layers: same per-launch tile shapes, small enough for multi-pass profiler captures
     "c2_small": Workload("c2_small", "preln_mlp", "bf16", L=8, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1012),
     # c4 with 4 decoder blocks: same per-launch shapes, small enough for multi-pass profiler captures
@@ -67,6 +72,11 @@ WORKLOADS = {
     "c2_twin": Workload("c2_twin", "preln_mlp", "bf16", L=5, d=256, hidden=1024, batch=1, seq=328, tokens=328, seed=2002),
     "c2_twin_f32": Workload("c2_twin_f32", "preln_mlp", "f32", L=5, d=96, hidden=200, batch=1, seq=77, tokens=77, seed=2012),
     "c3_twin": Workload("c3_twin", "rnn_tanh", "f32", L=200, d=128, in_dim=48, batch=6, tokens=6, seed=2003, loss="every_mse"),
+    "gru_twin": Workload("gru_twin", "gru", "f32", L=40, d=72, in_dim=12, batch=5, tokens=5, seed=2006, loss="every_mse"),
+    "gru_twin_long": Workload("gru_twin_long", "gru", "f32", L=300, d=64, in_dim=4, batch=12, tokens=12, seed=2016,
+                              loss="every_mse"),
+    "gru_twin_bf16": Workload("gru_twin_bf16", "gru", "bf16", L=24, d=64, in_dim=16, batch=6, tokens=6, seed=2026,
+                              loss="every_mse"),
     "c4_twin": Workload("c4_twin", "preln_transformer", "bf16", L=2, d=128, hidden=512, n_heads=2, head_dim=64,
                         seq=200, batch=2, tokens=400, seed=2004),
     "c4_twin_f32": Workload("c4_twin_f32", "preln_transformer", "f32", L=2, d=64, hidden=128, n_heads=2, head_dim=32,
@@ -84,6 +94,7 @@ def make_inputs(cfg: Workload, device="cpu"):
 
     Keys: mlp / preln_mlp: W1 [L,h,d], W2 [L,d,h], x0 [N,d], y [N,d].
     rnn_tanh: a [d], W [d,d], U [d,in], X [T,B,in], Y [T,B,d], x0 [B,d] (zeros).
+    gru: W [3d,d] (variance 1/d), U [3d,in] (variance 1/in), X, Y, x0 as for rnn_tanh.
     preln_transformer: Wq, Wk, Wv, Wo [L,d,d], W1 [L,h,d], W2 [L,d,h], x0 [N,d], y [N,d].
     Standard deviations: 0.02 for Transformer-style inputs weights and
     0.02 / sqrt(2 * steps) for the weights that write into the residual stream;
@@ -115,6 +126,13 @@ def make_inputs(cfg: Workload, device="cpu"):
         q = q * torch.sign(torch.diagonal(r)).unsqueeze(0)
         out["W"] = (0.5 * q).contiguous().to(dev).to(dt)
         out["U"] = _randn(gen, (d, nin), 1.0 / math.sqrt(nin), dev).to(dt)
+        out["X"] = _randn(gen, (T, B, nin), 1.0, dev).to(dt)
+        out["Y"] = _randn(gen, (T, B, d), 1.0, dev).to(dt)
+        out["x0"] = torch.zeros((B, d), device=dev, dtype=dt)
+    elif cfg.block == "gru":
+        T, d, B, nin = cfg.L, cfg.d, cfg.batch, cfg.in_dim
+        out["W"] = _randn(gen, (3 * d, d), 1.0 / math.sqrt(d), dev).to(dt)
+        out["U"] = _randn(gen, (3 * d, nin), 1.0 / math.sqrt(nin), dev).to(dt)
         out["X"] = _randn(gen, (T, B, nin), 1.0, dev).to(dt)
         out["Y"] = _randn(gen, (T, B, d), 1.0, dev).to(dt)
         out["x0"] = torch.zeros((B, d), device=dev, dtype=dt)
