@@ -268,8 +268,8 @@ def run_ours(args):
                     "frac": (3 * alg / tf32_peak) if alg else None, "algorithmic_tflops": alg,
                     "fp32_alu_peak_tflops": 148 * 128 * 2 * 1.965e9 / 1e12,
                     "peak_source": "of measured bf16 x nominal tf32/bf16 ratio" if peaks else "of fallback", "traffic": None}
-    # scan: read u (+ xhat when the LayerNorm finish is fused), write g
-    tensors = 2 + (1 if w.block in ("preln_mlp", "preln_transformer") else 0)  # per-step delta is added by the VJP GEMM epilogue
+    # scan: read u (+ xhat when the LayerNorm finish is fused, + the per-element gate of a GRU), write g
+    tensors = 2 + (1 if w.block in ("preln_mlp", "preln_transformer", "gru") else 0)  # per-step delta is added by the VJP GEMM epilogue
     scan_bytes = tensors * w.steps * w.tokens * w.d * es
     hbm = peaks.get("hbm_gbs", 6650.0)
     scan_iter_ms = None

@@ -171,3 +171,20 @@ def test_gamma_shifted_split_matches_oracle(name, gamma):
     pg = O.param_grads(st, caches, xs, O.highway_bp(st, caches, deltas, 2), groups)
     for n, v in pg.items():
         assert rel(np64(grads["d" + n]), v) < tol, n
+
+
+@pytest.mark.parametrize("name,ks", [("gru_twin", (1, 3)), ("c3_twin", (2,)), ("c2_twin", (2,)), ("c4_twin", (2,))])
+def test_cuda_core_fallback_matches_oracle(name, ks, monkeypatch):
+    """HBP_FORCE_SIMT=1 (read when a context is made) keeps every GEMM and the attention backward off the
+    tensor cores: the fallback kernels must meet the same bar."""
+    from oracle import run as orun
+    from paper_2501_17086_b200.workloads import WORKLOADS, make_inputs
+    from test_gpu_parity import compare, run_gpu
+    monkeypatch.setenv("HBP_FORCE_SIMT", "1")
+    w = WORKLOADS[name]
+    inp = make_inputs(w, "cuda")
+    gpu = run_gpu(w, inp, ks)
+    del gpu["ctx"]
+    kmax = max(ks)
+    ref = orun.run(w, inp, ks=ks, grads_for=("exact", kmax))
+    compare(w, gpu, ref, ks, ("exact", kmax))
