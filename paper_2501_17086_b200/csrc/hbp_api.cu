@@ -503,6 +503,7 @@ struct Run {
       if (c->lnpart && stats_ok) s.lnstat = c->lnstat;
     }
     s.scratch = c->scan_scratch; s.scratch_bytes = c->scan_scratch_bytes;
+    s.status = c->status;
     return s;
   }
   void set_last_state() {

@@ -1,0 +1,262 @@
+// Reverse scan over time for problems with few channels (Eq. 9 / Eq. 12 with diagonal K; the recurrent
+// workloads: hundreds to thousands of steps, 10^4..10^5 channels).  There are too few independent recurrences
+// to hide memory latency with threads, so each block hides it with a deep ring of TMA loads instead: a block
+// owns 512 bytes of channels (128 floats / 256 bf16) and walks all steps serially, one 32-bit word of channels
+// per lane; a producer warp keeps the ring of {kRows steps x 512 bytes} boxes full per input stream (u, a
+// separately given delta, an element-wise gate), and four consumer warps - one per scheduler, so that the
+// float <-> double conversions of the running value spread over all four conversion pipes - apply
+// g = a * g + u step by step and store g.  Every input byte is read once and every output byte written once,
+// with no scratch, no hand-over between blocks and nothing to wait for but this block's own loads.
+#include "tc_common.cuh"
+
+namespace hbp {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kRows = 8;                        // steps per ring stage
+constexpr int kRowBytes = 512;                  // channel bytes per block
+constexpr int kStageBytes = kRows * kRowBytes;  // per stream
+constexpr int kRingBudget = 192 * 1024;         // shared memory an SM gives to rings, split among its blocks
+constexpr int kMaxStages = 48;
+constexpr int kConsumerWarps = 4;
+
+template <typename T>
+struct RingAcc {
+  typedef float type;
+};
+template <>
+struct RingAcc<float> {
+  typedef double type;  // thousands of dependent steps at 1e-5: the running value is carried in double
+};
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+               "l"(tm), "r"(bar), "r"(c0), "r"(c1)
+               : "memory");
+}
+
+template <typename T>
+__device__ __forceinline__ void unpack_word(uint32_t w, float* f);
+template <>
+__device__ __forceinline__ void unpack_word<float>(uint32_t w, float* f) {
+  f[0] = __uint_as_float(w);
+}
+template <>
+__device__ __forceinline__ void unpack_word<bf16>(uint32_t w, float* f) {
+  f[0] = __uint_as_float(w << 16);
+  f[1] = __uint_as_float(w & 0xffff0000u);
+}
+
+// NS additive streams (0..2: u and/or a per-step delta), kElemGate: a gate value per element and step.
+// m0, m1: maps of the additive streams, mg: map of the gate; all [steps][rows * d] with boxes of
+// {512 bytes, kRows}.  Row y of every map is step y.
+template <typename T, int NS, bool kElemGate>
+__global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(const ScanArgs s,
+                                                                             const __grid_constant__ CUtensorMap m0,
+                                                                             const __grid_constant__ CUtensorMap m1,
+                                                                             const __grid_constant__ CUtensorMap mg,
+                                                                             int nstages) {
+  typedef typename RingAcc<T>::type A;
+  constexpr int EPT = 4 / (int)sizeof(T);  // channels per lane: one 32-bit word
+  constexpr int STREAMS = NS + (kElemGate ? 1 : 0);
+  extern __shared__ __align__(128) unsigned char ring_raw[];
+  unsigned char* ring = reinterpret_cast<unsigned char*>(((uintptr_t)ring_raw + 127) & ~(uintptr_t)127);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)nstages * STREAMS * kStageBytes);
+  int* abort_flag = reinterpret_cast<int*>(bars + 2 * nstages);
+  int* local_status = abort_flag + 1;
+  auto full_bar = [&](int i) { return smem_u32(bars + i); };
+  auto empty_bar = [&](int i) { return smem_u32(bars + nstages + i); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t state = s.rows * s.d;
+  const int x0 = (int)((int64_t)blockIdx.x * (kRowBytes / (int)sizeof(T)));
+  const int nsteps = s.l_hi - s.l_lo;
+  const int niter = (nsteps + kRows - 1) / kRows;
+  int* status = s.status ? s.status : local_status;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < nstages; ++i) {
+      mbar_init(full_bar(i), 1);
+      mbar_init(empty_bar(i), kConsumerWarps);
+    }
+    *abort_flag = 0;
+    *local_status = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  __syncthreads();
+
+  if (warp == kConsumerWarps) {
+    // ---- producer: one lane keeps the ring full ----------------------------------------------------
+    if (lane == 0) {
+      int issued = 0;
+      for (int k = 0; k < niter; ++k) {
+        const int slot = k % nstages;
+        if (k >= nstages && !mbar_wait(empty_bar(slot), (uint32_t)((k / nstages - 1) & 1), abort_flag, status)) break;
+        mbar_expect_tx(full_bar(slot), STREAMS * kStageBytes);
+        const int y = s.l_hi - (k + 1) * kRows;  // may start below step 0 in the last stage: zero fill
+        const uint32_t dst = smem_u32(ring + (size_t)slot * STREAMS * kStageBytes);
+        if (NS >= 1) tma_load_2d(dst, &m0, full_bar(slot), x0, y);
+        if (NS >= 2) tma_load_2d(dst + kStageBytes, &m1, full_bar(slot), x0, y);
+        if (kElemGate) tma_load_2d(dst + NS * kStageBytes, &mg, full_bar(slot), x0, y);
+        issued = k + 1;
+      }
+      // nothing of this block may still be in flight when it ends (only reachable with work left after an abort)
+      const int first = issued > nstages ? issued - nstages : 0;
+      for (int k = first; k < issued; ++k) {
+        const uint64_t t0 = global_ns();
+        while (!mbar_try_wait(full_bar(k % nstages), (uint32_t)((k / nstages) & 1)))
+          if (global_ns() - t0 > WAIT_LIMIT_NS) break;
+      }
+    }
+    return;
+  }
+
+  // ---- consumers: warp w owns 32-bit words [32 w, 32 (w + 1)) of the block's 512-byte row ---------------
+  const int word = warp * 32 + lane;
+  const int64_t e0 = (int64_t)x0 + (int64_t)word * EPT;
+  const bool live = e0 < state;
+  T* g = (T*)s.g;
+  A carry[EPT];
+  float a0[EPT];
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    carry[e] = live ? (A)to_f(g[(int64_t)s.l_hi * state + e0 + e]) : (A)0;
+    a0[e] = 1.0f;
+  }
+  if (!kElemGate && live && s.a && s.gate == HBP_GATE_CHANNEL_SHARED) {
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) a0[e] = to_f(((const T*)s.a)[(e0 + e) % s.d]);
+  }
+  for (int k = 0; k < niter; ++k) {
+    const int slot = k % nstages;
+    if (!mbar_wait(full_bar(slot), (uint32_t)((k / nstages) & 1), abort_flag, status)) break;
+    const unsigned char* stg = ring + (size_t)slot * STREAMS * kStageBytes + word * 4;
+    float uu[kRows][EPT], aa[kRows][EPT];
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) {
+        uu[r][e] = 0.0f;
+        aa[r][e] = a0[e];
+      }
+      if (NS >= 1) unpack_word<T>(*reinterpret_cast<const uint32_t*>(stg + r * kRowBytes), uu[r]);
+      if (NS >= 2) {
+        float t[EPT];
+        unpack_word<T>(*reinterpret_cast<const uint32_t*>(stg + kStageBytes + r * kRowBytes), t);
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) uu[r][e] += t[e];
+      }
+      if (kElemGate) unpack_word<T>(*reinterpret_cast<const uint32_t*>(stg + NS * kStageBytes + r * kRowBytes), aa[r]);
+    }
+    const int l_base = s.l_hi - (k + 1) * kRows;
+#pragma unroll
+    for (int r = kRows - 1; r >= 0; --r) {
+      const int l = l_base + r;
+      if (l < s.l_lo) break;
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) carry[e] = (A)aa[r][e] * carry[e] + (A)uu[r][e];
+      if (live) {
+        if (EPT == 1) {
+          g[(int64_t)l * state + e0] = from_f<T>((float)carry[0]);
+        } else {
+          *reinterpret_cast<__nv_bfloat162*>(g + (int64_t)l * state + e0) =
+              __floats2bfloat162_rn((float)carry[0], (float)carry[EPT - 1]);
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty_bar(slot));
+  }
+}
+
+bool make_map2(CUtensorMap* tm, const void* base, bool f32, int64_t steps, int64_t state) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || ((uintptr_t)base & 15u)) return false;
+  const cuuint64_t es = f32 ? 4 : 2;
+  if ((state * es) % 16) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)state, (cuuint64_t)steps};
+  cuuint64_t strides[1] = {(cuuint64_t)state * es};
+  cuuint32_t box[2] = {(cuuint32_t)(kRowBytes / es), (cuuint32_t)kRows}, estr[2] = {1, 1};
+  return fn(tm, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <typename T, int NS, bool kElemGate>
+void launch_ring(Launcher& lc, const ScanArgs& s, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& mg,
+                 unsigned grid, int nstages, size_t smem) {
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaFuncSetAttribute(scan_ring_kernel<T, NS, kElemGate>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    configured = smem;
+  }
+  scan_ring_kernel<T, NS, kElemGate><<<grid, (kConsumerWarps + 1) * 32, smem, lc.stream>>>(s, m0, m1, mg, nstages);
+  lc.count();
+  lc.check();
+}
+
+template <typename T>
+void dispatch_ring(Launcher& lc, const ScanArgs& s, int ns, bool eg, const CUtensorMap& m0, const CUtensorMap& m1,
+                   const CUtensorMap& mg, unsigned grid, int nstages, size_t smem) {
+  if (eg) {
+    if (ns == 0) launch_ring<T, 0, true>(lc, s, m0, m1, mg, grid, nstages, smem);
+    else if (ns == 1) launch_ring<T, 1, true>(lc, s, m0, m1, mg, grid, nstages, smem);
+    else launch_ring<T, 2, true>(lc, s, m0, m1, mg, grid, nstages, smem);
+  } else {
+    if (ns == 1) launch_ring<T, 1, false>(lc, s, m0, m1, mg, grid, nstages, smem);
+    else launch_ring<T, 2, false>(lc, s, m0, m1, mg, grid, nstages, smem);
+  }
+}
+
+}  // namespace
+
+bool scan_ring(Launcher& lc, const ScanArgs& s, int min_blocks) {
+  if (s.xhat || s.keep != 1.0f || s.gamma != 0.0f) return false;
+  if (s.gate == HBP_GATE_CHANNEL_PER_STEP && s.a) return false;  // a small [steps][d] table: not a stream of this shape
+  const bool f32 = s.dtype == HBP_F32;
+  const int64_t state = s.rows * s.d;
+  const int nsteps = s.l_hi - s.l_lo;
+  if (nsteps < 2 * kRows || state <= 0 || state > 0x7fffffff) return false;
+  const int row_elems = kRowBytes / (f32 ? 4 : 2);
+  const unsigned grid = (unsigned)((state + row_elems - 1) / row_elems);
+  if ((int64_t)grid < (int64_t)min_blocks) return false;
+  // the additive streams: u, and delta when it is given per step and not already inside u
+  const void* streams[2] = {nullptr, nullptr};
+  int64_t stream_rows[2] = {0, 0};
+  int ns = 0;
+  if (s.u) {
+    streams[ns] = s.u;
+    stream_rows[ns++] = s.L;
+  }
+  if (s.delta && s.loss == HBP_LOSS_EVERY_STEP && !(s.u && s.u_has_delta)) {
+    streams[ns] = s.delta;
+    stream_rows[ns++] = (int64_t)s.L + 1;
+  }
+  const bool eg = s.a && s.gate == kGateElement;
+  if (ns == 0 && !eg) return false;  // nothing to stream: a pure broadcast
+  CUtensorMap m0, m1, mg;
+  if (ns >= 1 && !make_map2(&m0, streams[0], f32, stream_rows[0], state)) return false;
+  if (ns >= 2 && !make_map2(&m1, streams[1], f32, stream_rows[1], state)) return false;
+  if (eg && !make_map2(&mg, s.a, f32, s.L, state)) return false;
+  if (ns == 0) m0 = mg;  // unused maps still have to be valid objects
+  if (ns < 2) m1 = m0;
+  if (!eg) mg = m0;
+  const int nstreams = ns + (eg ? 1 : 0);
+  const int sms = sm_count();
+  int per_sm = (int)((grid + sms - 1) / sms);
+  if (per_sm > 4) per_sm = 4;
+  int nstages = kRingBudget / per_sm / (nstreams * kStageBytes);
+  const int niter = (nsteps + kRows - 1) / kRows;
+  if (nstages > niter) nstages = niter;
+  if (nstages > kMaxStages) nstages = kMaxStages;
+  if (nstages < 2) return false;
+  const size_t smem = (size_t)nstages * nstreams * kStageBytes + (size_t)nstages * 16 + 16 + 128;
+  if (f32) dispatch_ring<float>(lc, s, ns, eg, m0, m1, mg, grid, nstages, smem);
+  else dispatch_ring<bf16>(lc, s, ns, eg, m0, m1, mg, grid, nstages, smem);
+  return true;
+}
+
+}  // namespace hbp
