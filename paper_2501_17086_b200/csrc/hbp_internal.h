@@ -118,9 +118,9 @@ struct ScanArgs {
 };
 size_t scan_scratch_bytes(int dtype, int L, int64_t rows, int d);
 void scan_reverse(Launcher& lc, const ScanArgs& s);
-// TMA-ring scan, serial in time, for few channels (scan_ring.cu); false if the problem does not qualify or
-// would make fewer than min_blocks blocks (nothing launched then).
-bool scan_ring(Launcher& lc, const ScanArgs& s, int min_blocks);
+// TMA-ring scan, serial in time, for few channels (scan_ring.cu); false if the problem does not qualify
+// (nothing launched then).
+bool scan_ring(Launcher& lc, const ScanArgs& s);
 // lnstat[l][row] = {rstd, sum_slots s1 / d, sum_slots s2 / d, 0} from the GEMM's partial sums.
 void ln_stats_finish(Launcher& lc, const float2* stats, int slots, const float* rstd, float4* lnstat, int64_t count,
                      int d);

@@ -317,7 +317,6 @@ __global__ void __launch_bounds__(1024) scan_depth_ln_kernel(const ScanArgs s) {
 // carry-in, writing g.  Scratch: S (then the carry-ins) [nchunks][rows*d] and P likewise, in the
 // accumulator type (double for float data).
 constexpr int kChunk = 32;
-constexpr int kRingMinBlocks = 296;  // two blocks per SM
 
 template <typename T, bool kApply>
 __global__ void __launch_bounds__(128) scan_chunk_kernel(const ScanArgs s, typename Acc<T>::type* __restrict__ S,
@@ -538,9 +537,9 @@ void scan_reverse(Launcher& lc, const ScanArgs& s) {
   }
   const int steps = s.l_hi - s.l_lo;
   const size_t need = scan_scratch_bytes(s.dtype, steps, s.rows, s.d);
-  // few channels, many steps: with enough blocks to put several warps on every scheduler, one serial pass in
-  // time behind a ring of TMA loads reads and writes every byte once
-  if (need > 0 && scan_ring(lc, s, kRingMinBlocks)) return;
+  // few channels, many steps: one serial pass in time behind a ring of TMA loads reads and writes every byte
+  // once; the three-phase form below remains for what that kernel does not take (a gate table per step)
+  if (need > 0 && scan_ring(lc, s)) return;
   if (need > 0 && s.scratch && s.scratch_bytes >= need && s.keep == 1.0f && s.gamma == 0.0f) {
     const int nchunks = (steps + kChunk - 1) / kChunk;
     dim3 grid((unsigned)((nvec + 127) / 128), nchunks);

@@ -2,11 +2,13 @@
 // workloads: hundreds to thousands of steps, 10^4..10^5 channels).  There are too few independent recurrences
 // to hide memory latency with threads, so each block hides it with a deep ring of TMA loads instead: a block
 // owns 512 bytes of channels (128 floats / 256 bf16) and walks all steps serially, one 32-bit word of channels
-// per lane; a producer warp keeps the ring of {kRows steps x 512 bytes} boxes full per input stream (u, a
+// per lane; a producer warp keeps the ring of {8..64 steps x 512 bytes} boxes full per input stream (u, a
 // separately given delta, an element-wise gate), and four consumer warps - one per scheduler, so that the
 // float <-> double conversions of the running value spread over all four conversion pipes - apply
 // g = a * g + u step by step and store g.  Every input byte is read once and every output byte written once,
 // with no scratch, no hand-over between blocks and nothing to wait for but this block's own loads.
+#include <type_traits>
+
 #include "tc_common.cuh"
 
 namespace hbp {
@@ -15,11 +17,11 @@ namespace {
 
 using namespace tc;
 
-constexpr int kRows = 8;                        // steps per ring stage
+constexpr int kMaxRows = 64;                    // steps per ring stage (one TMA box per stream): 8, 16, 32 or 64
+constexpr int kSubRows = 8;                     // steps a consumer takes from shared memory at a time
 constexpr int kRowBytes = 512;                  // channel bytes per block
-constexpr int kStageBytes = kRows * kRowBytes;  // per stream
 constexpr int kRingBudget = 192 * 1024;         // shared memory an SM gives to rings, split among its blocks
-constexpr int kMaxStages = 48;
+constexpr int kMaxStages = 24;
 constexpr int kConsumerWarps = 4;
 
 template <typename T>
@@ -51,16 +53,18 @@ __device__ __forceinline__ void unpack_word<bf16>(uint32_t w, float* f) {
 
 // NS additive streams (0..2: u and/or a per-step delta), kElemGate: a gate value per element and step.
 // m0, m1: maps of the additive streams, mg: map of the gate; all [steps][rows * d] with boxes of
-// {512 bytes, kRows}.  Row y of every map is step y.
+// {512 bytes, rows_ps}.  Row y of every map is step y.
 template <typename T, int NS, bool kElemGate>
 __global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(const ScanArgs s,
                                                                              const __grid_constant__ CUtensorMap m0,
                                                                              const __grid_constant__ CUtensorMap m1,
                                                                              const __grid_constant__ CUtensorMap mg,
-                                                                             int nstages) {
+                                                                             int nstages, int rows_ps) {
   typedef typename RingAcc<T>::type A;
   constexpr int EPT = 4 / (int)sizeof(T);  // channels per lane: one 32-bit word
   constexpr int STREAMS = NS + (kElemGate ? 1 : 0);
+  const int kRows = rows_ps;                       // steps per ring stage
+  const int kStageBytes = rows_ps * kRowBytes;  // per stream
   extern __shared__ __align__(128) unsigned char ring_raw[];
   unsigned char* ring = reinterpret_cast<unsigned char*>(((uintptr_t)ring_raw + 127) & ~(uintptr_t)127);
   uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)nstages * STREAMS * kStageBytes);
@@ -130,13 +134,13 @@ __global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(co
 #pragma unroll
     for (int e = 0; e < EPT; ++e) a0[e] = to_f(((const T*)s.a)[(e0 + e) % s.d]);
   }
-  for (int k = 0; k < niter; ++k) {
-    const int slot = k % nstages;
-    if (!mbar_wait(full_bar(slot), (uint32_t)((k / nstages) & 1), abort_flag, status)) break;
-    const unsigned char* stg = ring + (size_t)slot * STREAMS * kStageBytes + word * 4;
-    float uu[kRows][EPT], aa[kRows][EPT];
+  T* gp = g + (int64_t)(s.l_hi - 1) * state + e0;  // where the next step's value goes
+  // kSub rows of one stage, later steps first; `check` = the stage reaches below the first step
+  auto sub_block = [&](const unsigned char* stg, int l_top, auto check) {
+    constexpr bool kCheck = decltype(check)::value;
+    float uu[kSubRows][EPT], aa[kSubRows][EPT];
 #pragma unroll
-    for (int r = 0; r < kRows; ++r) {
+    for (int r = 0; r < kSubRows; ++r) {
 #pragma unroll
       for (int e = 0; e < EPT; ++e) {
         uu[r][e] = 0.0f;
@@ -151,35 +155,45 @@ __global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(co
       }
       if (kElemGate) unpack_word<T>(*reinterpret_cast<const uint32_t*>(stg + NS * kStageBytes + r * kRowBytes), aa[r]);
     }
-    const int l_base = s.l_hi - (k + 1) * kRows;
 #pragma unroll
-    for (int r = kRows - 1; r >= 0; --r) {
-      const int l = l_base + r;
-      if (l < s.l_lo) break;
+    for (int r = kSubRows - 1; r >= 0; --r) {
+      if (kCheck && l_top - (kSubRows - 1 - r) < s.l_lo) break;
 #pragma unroll
       for (int e = 0; e < EPT; ++e) carry[e] = (A)aa[r][e] * carry[e] + (A)uu[r][e];
       if (live) {
-        if (EPT == 1) {
-          g[(int64_t)l * state + e0] = from_f<T>((float)carry[0]);
-        } else {
-          *reinterpret_cast<__nv_bfloat162*>(g + (int64_t)l * state + e0) =
-              __floats2bfloat162_rn((float)carry[0], (float)carry[EPT - 1]);
-        }
+        if (EPT == 1) *gp = from_f<T>((float)carry[0]);
+        else *reinterpret_cast<__nv_bfloat162*>(gp) = __floats2bfloat162_rn((float)carry[0], (float)carry[EPT - 1]);
       }
+      gp -= state;
+    }
+  };
+  for (int k = 0; k < niter; ++k) {
+    const int slot = k % nstages;
+    if (!mbar_wait(full_bar(slot), (uint32_t)((k / nstages) & 1), abort_flag, status)) break;
+    const unsigned char* stg = ring + (size_t)slot * STREAMS * kStageBytes + word * 4;
+    const int l_base = s.l_hi - (k + 1) * kRows;
+    if (l_base >= s.l_lo) {
+#pragma unroll 1
+      for (int sb = kRows / kSubRows - 1; sb >= 0; --sb)
+        sub_block(stg + sb * kSubRows * kRowBytes, l_base + sb * kSubRows + kSubRows - 1, std::false_type());
+    } else {
+#pragma unroll 1
+      for (int sb = kRows / kSubRows - 1; sb >= 0; --sb)
+        sub_block(stg + sb * kSubRows * kRowBytes, l_base + sb * kSubRows + kSubRows - 1, std::true_type());
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(empty_bar(slot));
   }
 }
 
-bool make_map2(CUtensorMap* tm, const void* base, bool f32, int64_t steps, int64_t state) {
+bool make_map2(CUtensorMap* tm, const void* base, bool f32, int64_t steps, int64_t state, int rows_ps) {
   EncodeTiledFn fn = encode_fn();
   if (!fn || ((uintptr_t)base & 15u)) return false;
   const cuuint64_t es = f32 ? 4 : 2;
   if ((state * es) % 16) return false;
   cuuint64_t dims[2] = {(cuuint64_t)state, (cuuint64_t)steps};
   cuuint64_t strides[1] = {(cuuint64_t)state * es};
-  cuuint32_t box[2] = {(cuuint32_t)(kRowBytes / es), (cuuint32_t)kRows}, estr[2] = {1, 1};
+  cuuint32_t box[2] = {(cuuint32_t)(kRowBytes / es), (cuuint32_t)rows_ps}, estr[2] = {1, 1};
   return fn(tm, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
             strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -187,42 +201,41 @@ bool make_map2(CUtensorMap* tm, const void* base, bool f32, int64_t steps, int64
 
 template <typename T, int NS, bool kElemGate>
 void launch_ring(Launcher& lc, const ScanArgs& s, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& mg,
-                 unsigned grid, int nstages, size_t smem) {
+                 unsigned grid, int nstages, int rows_ps, size_t smem) {
   static size_t configured = 0;
   if (smem > configured) {
     cudaFuncSetAttribute(scan_ring_kernel<T, NS, kElemGate>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     configured = smem;
   }
-  scan_ring_kernel<T, NS, kElemGate><<<grid, (kConsumerWarps + 1) * 32, smem, lc.stream>>>(s, m0, m1, mg, nstages);
+  scan_ring_kernel<T, NS, kElemGate><<<grid, (kConsumerWarps + 1) * 32, smem, lc.stream>>>(s, m0, m1, mg, nstages, rows_ps);
   lc.count();
   lc.check();
 }
 
 template <typename T>
 void dispatch_ring(Launcher& lc, const ScanArgs& s, int ns, bool eg, const CUtensorMap& m0, const CUtensorMap& m1,
-                   const CUtensorMap& mg, unsigned grid, int nstages, size_t smem) {
+                   const CUtensorMap& mg, unsigned grid, int nstages, int rows_ps, size_t smem) {
   if (eg) {
-    if (ns == 0) launch_ring<T, 0, true>(lc, s, m0, m1, mg, grid, nstages, smem);
-    else if (ns == 1) launch_ring<T, 1, true>(lc, s, m0, m1, mg, grid, nstages, smem);
-    else launch_ring<T, 2, true>(lc, s, m0, m1, mg, grid, nstages, smem);
+    if (ns == 0) launch_ring<T, 0, true>(lc, s, m0, m1, mg, grid, nstages, rows_ps, smem);
+    else if (ns == 1) launch_ring<T, 1, true>(lc, s, m0, m1, mg, grid, nstages, rows_ps, smem);
+    else launch_ring<T, 2, true>(lc, s, m0, m1, mg, grid, nstages, rows_ps, smem);
   } else {
-    if (ns == 1) launch_ring<T, 1, false>(lc, s, m0, m1, mg, grid, nstages, smem);
-    else launch_ring<T, 2, false>(lc, s, m0, m1, mg, grid, nstages, smem);
+    if (ns == 1) launch_ring<T, 1, false>(lc, s, m0, m1, mg, grid, nstages, rows_ps, smem);
+    else launch_ring<T, 2, false>(lc, s, m0, m1, mg, grid, nstages, rows_ps, smem);
   }
 }
 
 }  // namespace
 
-bool scan_ring(Launcher& lc, const ScanArgs& s, int min_blocks) {
+bool scan_ring(Launcher& lc, const ScanArgs& s) {
   if (s.xhat || s.keep != 1.0f || s.gamma != 0.0f) return false;
   if (s.gate == HBP_GATE_CHANNEL_PER_STEP && s.a) return false;  // a small [steps][d] table: not a stream of this shape
   const bool f32 = s.dtype == HBP_F32;
   const int64_t state = s.rows * s.d;
   const int nsteps = s.l_hi - s.l_lo;
-  if (nsteps < 2 * kRows || state <= 0 || state > 0x7fffffff) return false;
+  if (nsteps < 4 * kSubRows || state <= 0 || state > 0x7fffffff) return false;
   const int row_elems = kRowBytes / (f32 ? 4 : 2);
   const unsigned grid = (unsigned)((state + row_elems - 1) / row_elems);
-  if ((int64_t)grid < (int64_t)min_blocks) return false;
   // the additive streams: u, and delta when it is given per step and not already inside u
   const void* streams[2] = {nullptr, nullptr};
   int64_t stream_rows[2] = {0, 0};
@@ -237,25 +250,29 @@ bool scan_ring(Launcher& lc, const ScanArgs& s, int min_blocks) {
   }
   const bool eg = s.a && s.gate == kGateElement;
   if (ns == 0 && !eg) return false;  // nothing to stream: a pure broadcast
-  CUtensorMap m0, m1, mg;
-  if (ns >= 1 && !make_map2(&m0, streams[0], f32, stream_rows[0], state)) return false;
-  if (ns >= 2 && !make_map2(&m1, streams[1], f32, stream_rows[1], state)) return false;
-  if (eg && !make_map2(&mg, s.a, f32, s.L, state)) return false;
-  if (ns == 0) m0 = mg;  // unused maps still have to be valid objects
-  if (ns < 2) m1 = m0;
-  if (!eg) mg = m0;
   const int nstreams = ns + (eg ? 1 : 0);
   const int sms = sm_count();
   int per_sm = (int)((grid + sms - 1) / sms);
   if (per_sm > 4) per_sm = 4;
-  int nstages = kRingBudget / per_sm / (nstreams * kStageBytes);
-  const int niter = (nsteps + kRows - 1) / kRows;
+  // the longest stage (fewest producer round trips) that still leaves a ring of at least four stages
+  const int budget = kRingBudget / per_sm / nstreams;
+  int rows_ps = kMaxRows;
+  while (rows_ps > kSubRows && (budget / (rows_ps * kRowBytes) < 4 || nsteps < 2 * rows_ps)) rows_ps /= 2;
+  int nstages = budget / (rows_ps * kRowBytes);
+  const int niter = (nsteps + rows_ps - 1) / rows_ps;
   if (nstages > niter) nstages = niter;
   if (nstages > kMaxStages) nstages = kMaxStages;
   if (nstages < 2) return false;
-  const size_t smem = (size_t)nstages * nstreams * kStageBytes + (size_t)nstages * 16 + 16 + 128;
-  if (f32) dispatch_ring<float>(lc, s, ns, eg, m0, m1, mg, grid, nstages, smem);
-  else dispatch_ring<bf16>(lc, s, ns, eg, m0, m1, mg, grid, nstages, smem);
+  CUtensorMap m0, m1, mg;
+  if (ns >= 1 && !make_map2(&m0, streams[0], f32, stream_rows[0], state, rows_ps)) return false;
+  if (ns >= 2 && !make_map2(&m1, streams[1], f32, stream_rows[1], state, rows_ps)) return false;
+  if (eg && !make_map2(&mg, s.a, f32, s.L, state, rows_ps)) return false;
+  if (ns == 0) m0 = mg;  // unused maps still have to be valid objects
+  if (ns < 2) m1 = m0;
+  if (!eg) mg = m0;
+  const size_t smem = (size_t)nstages * nstreams * rows_ps * kRowBytes + (size_t)nstages * 16 + 16 + 128;
+  if (f32) dispatch_ring<float>(lc, s, ns, eg, m0, m1, mg, grid, nstages, rows_ps, smem);
+  else dispatch_ring<bf16>(lc, s, ns, eg, m0, m1, mg, grid, nstages, rows_ps, smem);
   return true;
 }
 
