@@ -114,7 +114,9 @@ __device__ __forceinline__ void scan_step(const ScanArgs& s, int l, int64_t stat
 }
 
 // ---- depth scan, no LayerNorm: one thread per 16-byte channel group, serial over l -----------------
-template <typename T>
+// kShift: the shifted split (gamma > 0), which also reads the previous iterate; compiled apart so that the plain
+// scan carries no registers for it
+template <typename T, bool kShift>
 __global__ void __launch_bounds__(256) scan_depth_kernel(const ScanArgs s) {
   constexpr int V = Vec<T>::N;
   const int64_t state_elems = s.rows * s.d;
@@ -127,13 +129,15 @@ __global__ void __launch_bounds__(256) scan_depth_kernel(const ScanArgs s) {
   typedef typename Acc<T>::type A;
   A carry[V];
   ldv<T>(g + (int64_t)s.l_hi * state_elems + off).get(carry);
-  float old_next[V];  // shifted split: g_{l+1} of the previous iterate
+  float old_next[kShift ? V : 1];  // shifted split: g_{l+1} of the previous iterate
+  if (kShift) {
 #pragma unroll
-  for (int i = 0; i < V; ++i) old_next[i] = (float)carry[i];
+    for (int i = 0; i < V; ++i) old_next[i] = (float)carry[i];
+  }
   for (int l = s.l_hi - 1; l >= s.l_lo; --l) {
     A val[V];
     scan_step<T>(s, l, state_elems, off, ch, carry, val);
-    if (s.gamma != 0.0f) {
+    if (kShift) {
 #pragma unroll
       for (int i = 0; i < V; ++i) val[i] += s.gamma * old_next[i];
       ldv<T>(g + (int64_t)l * state_elems + off).get(old_next);  // before it is overwritten below
@@ -149,7 +153,7 @@ __global__ void __launch_bounds__(256) scan_depth_kernel(const ScanArgs s) {
 // ---- depth scan with the LayerNorm-backward finish from prepared row statistics ---------------------
 // Same streaming form as above: lnstat[l][row] = {rstd, mean(dy), mean(dy * xhat)} comes from the GEMM that
 // produced dy, so no reduction is needed here.  u holds dy, the VJP is rstd * (dy - m1 - xhat * m2).
-template <typename T>
+template <typename T, bool kShift>
 __global__ void __launch_bounds__(256) scan_depth_lnstat_kernel(const ScanArgs s) {
   constexpr int V = Vec<T>::N;
   const int64_t state_elems = s.rows * s.d;
@@ -160,10 +164,12 @@ __global__ void __launch_bounds__(256) scan_depth_lnstat_kernel(const ScanArgs s
   const int64_t row = off / s.d;
   const int ch = (int)(off - row * s.d);
   T* g = (T*)s.g;
-  float carry[V], old_next[V];
+  float carry[V], old_next[kShift ? V : 1];
   ldv<T>(g + (int64_t)s.l_hi * state_elems + off).get(carry);
+  if (kShift) {
 #pragma unroll
-  for (int i = 0; i < V; ++i) old_next[i] = carry[i];
+    for (int i = 0; i < V; ++i) old_next[i] = carry[i];
+  }
   for (int l = s.l_hi - 1; l >= s.l_lo; --l) {
     float dy[V], xh[V], val[V];
     ldv_stream<T>((const T*)s.u + (int64_t)l * state_elems + off).get(dy);
@@ -181,7 +187,7 @@ __global__ void __launch_bounds__(256) scan_depth_lnstat_kernel(const ScanArgs s
     }
 #pragma unroll
     for (int i = 0; i < V; ++i) val[i] += st.x * (dy[i] - st.y - xh[i] * st.z);
-    if (s.gamma != 0.0f) {
+    if (kShift) {
 #pragma unroll
       for (int i = 0; i < V; ++i) val[i] += s.gamma * old_next[i];
       ldv<T>(g + (int64_t)l * state_elems + off).get(old_next);
@@ -521,8 +527,14 @@ void scan_reverse(Launcher& lc, const ScanArgs& s) {
   const int64_t nvec = s.rows * s.d / V;
   if (s.xhat && s.lnstat) {
     const unsigned grid = (unsigned)((nvec + 255) / 256);
-    if (s.dtype == HBP_F32) scan_depth_lnstat_kernel<float><<<grid, 256, 0, lc.stream>>>(s);
-    else scan_depth_lnstat_kernel<bf16><<<grid, 256, 0, lc.stream>>>(s);
+    const bool shift = s.gamma != 0.0f;
+    if (s.dtype == HBP_F32) {
+      if (shift) scan_depth_lnstat_kernel<float, true><<<grid, 256, 0, lc.stream>>>(s);
+      else scan_depth_lnstat_kernel<float, false><<<grid, 256, 0, lc.stream>>>(s);
+    } else {
+      if (shift) scan_depth_lnstat_kernel<bf16, true><<<grid, 256, 0, lc.stream>>>(s);
+      else scan_depth_lnstat_kernel<bf16, false><<<grid, 256, 0, lc.stream>>>(s);
+    }
     lc.count();
     lc.check();
     return;
@@ -562,8 +574,14 @@ void scan_reverse(Launcher& lc, const ScanArgs& s) {
     return;
   }
   const unsigned grid = (unsigned)((nvec + 255) / 256);
-  if (s.dtype == HBP_F32) scan_depth_kernel<float><<<grid, 256, 0, lc.stream>>>(s);
-  else scan_depth_kernel<bf16><<<grid, 256, 0, lc.stream>>>(s);
+  const bool shift = s.gamma != 0.0f;
+  if (s.dtype == HBP_F32) {
+    if (shift) scan_depth_kernel<float, true><<<grid, 256, 0, lc.stream>>>(s);
+    else scan_depth_kernel<float, false><<<grid, 256, 0, lc.stream>>>(s);
+  } else {
+    if (shift) scan_depth_kernel<bf16, true><<<grid, 256, 0, lc.stream>>>(s);
+    else scan_depth_kernel<bf16, false><<<grid, 256, 0, lc.stream>>>(s);
+  }
   lc.count();
   lc.check();
 }
