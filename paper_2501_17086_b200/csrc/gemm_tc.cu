@@ -25,12 +25,24 @@ using namespace tc;
 
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int A_BYTES = BM * BK * 2;
+// Single CTA: a 128 x 256 tile, stages of {A 128 x 64, B 256 x 64}.  CTA pair (two CTAs of a cluster on one
+// 256 x 256 tile, tcgen05 cta_group::2): each CTA stages its own 128 rows of A and its own 128 of the 256
+// columns of B, so a stage is 32 KB instead of 48 KB for the same flops per SM, and six stages fit.
+template <bool kPair>
+struct Mode {
+  static constexpr int kStages = kPair ? 6 : 4;
+  static constexpr int kBRows = kPair ? 128 : 256;
+  static constexpr int kBBytes = kBRows * BK * 2;
+  static constexpr int kStageBytes = A_BYTES + kBBytes;
+  static constexpr int kTileM = kPair ? 256 : 128;
+};
+constexpr int RING_BYTES = 4 * (A_BYTES + 256 * BK * 2);  // = 6 stages of the pair mode
 constexpr int EPI_WARPS = 8, THREADS = 64 + 32 * EPI_WARPS;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int EPI_BUF_BYTES = 4096;  // 32 rows x 128 bytes per epilogue warp
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * EPI_BUF_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int SMEM_BYTES = RING_BYTES + EPI_WARPS * EPI_BUF_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 struct TcParams {
   int M, N, K, batch;
@@ -100,12 +112,21 @@ __device__ __forceinline__ void residual_chunk(const TcParams& p, int b, int row
 }
 
 // ------------------------------------------------------------------------------------------- kernel
+template <bool kPair>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
                const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
                const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmD2,
                const __grid_constant__ CUtensorMap tmE, const TcParams p) {
+  constexpr int STAGES = Mode<kPair>::kStages, STAGE_BYTES = Mode<kPair>::kStageBytes;
+  constexpr int B_ROWS = Mode<kPair>::kBRows, TILE_M = Mode<kPair>::kTileM;
+  // pair mode: rank of this CTA in its pair; the even CTA (leader) owns the pipeline's full barriers and
+  // issues the MMAs, its peer's tile loads signal the leader's barriers
+  const uint32_t rank = kPair ? cluster_ctarank() : 0u;
+  const bool leader = rank == 0;
+  const int first_tile = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int tile_step = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   extern __shared__ uint8_t smem_raw[];
   // the swizzled tiles need 1024-byte alignment
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -132,7 +153,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(accf_bar(a), 1);
-      mbar_init(acce_bar(a), EPI_WARPS);
+      mbar_init(acce_bar(a), kPair ? 2 * EPI_WARPS : EPI_WARPS);  // pair: both CTAs' epilogue warps arrive at the leader
     }
     mbar_init(drain_bar, 1);
     for (int w = 0; w < EPI_WARPS; ++w) mbar_init(epi_bar(w), 1);
@@ -141,13 +162,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (kPair) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync();  // the peer's barriers and tensor memory exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int tiles_per_batch = p.m_tiles * p.n_tiles;
@@ -162,10 +191,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0;
       uint32_t issued_mask = 0, issued_parity = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+      for (int tile = first_tile; tile < p.num_tiles && ok; tile += tile_step) {
         const int zc = tile / tiles_per_batch, r = tile % tiles_per_batch;
         const int b = zc % p.batch, split = zc / p.batch;
-        const int m0 = (r / p.n_tiles) * BM, n0 = (r % p.n_tiles) * BN;  // n fastest: a wave shares few A row-panels
+        // n fastest: a wave shares few A row-panels.  This CTA's rows of A and (pair) its half of B's columns
+        const int m0 = (r / p.n_tiles) * TILE_M + (int)rank * BM, n0 = (r % p.n_tiles) * BN + (int)rank * (BN - B_ROWS);
         const int kb_lo = split * p.kb_per_split, kb_hi = min(p.k_blocks, kb_lo + p.kb_per_split);
         for (int seg = 0; seg < p.segs && ok; ++seg) {
           const CUtensorMap* mA = seg == 0 ? &tmA : (seg == 1 ? &tmA1 : &tmA2);
@@ -173,26 +203,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int kb = kb_lo; kb < kb_hi; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
             const uint32_t sA = base + stage * STAGE_BYTES, sB = sA + A_BYTES;
-            const uint32_t fb = full_bar(stage);
-            mbar_expect_tx(fb, STAGE_BYTES);
+            // pair: all four tile loads of a stage (two per CTA) complete on the leader's barrier
+            const uint32_t fb = kPair ? map_to_cta(full_bar(stage), 0) : full_bar(stage);
+            if (leader) mbar_expect_tx(full_bar(stage), kPair ? 2 * STAGE_BYTES : STAGE_BYTES);
             issued_mask |= 1u << stage;
             issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
             const int k0 = kb * row_elems;
+            auto load = [&](uint32_t dst, const CUtensorMap* tm, int c0, int c1) {
+              if (kPair) tma_load_3d_pair(dst, tm, fb, c0, c1, b);
+              else tma_load_3d(dst, tm, fb, c0, c1, b);
+            };
             if (p.a_mn) {
-              for (int i = 0; i < BM / row_elems; ++i) tma_load_3d(sA + i * mn_block, mA, fb, m0 + row_elems * i, k0, b);
+              for (int i = 0; i < BM / row_elems; ++i) load(sA + i * mn_block, mA, m0 + row_elems * i, k0);
             } else {
-              tma_load_3d(sA, mA, fb, k0, m0, b);
+              load(sA, mA, k0, m0);
             }
             if (p.b_mn) {
-              for (int i = 0; i < BN / row_elems; ++i) tma_load_3d(sB + i * mn_block, mB, fb, n0 + row_elems * i, k0, b);
+              for (int i = 0; i < B_ROWS / row_elems; ++i) load(sB + i * mn_block, mB, n0 + row_elems * i, k0);
             } else {
-              tma_load_3d(sB, mB, fb, k0, n0, b);
+              load(sB, mB, k0, n0);
             }
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
           }
         }
       }
-      if (!ok) {
+      if (!ok && leader) {
         // leave no copy of ours in flight: wait (bounded) for every stage armed last
         for (int s = 0; s < STAGES; ++s)
           if (issued_mask & (1u << s)) {
@@ -204,17 +239,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && leader) {
       const uint32_t fmt = p.tf32 ? 2u : 1u;  // operand format: tf32 or bf16
       const uint32_t idesc = (1u << 4) /*fp32 accumulate*/ | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn << 15) |
-                             ((uint32_t)p.b_mn << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                             ((uint32_t)p.b_mn << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
       // one instruction consumes 32 bytes of K: 32 bytes along a K-major row, or 16 rows of an MN-major bf16 block
       const uint32_t a_step = p.a_mn ? 2048u : 32u, b_step = p.b_mn ? 2048u : 32u;
       const uint32_t a_lead = p.a_mn ? mn_block : 16u, b_lead = p.b_mn ? mn_block : 16u;
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+      for (int tile = first_tile; tile < p.num_tiles && ok; tile += tile_step) {
         if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)acc * BN;
@@ -229,19 +264,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int k = 0; k < 4; ++k) {
             const uint64_t ad = make_desc(sA + k * a_step, a_lead, 1024u);
             const uint64_t bd = make_desc(sB + k * b_step, b_lead, 1024u);
-            if (p.tf32) tc_mma_tf32(tmem_d, ad, bd, idesc, (first && k == 0) ? 0u : 1u);
-            else tc_mma(tmem_d, ad, bd, idesc, (first && k == 0) ? 0u : 1u);
+            const uint32_t accum = (first && k == 0) ? 0u : 1u;
+            if (kPair) {
+              if (p.tf32) tc_mma_tf32_pair(tmem_d, ad, bd, idesc, accum);
+              else tc_mma_pair(tmem_d, ad, bd, idesc, accum);
+            } else {
+              if (p.tf32) tc_mma_tf32(tmem_d, ad, bd, idesc, accum);
+              else tc_mma(tmem_d, ad, bd, idesc, accum);
+            }
           }
           first = 0;
-          tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if (kPair) tc_commit_pair(empty_bar(stage));
+          else tc_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        tc_commit(accf_bar(acc));  // accumulator complete
+        if (kPair) tc_commit_pair(accf_bar(acc));  // accumulator complete (each CTA holds its 128 rows of it)
+        else tc_commit(accf_bar(acc));
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
       if (!ok) {  // let issued MMAs finish before the tensor memory is freed
-        tc_commit(drain_bar);
+        if (kPair) tc_commit_pair(drain_bar);
+        else tc_commit(drain_bar);
         uint64_t t0 = global_ns();
         while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < 100000000ull) {
         }
@@ -260,10 +305,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool has_e = p.epi == EPI_MUL || p.epi == EPI_STORE_LN || p.epi == EPI_ADD;
     const int cw = p.d_f32 ? 32 : 64;      // accumulator columns per staged chunk (128 bytes of output per row)
     const int nchunks = 128 / cw;
-    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+    const uint32_t acce_target[2] = {kPair ? map_to_cta(acce_bar(0), 0) : acce_bar(0),
+                                     kPair ? map_to_cta(acce_bar(1), 0) : acce_bar(1)};
+    auto release_acc = [&](int a) {
+      if (kPair) mbar_arrive_cluster(acce_target[a]);
+      else mbar_arrive(acce_bar(a));
+    };
+    for (int tile = first_tile; tile < p.num_tiles; tile += tile_step) {
       // b indexes the outputs: with split-K it is split * batch + batch entry (partial sums [split][batch][M][N])
       const int b = tile / tiles_per_batch, r = tile % tiles_per_batch;
-      const int m0 = (r / p.n_tiles) * BM, n0 = (r % p.n_tiles) * BN;  // n fastest: a wave shares few A row-panels
+      const int m0 = (r / p.n_tiles) * TILE_M + (int)rank * BM, n0 = (r % p.n_tiles) * BN;  // this CTA's 128 rows
       const int row0 = m0 + quarter * 32, colw = n0 + half * 128;
       if (has_e && lane == 0) {  // the buffer is free here: fetch the first chunk of E while the MMAs still run
         mbar_expect_tx(ebar, EPI_BUF_BYTES);
@@ -282,7 +333,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(acce_bar(acc));
+        if (lane == 0) release_acc(acc);
       } else {
         bool ok = true;
         float s1 = 0.0f, s2 = 0.0f;  // EPI_STORE_LN: row sums of acc and acc * E over the current 64 columns
@@ -294,7 +345,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (c == nchunks - 1) {  // last read of this accumulator: hand it back to the MMA warp
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acce_bar(acc));
+            if (lane == 0) release_acc(acc);
           }
           const int col = colw + c * cw;
           if (has_e) {
@@ -391,9 +442,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   tc_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync();  // neither CTA leaves (or frees) while its peer may still read its tiles or signal its barriers
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if (kPair) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
@@ -519,15 +572,21 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   if (g.epi == EPI_MUL && !g.E) return false;
   if (g.epi == EPI_RESID && !g.R && !g.E) return false;
 
+  // CTA pairs only on request and when there are at least two 128-row blocks: measured on the MLP shapes the
+  // pair mode halves the MMA thread's waits for operands but its MMAs run slower (about 200 cycles against
+  // about 175 per 128 x 256 x 16 of work per SM), which nets out even
+  const int sms = sm_count();
+  const bool pair = g_gemm_pair && sms >= 2 && g.M > BM;
+  const int b_rows = pair ? Mode<true>::kBRows : Mode<false>::kBRows;
   CUtensorMap tmA, tmB;
   if (!make_map(&tmA, A0, g.M, g.K, g.batch, a_sm, a_sk, g.a_sb, a_mn, BM, f32)) return false;
-  if (!make_map(&tmB, B0, g.N, g.K, g.batch, b_sn, b_sk, g.b_sb, b_mn, BN, f32)) return false;
+  if (!make_map(&tmB, B0, g.N, g.K, g.batch, b_sn, b_sk, g.b_sb, b_mn, b_rows, f32)) return false;
   // float: segments A_hi B_lo, A_lo B_hi, A_hi B_hi - the small terms first, so that only the last segment adds
   // to an accumulator of full magnitude (the tensor core's fp32 accumulation does not round to nearest)
   CUtensorMap tmA1 = tmA, tmB1 = tmB, tmA2 = tmA, tmB2 = tmB;
   if (f32) {
     CUtensorMap a_lo, b_lo;
-    if (!make_map(&b_lo, g.B_lo, g.N, g.K, g.batch, b_sn, b_sk, g.b_sb, b_mn, BN, true)) return false;
+    if (!make_map(&b_lo, g.B_lo, g.N, g.K, g.batch, b_sn, b_sk, g.b_sb, b_mn, b_rows, true)) return false;
     if (!make_map(&a_lo, g.A_lo, g.M, g.K, g.batch, a_sm, a_sk, g.a_sb, a_mn, BM, true)) return false;
     tmA2 = tmA; tmB2 = tmB;      // segment 2: hi x hi
     tmA1 = a_lo; tmB1 = tmB;     // segment 1: lo x hi
@@ -554,7 +613,8 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
 
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+    if (cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return false;
     }
@@ -562,7 +622,7 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   }
   TcParams p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.batch = g.batch;
-  p.m_tiles = (g.M + BM - 1) / BM;
+  p.m_tiles = pair ? (g.M + 255) / 256 : (g.M + BM - 1) / BM;
   p.n_tiles = (g.N + BN - 1) / BN;
   p.num_tiles = p.m_tiles * p.n_tiles * g.batch * splits;
   p.k_blocks = k_blocks;
@@ -577,8 +637,26 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   p.R = g.R;
   p.stats = g.stats; p.stats_sb = g.stats_sb;
   p.status = status_word;
-  const int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
-  gemm_tc_kernel<<<grid, THREADS, SMEM_BYTES, lc.stream>>>(tmA, tmB, tmA1, tmB1, tmA2, tmB2, tmD, tmD2, tmE, p);
+  if (pair) {
+    const int pairs = p.num_tiles < sms / 2 ? p.num_tiles : sms / 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = lc.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<true>, tmA, tmB, tmA1, tmB1, tmA2, tmB2, tmD, tmD2, tmE, p);
+    if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
+  } else {
+    const int grid = p.num_tiles < sms ? p.num_tiles : sms;
+    gemm_tc_kernel<false><<<grid, THREADS, SMEM_BYTES, lc.stream>>>(tmA, tmB, tmA1, tmB1, tmA2, tmB2, tmD, tmD2, tmE, p);
+  }
   lc.count();
   lc.check();
   if (splits > 1) reduce_splitk(lc, g.partial, (float*)g.D, splits, (int64_t)g.batch * g.M * g.N);

@@ -10,6 +10,7 @@
 
 namespace hbp {
 bool g_force_simt = false;
+bool g_gemm_pair = false;
 
 bool gemm(Launcher& lc, const GemmArgs& g, int* status_word) {
   if (!g_force_simt && gemm_tc(lc, g, status_word)) return true;
@@ -611,6 +612,8 @@ hbp_status hbp_create(const hbp_config* cfg, void* workspace, size_t workspace_b
   c->ws_bytes = workspace_bytes;
   const char* env = std::getenv("HBP_FORCE_SIMT");
   g_force_simt = env && env[0] == '1';
+  const char* pm = std::getenv("HBP_GEMM_PAIR");
+  g_gemm_pair = pm && pm[0] == '1';
   if (cudaMemset(c->status, 0, 256) != cudaSuccess) {
     delete c;
     return HBP_ERR_CUDA;

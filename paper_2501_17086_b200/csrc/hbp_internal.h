@@ -84,6 +84,9 @@ int gemm_tc_stats_slots(int N);
 // Set from the environment variable HBP_FORCE_SIMT=1 when a context is created: keeps every GEMM
 // on the CUDA-core kernel (used to cross-check the tensor-core kernel).
 extern bool g_force_simt;
+// Set from the environment variable HBP_GEMM_PAIR=1 when a context is created: the tensor-core GEMM then pairs
+// CTAs (cta_group::2, 256 x 256 tiles) wherever the problem has two row blocks; otherwise single CTAs.
+extern bool g_gemm_pair;
 
 // ---------------------------------------------------------------- scans and elementwise (scan.cu)
 // Internal gate kind beside the public hbp_gate values: a[L][rows][d], one gate per element and step (the

@@ -188,3 +188,21 @@ def test_cuda_core_fallback_matches_oracle(name, ks, monkeypatch):
     kmax = max(ks)
     ref = orun.run(w, inp, ks=ks, grads_for=("exact", kmax))
     compare(w, gpu, ref, ks, ("exact", kmax))
+
+
+@pytest.mark.parametrize("mode", ["0", "1"])
+@pytest.mark.parametrize("name,ks", [("c2_twin", (2,)), ("c5_twin", (3,)), ("c4_twin", (2,)), ("c3_twin", (2,)), ("gru_twin", (2,))])
+def test_gemm_single_cta_and_cta_pair_modes_match_oracle(name, ks, mode, monkeypatch):
+    """HBP_GEMM_PAIR (read when a context is made): 0 keeps the tensor-core GEMM on single CTAs (128 x 256 tiles),
+    1 pairs CTAs (256 x 256 tiles) wherever two row blocks exist; both must meet the bar on every twin."""
+    from oracle import run as orun
+    from paper_2501_17086_b200.workloads import WORKLOADS, make_inputs
+    from test_gpu_parity import compare, run_gpu
+    monkeypatch.setenv("HBP_GEMM_PAIR", mode)
+    w = WORKLOADS[name]
+    inp = make_inputs(w, "cuda")
+    gpu = run_gpu(w, inp, ks)
+    del gpu["ctx"]
+    kmax = max(ks)
+    ref = orun.run(w, inp, ks=ks, grads_for=("exact", kmax))
+    compare(w, gpu, ref, ks, ("exact", kmax))
