@@ -268,7 +268,10 @@ void launch_bwd(Launcher& lc, const AttnArgs& a) {
     else fn<bf16, 128>(lc, a);                                                     \
   }
 
-void attention_fwd(Launcher& lc, const AttnArgs& a) { HBP_ATTN_DISPATCH(launch_fwd) }
+void attention_fwd(Launcher& lc, const AttnArgs& a) {
+  if (!g_force_simt && attention_fwd_tc(lc, a, a.status)) return;  // bf16, head dimension 64: tensor cores
+  HBP_ATTN_DISPATCH(launch_fwd)
+}
 void attention_bwd(Launcher& lc, const AttnArgs& a) { HBP_ATTN_DISPATCH(launch_bwd) }
 
 }  // namespace hbp

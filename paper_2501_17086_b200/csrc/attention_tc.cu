@@ -313,6 +313,224 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
   }
 }
 
+// ------------------------------------------------------------------------------------------- forward
+// Causal attention forward, one CTA per 128 queries (bf16, head dimension 64), in two sweeps over the key blocks
+// so that the output accumulator in tensor memory never has to be rescaled:
+//   sweep 1:  S = Q K^T per 64-key block; every softmax thread keeps the running maximum and sum of exponentials of
+//             its row over its 32 columns; the two halves of a row are merged into the row's log-sum-exp;
+//   sweep 2:  S again, P = exp(S/sqrt(dh) - lse) (already normalised), O += P V.
+// Same roles, barriers and pipelining as the backward kernels: the score MMAs of the next block run under the
+// exponentials of the current one.  Barrier slots: 1-2 full[2], 3-4 empty[2], 5 scores ready, 6 probabilities
+// ready, 7 all MMAs done, 8 scores copied out, 0 the Q tile.
+constexpr uint32_t FWD_TMEM_COLS = 128;  // scores [0,64), output accumulator [64,128)
+constexpr int FWD_SMEM_BYTES = BIG_BYTES + 4 * SMALL_BYTES + PS_BYTES + 2048 /*row statistics*/ + 256 /*barriers*/ + 1024;
+
+__global__ void __launch_bounds__(THREADS, 3)
+attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO, float* lse_out,
+                   const AttnTcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t sQ = base;
+  const uint32_t sSmall = base + BIG_BYTES;       // [buf][K tile, V tile]
+  const uint32_t sP = sSmall + 4 * SMALL_BYTES;   // P as bf16, later the output staging
+  constexpr int VEC_OFF = BIG_BYTES + 4 * SMALL_BYTES + PS_BYTES;
+  float* vec = reinterpret_cast<float*>(aligned + VEC_OFF);  // [2 halves][128 rows] of {max, sum}
+  uint64_t* bar_mem = reinterpret_cast<uint64_t*>(aligned + VEC_OFF + 2048);
+  const uint32_t bars = smem_u32(bar_mem);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 10);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int blk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int q0 = blk * BIG;
+  const int n_kb = min((p.S + SMALL - 1) / SMALL, (min(p.S, q0 + BIG) + SMALL - 1) / SMALL);  // key blocks up to the diagonal
+  const int n_it = 2 * n_kb;  // sweep 1 then sweep 2
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 9; ++i) mbar_init(bar_at(bars, i), (i == 6 || i == 8) ? SOFTMAX_WARPS : 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(FWD_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tS = tmem, tO = tmem + 64;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(bar_at(bars, 0), BIG_BYTES);
+      tma_load_4d(sQ, &tmQ, bar_at(bars, 0), 0, q0, h, b);
+      bool ok = true;
+      int last_buf_parity[2] = {-1, -1};
+      for (int it = 0; it < n_it && ok; ++it) {
+        const int buf = it & 1;
+        const uint32_t ph = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(bar_at(bars, 3 + buf), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        const bool second = it >= n_kb;
+        const int r0 = (second ? it - n_kb : it) * SMALL;
+        mbar_expect_tx(bar_at(bars, 1 + buf), second ? 2 * SMALL_BYTES : SMALL_BYTES);
+        last_buf_parity[buf] = (int)ph;
+        tma_load_4d(sSmall + (2 * buf) * SMALL_BYTES, &tmK, bar_at(bars, 1 + buf), 0, r0, h, b);
+        if (second) tma_load_4d(sSmall + (2 * buf + 1) * SMALL_BYTES, &tmV, bar_at(bars, 1 + buf), 0, r0, h, b);
+      }
+      if (!ok) {  // leave no copy of ours in flight
+        for (int buf = 0; buf < 2; ++buf)
+          if (last_buf_parity[buf] >= 0) {
+            const uint64_t t0 = global_ns();
+            while (!mbar_try_wait(bar_at(bars, 1 + buf), (uint32_t)last_buf_parity[buf]) &&
+                   global_ns() - t0 < 100000000ull) {
+            }
+          }
+        const uint64_t t0 = global_ns();
+        while (!mbar_try_wait(bar_at(bars, 0), 0) && global_ns() - t0 < 100000000ull) {
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      auto issue_scores = [&](int it) {
+        const uint32_t s0 = sSmall + (2 * (it & 1)) * SMALL_BYTES;
+#pragma unroll
+        for (int k = 0; k < DH / 16; ++k)
+          tc_mma(tS, make_desc(sQ + 32 * k, 16, 1024), make_desc(s0 + 32 * k, 16, 1024), IDESC_KK, k != 0);
+        tc_commit(bar_at(bars, 5));
+        if (it < n_kb) tc_commit(bar_at(bars, 3 + (it & 1)));  // sweep 1: the K tile is free once the scores are formed
+      };
+      bool ok = mbar_wait(bar_at(bars, 0), 0, abort_flag, p.status);
+      ok = ok && mbar_wait(bar_at(bars, 1), 0, abort_flag, p.status);
+      tc_fence_after();
+      if (ok) issue_scores(0);
+      for (int it = 0; it < n_it && ok; ++it) {
+        const int buf = it & 1;
+        if (it + 1 < n_it) {
+          const int nb = (it + 1) & 1;
+          if (!mbar_wait(bar_at(bars, 1 + nb), (uint32_t)((it + 1) >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+          if (!mbar_wait(bar_at(bars, 8), (uint32_t)it & 1u, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          issue_scores(it + 1);
+        }
+        if (it < n_kb) continue;
+        const int j = it - n_kb;
+        if (!mbar_wait(bar_at(bars, 6), (uint32_t)j & 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t s1 = sSmall + (2 * buf + 1) * SMALL_BYTES;
+#pragma unroll
+        for (int k = 0; k < SMALL / 16; ++k)  // O += P V: contraction over the 64 keys, V is an MN-major operand
+          tc_mma(tO, make_desc(sP + 32 * k, 16, 1024), make_desc(s1 + 2048 * k, 8192, 1024), IDESC_KMN,
+                 (j != 0 ? 1u : 0u) | (k != 0));
+        tc_commit(bar_at(bars, 3 + buf));
+      }
+      tc_commit(bar_at(bars, 7));
+      if (!ok) {
+        const uint64_t t0 = global_ns();
+        while (!mbar_try_wait(bar_at(bars, 7), 0) && global_ns() - t0 < 100000000ull) {
+        }
+      }
+    }
+  } else {
+    const int ch = (warp - 2) >> 2;        // which 32 of the block's 64 key columns this warp handles
+    const int quarter = warp & 3;          // TMEM lane quarter this warp may read
+    const int row = quarter * 32 + lane;   // query row of the tile
+    const int grow = q0 + row;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const float scale2 = p.scale * LOG2E;
+    float m_run = -INFINITY, l_run = 0.0f, lse2 = 0.0f;
+    bool ok = true;  // false after a wait gave up: keep pace with the named barriers, do no more work
+    for (int it = 0; it < n_it; ++it) {
+      const bool second = it >= n_kb;
+      const int j = second ? it - n_kb : it;
+      const int c0 = j * SMALL;
+      if (it == n_kb) {  // between the sweeps: merge the two halves of every row into its log-sum-exp
+        vec[ch * 256 + row] = m_run;
+        vec[ch * 256 + 128 + row] = l_run;
+        named_barrier_softmax();
+        const float m0 = vec[row], l0 = vec[128 + row], m1 = vec[256 + row], l1 = vec[256 + 128 + row];
+        const float mm = fmaxf(m0, m1);  // finite: key 0 is visible to every query
+        const float ll = l0 * fast_exp2(m0 - mm) + l1 * fast_exp2(m1 - mm);
+        lse2 = mm + __log2f(ll);
+        if (ch == 0 && grow < p.S && ok) lse_out[((int64_t)b * p.H + h) * p.S + grow] = lse2 * (1.0f / LOG2E);
+      }
+      if (!ok) continue;
+      if (!mbar_wait(bar_at(bars, 5), (uint32_t)it & 1u, abort_flag, p.status)) { ok = false; continue; }
+      tc_fence_after();
+      float sc[32];
+      tc_ld32(tS + lane_addr + ch * 32, sc);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_at(bars, 8));
+      const bool full = (c0 + SMALL - 1 <= q0) && (c0 + SMALL <= p.S);  // no element of the block is masked
+      if (!second) {
+        float bm = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const int col = c0 + ch * 32 + c;
+          const bool vis = full || ((col <= grow) && (col < p.S));
+          sc[c] = vis ? sc[c] * scale2 : -INFINITY;
+          bm = fmaxf(bm, sc[c]);
+        }
+        if (bm > -INFINITY) {
+          const float mn = fmaxf(m_run, bm);
+          float sum = 0.0f;
+#pragma unroll
+          for (int c = 0; c < 32; ++c) sum += fast_exp2(sc[c] - mn);
+          l_run = l_run * fast_exp2(m_run - mn) + sum;
+          m_run = mn;
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const int col = c0 + ch * 32 + c;
+          const bool vis = full || ((col <= grow) && (col < p.S));
+          sc[c] = vis ? fast_exp2(fmaf(sc[c], scale2, -lse2)) : 0.0f;
+        }
+        // the accumulating MMAs of the previous block read the probability tile: wait until they are done
+        if (j > 0 && !mbar_wait(bar_at(bars, 3 + ((it - 1) & 1)), (uint32_t)((it - 1) >> 1) & 1u, abort_flag, p.status)) {
+          ok = false;
+          continue;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) st_shared16(swz(sP, row, ch * 4 + u), pack8(sc + 8 * u));
+        fence_async_smem();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_at(bars, 6));
+      }
+    }
+    // ---- epilogue: O -> bf16 -> shared -> TMA store
+    ok = ok && mbar_wait(bar_at(bars, 7), 0, abort_flag, p.status);
+    if (ok) {
+      tc_fence_after();
+      float v[32];
+      tc_ld32(tO + lane_addr + ch * 32, v);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) st_shared16(swz(sP, row, ch * 4 + u), pack8(v + 8 * u));
+      fence_async_smem();
+    }
+    named_barrier_softmax();
+    if (threadIdx.x == 64 && ok) {
+      tma_store_4d(&tmO, sP, 0, q0, h, b);
+      tma_store_wait_all();
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(FWD_TMEM_COLS) : "memory");
+  }
+}
+
 constexpr int SMEM_BYTES = 2 * BIG_BYTES + 4 * SMALL_BYTES + 2 * PS_BYTES + 1024 /*vectors*/ + 256 /*barriers*/ + 1024;
 
 // 4-D map {dh, sequence, head, batch} of one [tokens][ld] tensor's column block starting at `base`.
@@ -374,6 +592,39 @@ bool attention_bwd_tc(Launcher& lc, const AttnArgs& a, int* status_word) {
   // dQ: big tiles Q, dO; small tiles K, V
   attn_bwd_tc_kernel<false><<<grid, THREADS, SMEM_BYTES, lc.stream>>>(qB, oB, kS, vS, dq, dq, p);
   lc.count(2);
+  lc.check();
+  return true;
+}
+
+// Causal attention forward (O and the log-sum-exp) on the tensor cores; false (nothing launched) when the problem
+// does not fit this kernel.
+bool attention_fwd_tc(Launcher& lc, const AttnArgs& a, int* status_word) {
+  if (a.dtype != HBP_BF16 || a.head_dim != DH || !status_word) return false;
+  const int d = a.heads * DH;
+  const int64_t ld3 = 3 * (int64_t)d;
+  if (((uintptr_t)a.qkv | (uintptr_t)a.o) & 15u) return false;
+  if (d % 8) return false;
+  const bf16* qkv = (const bf16*)a.qkv;
+  CUtensorMap q, k, v, o;
+  if (!(make_map4(&q, qkv, a.seq, a.heads, a.batch, ld3, BIG) && make_map4(&k, qkv + d, a.seq, a.heads, a.batch, ld3, SMALL) &&
+        make_map4(&v, qkv + 2 * d, a.seq, a.heads, a.batch, ld3, SMALL) && make_map4(&o, a.o, a.seq, a.heads, a.batch, d, BIG)))
+    return false;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM_BYTES) != cudaSuccess) {
+      cudaGetLastError();
+      return false;
+    }
+    attr_set = true;
+  }
+  AttnTcParams p;
+  p.S = a.seq; p.H = a.heads; p.B = a.batch;
+  p.lse = nullptr; p.drow = nullptr; p.d_sb = p.d_sh = p.d_sq = 0;
+  p.scale = 1.0f / sqrtf((float)DH);
+  p.status = status_word;
+  dim3 grid((a.seq + BIG - 1) / BIG, a.heads, a.batch);
+  attn_fwd_tc_kernel<<<grid, THREADS, FWD_SMEM_BYTES, lc.stream>>>(q, k, v, o, a.lse, p);
+  lc.count();
   lc.check();
   return true;
 }

@@ -755,6 +755,7 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
         t.qkv = r.at(ctx->QKV, (int64_t)b * 3 * state);
         t.o = r.at(ctx->O, (int64_t)b * state);
         t.lse = ctx->lse + (int64_t)b * f.batch * f.n_heads * f.seq;
+        t.status = ctx->status;
         attention_fwd(r.lc, t);
         GemmArgs o = r.base_args();
         o.M = (int)N; o.N = (int)d; o.K = (int)d;

@@ -186,6 +186,8 @@ void attention_fwd(Launcher& lc, const AttnArgs& a);
 void attention_bwd(Launcher& lc, const AttnArgs& a);
 // Tensor-core dQ/dK/dV (attention_tc.cu); false if the problem does not qualify (nothing launched).
 bool attention_bwd_tc(Launcher& lc, const AttnArgs& a, int* status_word);
+// Tensor-core forward (attention_tc.cu), same conditions.
+bool attention_fwd_tc(Launcher& lc, const AttnArgs& a, int* status_word);
 
 // ---------------------------------------------------------------- device math
 __device__ __forceinline__ float gelu_f(float z) { return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f)); }
