@@ -82,3 +82,64 @@ def test_full_size_sampled_units(name, ks, rows):
     kmax = max(ks)
     for l in range(w.steps - kmax, w.steps + 1):
         assert rel(got[kmax][l], got["exact"][l]) < tol_exact
+
+
+def _run_shard(w_shard, inp, rows, delta_rows):
+    """hbp_backward(k=2) with parameter gradients on the token shard `rows` of a workload (full weights)."""
+    from paper_2501_17086_b200 import harness
+    ctx = harness.make_context(w_shard)
+    params = harness.params_for(w_shard, inp)
+    x_all = ctx.forward(params, inp["x0"][rows].contiguous(), None)
+    grads = ctx.new_grads()
+    ctx.backward(params, 2, delta_rows, x_all, None, grads=grads)
+    ctx.sync_status()
+    return x_all, grads
+
+
+def test_full_size_parameter_gradients_by_shard_additivity():
+    """Parameter gradients are sums over tokens: on c2 the gradients of the whole batch must equal the sum of the
+    gradients of its two halves (each run as its own problem with the same delta rows), and a small shard must
+    match the oracle run on those tokens with the full weights."""
+    import dataclasses
+    from paper_2501_17086_b200 import harness
+    w = WORKLOADS["c2"]
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * 2**30:
+        pytest.skip("needs about 40 GB of free device memory")
+    inp = make_inputs(w, "cuda")
+    ctx = harness.make_context(w)
+    params = harness.params_for(w, inp)
+    x_all = ctx.forward(params, inp["x0"], None)
+    delta = harness.loss_delta(w, x_all, inp)          # [N, d], normalised by the full problem size
+    whole = ctx.new_grads()
+    ctx.backward(params, 2, delta, x_all, None, grads=whole)
+    ctx.sync_status()
+    del ctx, x_all
+    torch.cuda.empty_cache()
+
+    half = w.tokens // 2
+    w_half = dataclasses.replace(w, tokens=half, batch=w.batch // 2)
+    total = None
+    for lo in (0, half):
+        rows = torch.arange(lo, lo + half, device="cuda")
+        _, g = _run_shard(w_half, inp, rows, delta[rows].contiguous())
+        total = g if total is None else {n: total[n] + g[n] for n in g}
+        torch.cuda.empty_cache()
+    for n in whole:
+        err = float((whole[n].double() - total[n].double()).norm() / total[n].double().norm())
+        assert err < 2e-3, f"{n}: whole vs sum of halves {err:.3e}"   # same bf16 products, other summation order
+
+    # a 48-token shard against the oracle (tokens are independent, so its delta rows are the whole problem's)
+    rows = torch.tensor([0, 1, 2, 3, 130, 131, 4099, 8191] + list(range(1000, 1040)), device="cuda")
+    w_small = dataclasses.replace(w, tokens=int(rows.numel()), batch=1, seq=int(rows.numel()))
+    x_small, g_small = _run_shard(w_small, inp, rows, delta[rows].contiguous())
+    stack, x0, groups = orun.build_stack(w, inp, rows.cpu())
+    from oracle import hbp_oracle as O
+    xs, caches = O.forward(stack, x0)
+    deltas = orun.loss_deltas(w, xs, inp, rows.cpu())
+    gk = O.highway_bp(stack, caches, deltas, 2)
+    ref = O.param_grads(stack, caches, xs, gk, groups)
+    for n, v in ref.items():
+        got = g_small["d" + n].double().cpu().numpy()
+        err = float(np.linalg.norm(got - v) / np.linalg.norm(v))
+        assert err < TOL[w.dtype], f"{n}: shard vs oracle {err:.3e}"
