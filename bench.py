@@ -210,7 +210,7 @@ class ClockSampler:
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2501_17086_b200 import harness
+    from paper_2501_17086_b200 import binding, harness
     from paper_2501_17086_b200.workloads import WORKLOADS, make_inputs
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -359,6 +359,20 @@ def run_ours(args):
         fn = lambda: ctx.exact(params, delta, x_all, xin, g_all=g_all, grads=grads)
         fn()
         detail["exact_bp_ms"] = timed_local(torch, fn, 3)
+        # Figure 5's quantity on this synthetic workload: cosine similarity of the k-iteration estimate with the
+        # exact gradient, per state, computed on the device (hbp_compare); minimum and median over the states
+        try:
+            g_exact = g_all.clone()
+            cos = {}
+            for kx in (1, 2, 4, 8):
+                ctx.backward(params, kx, delta, x_all, xin, g_all=g_all, grads=None)
+                s4 = binding.compare(g_all[:-1], g_exact[:-1], segments=w.steps)
+                c = s4[:, 0] / torch.sqrt(s4[:, 1] * s4[:, 2]).clamp_min(1e-300)
+                cos[f"k{kx}"] = {"min": float(c.min()), "median": float(c.median()), "last_quarter_min": float(c[3 * w.steps // 4:].min())}
+            detail["cosine_vs_exact"] = cos
+            del g_exact
+        except torch.OutOfMemoryError:
+            detail["cosine_vs_exact"] = None
         line["detail"] = detail
         if world == 1:
             sample = {"c2": 16, "c5": 4, "c4": 1, "c3": 2}.get(w.name, 8)

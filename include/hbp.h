@@ -173,6 +173,16 @@ size_t hbp_cumsumprod_static_max_bytes(void);
 hbp_status hbp_cumsumprod_static(int32_t dtype, int32_t gate, int32_t loss, int32_t L, int64_t rows, int32_t d,
                                  const void* u, const void* delta, const void* a, void* g, void* cuda_stream);
 
+/* Agreement of two gradient estimates, the quantities behind Figure 5 (cosine similarity of the k-iteration estimate
+ * with the true gradient; norm of an iteration's step relative to the total): a and b hold `segments` consecutive
+ * blocks of `elems` elements of `dtype` (states g_l, or float parameter gradients); out [segments][4] doubles (device)
+ * receives <a,b>, |a|^2, |b|^2, |a-b|^2 per segment, summed in double in a fixed order.  scratch: device memory of
+ * hbp_compare_scratch_bytes(segments) bytes, 8-byte aligned.  cos = out[0] / sqrt(out[1] out[2]); relative step =
+ * sqrt(out[3] / out[2]). */
+size_t hbp_compare_scratch_bytes(int32_t segments);
+hbp_status hbp_compare(int32_t dtype, int32_t segments, int64_t elems, const void* a, const void* b, double* out,
+                       void* scratch, size_t scratch_bytes, void* cuda_stream);
+
 /* Copies the context's device status word to the host after synchronising the stream: HBP_OK, or the
  * error a kernel recorded (HBP_ERR_TIMEOUT when a bounded wait gave up).  The only synchronising call. */
 hbp_status hbp_sync_status(hbp_ctx* ctx, void* cuda_stream);

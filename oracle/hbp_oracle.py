@@ -515,3 +515,11 @@ def path_sum(deltas, J, K, i, k):
                     vec = vec @ (J[m] if m in chosen else K[m])
                 total = total + vec
     return total
+
+
+def agreement(a, b):
+    """The four sums behind Figure 5 for two gradient estimates: <a,b>, |a|^2, |b|^2, |a-b|^2 (cosine similarity =
+    first / sqrt(second * third); relative size of a step = sqrt(fourth / third))."""
+    a, b = _f64(a).reshape(-1), _f64(b).reshape(-1)
+    d = a - b
+    return np.array([a @ b, a @ a, b @ b, d @ d])

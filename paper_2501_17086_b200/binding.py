@@ -22,7 +22,7 @@ LOSS_FINAL, LOSS_EVERY_STEP = 0, 1
 EXPORTS = ["hbp_workspace_bytes", "hbp_create", "hbp_forward", "hbp_backward", "hbp_exact",
            "hbp_cumsumprod_scratch_bytes", "hbp_cumsumprod", "hbp_sync_status", "hbp_launch_count",
            "hbp_profile_enable", "hbp_profile_read", "hbp_cumsumprod_static", "hbp_cumsumprod_static_max_bytes",
-           "hbp_status_string", "hbp_destroy"]
+           "hbp_compare_scratch_bytes", "hbp_compare", "hbp_status_string", "hbp_destroy"]
 
 
 class HbpError(RuntimeError):
@@ -61,6 +61,8 @@ def _load():
     lib.hbp_cumsumprod.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.hbp_cumsumprod_static.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp]
     lib.hbp_cumsumprod_static_max_bytes.argtypes = []
+    lib.hbp_compare_scratch_bytes.argtypes = [i32]
+    lib.hbp_compare.argtypes = [i32, i32, i64, vp, vp, vp, vp, sz, vp]
     lib.hbp_sync_status.argtypes = [vp, vp]
     lib.hbp_profile_enable.argtypes = [vp, i32]
     lib.hbp_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(i64)]
@@ -71,8 +73,8 @@ def _load():
     lib.hbp_destroy.argtypes = [vp]
     lib.hbp_destroy.restype = None
     for name in EXPORTS:
-        if name == "hbp_cumsumprod_static_max_bytes":
-            lib.hbp_cumsumprod_static_max_bytes.restype = sz
+        if name in ("hbp_cumsumprod_static_max_bytes", "hbp_compare_scratch_bytes"):
+            getattr(lib, name).restype = sz
         elif name not in ("hbp_launch_count", "hbp_status_string", "hbp_destroy"):
             getattr(lib, name).restype = C.c_int
     return lib
@@ -274,3 +276,17 @@ def cumsumprod_static(u, delta, a=None, gate=None, loss=LOSS_FINAL, g=None):
     _check(lib.hbp_cumsumprod_static(_dtype_code(u.dtype), gate, loss, L, rows, d, _ptr(u), _ptr(delta), _ptr(a),
                                      _ptr(g), _stream()), "hbp_cumsumprod_static")
     return g
+
+
+def compare(a, b, segments=1):
+    """<a,b>, |a|^2, |b|^2, |a-b|^2 per segment of two equally shaped tensors split into ``segments`` consecutive
+    blocks (e.g. the states g_l of two estimates): a float64 tensor [segments, 4] on the device.  The cosine
+    similarity of Figure 5 is out[:, 0] / sqrt(out[:, 1] * out[:, 2])."""
+    assert a.shape == b.shape and a.dtype == b.dtype and a.is_contiguous() and b.is_contiguous()
+    assert a.numel() % segments == 0
+    out = torch.empty((segments, 4), dtype=torch.float64, device=a.device)
+    need = int(lib.hbp_compare_scratch_bytes(segments))
+    scratch = torch.empty(need, dtype=torch.uint8, device=a.device)
+    _check(lib.hbp_compare(_dtype_code(a.dtype), segments, a.numel() // segments, _ptr(a), _ptr(b), _ptr(out),
+                           _ptr(scratch), need, _stream()), "hbp_compare")
+    return out

@@ -906,6 +906,21 @@ hbp_status hbp_exact(hbp_ctx* ctx, const hbp_params* params, const void* delta, 
   return backward_common(ctx, params, 0, true, delta, x_all, inputs, g_all, grads, cuda_stream);
 }
 
+size_t hbp_compare_scratch_bytes(int32_t segments) { return segments > 0 ? compare_scratch_bytes(segments) : 0; }
+
+hbp_status hbp_compare(int32_t dtype, int32_t segments, int64_t elems, const void* a, const void* b, double* out,
+                       void* scratch, size_t scratch_bytes, void* cuda_stream) {
+  if (dtype != HBP_F32 && dtype != HBP_BF16) return HBP_ERR_DTYPE;
+  if (segments <= 0 || segments > 65535 || elems <= 0) return HBP_ERR_SHAPE;
+  if (!a || !b || !out || !scratch) return HBP_ERR_INVALID_ARG;
+  if (((uintptr_t)out | (uintptr_t)scratch) & 7u) return HBP_ERR_SHAPE;
+  if (scratch_bytes < compare_scratch_bytes(segments)) return HBP_ERR_WORKSPACE;
+  Launcher lc;
+  lc.stream = (cudaStream_t)cuda_stream;
+  compare_segments(lc, dtype, a, b, segments, elems, out, (double*)scratch);
+  return lc.err == cudaSuccess ? HBP_OK : HBP_ERR_CUDA;
+}
+
 hbp_status hbp_cumsumprod_scratch_bytes(int32_t dtype, int32_t L, int64_t rows, int32_t d, size_t* bytes) {
   if (!bytes) return HBP_ERR_INVALID_ARG;
   if (dtype != HBP_F32 && dtype != HBP_BF16) return HBP_ERR_DTYPE;

@@ -151,6 +151,13 @@ void rnn_backward_step(Launcher& lc, int dtype, const void* W, const void* deriv
                        const double* g_in, double* g_out, void* g_store, int B, int d);
 void convert_to_f64(Launcher& lc, int dtype, const void* src, double* dst, int64_t elems);
 
+// ---------------------------------------------------------------- diagnostics (diag.cu)
+// out[seg][4] = {<a,b>, |a|^2, |b|^2, |a-b|^2} over `elems` elements per segment; scratch holds
+// compare_scratch_bytes(segments) bytes.
+size_t compare_scratch_bytes(int segments);
+void compare_segments(Launcher& lc, int dtype, const void* a, const void* b, int segments, int64_t elems, double* out,
+                      double* scratch);
+
 // ---------------------------------------------------------------- GRU (gru.cu)
 // One forward step in double from the double master state; writes the new master, the stored state, the
 // gate z [B][d] and the VJP coefficients c4 [B][4d] = [c_r | c_z | c_nr | c_n].

@@ -206,3 +206,21 @@ def test_gemm_single_cta_and_cta_pair_modes_match_oracle(name, ks, mode, monkeyp
     kmax = max(ks)
     ref = orun.run(w, inp, ks=ks, grads_for=("exact", kmax))
     compare(w, gpu, ref, ks, ("exact", kmax))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_compare_matches_the_definition(dtype):
+    from paper_2501_17086_b200 import binding as B
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(77)
+    a = torch.randn((7, 33, 40), generator=gen, device="cuda").to(dtype)
+    b = (a.float() + 0.1 * torch.randn((7, 33, 40), generator=gen, device="cuda")).to(dtype)
+    got = B.compare(a, b, segments=7).cpu().numpy()
+    again = B.compare(a, b, segments=7).cpu().numpy()
+    assert (got == again).all()                       # fixed summation order
+    for l in range(7):
+        want = O.agreement(np64(a[l]), np64(b[l]))
+        np.testing.assert_allclose(got[l], want, rtol=1e-6)   # products of floats, accumulated in double
+    with pytest.raises(B.HbpError):
+        B.lib.hbp_compare.restype = C.c_int
+        B._check(B.lib.hbp_compare(0, 0, 10, None, None, None, None, 0, None), "hbp_compare")

@@ -555,3 +555,15 @@ def test_gru_path_sums_with_state_dependent_gate():
         np.testing.assert_allclose(a, b, rtol=1e-11, atol=1e-12)
     for a, b in zip(O.highway_bp_folded(st, caches, deltas, 2), O.highway_bp(st, caches, deltas, 2)):
         np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
+
+
+# ---------------------------------------------- 12. agreement sums (Figure 5)
+def test_agreement_sums_on_known_vectors():
+    a = np.array([3.0, 0.0, 4.0])
+    b = np.array([0.0, 2.0, 4.0])
+    s = O.agreement(a, b)
+    np.testing.assert_allclose(s, [16.0, 25.0, 20.0, 13.0])
+    # the polarisation identity ties the four together; identical inputs give cosine 1 and step 0
+    assert abs(s[3] - (s[1] + s[2] - 2 * s[0])) < 1e-12
+    t = O.agreement(a, a)
+    assert t[0] == t[1] == t[2] and t[3] == 0.0
