@@ -148,6 +148,24 @@ hbp_status hbp_backward(hbp_ctx* ctx, const hbp_params* params, int32_t k, const
 hbp_status hbp_exact(hbp_ctx* ctx, const hbp_params* params, const void* delta, const void* x_all,
                      const void* inputs, void* g_all, const hbp_grads* grads, void* cuda_stream);
 
+/* The pieces of hbp_backward on their own, for callers that run the iterations themselves - in particular for
+ * splitting the stack over several GPUs by layers (Section 6's layer-parallel setting: every GPU holds a contiguous
+ * range of layers as its own context and the scan's carry crosses GPUs between the calls).
+ *  hbp_iterate      one iteration in place (Eq. 8, then Eq. 9 and 11): u_l = J_l^T g_all[l+1] for every step from the
+ *                   iterate as given (g_all[steps] included: the owner of the following layers supplies it), then
+ *                   g_all[steps] = delta_L and g_all[l] = delta_l + a_l (.) g_all[l+1] + u_l.  g^0 followed by k calls
+ *                   with the loss gradient as delta is hbp_backward(k).  A GPU that does not hold the last layer passes
+ *                   zeros as delta: its scan then starts from a zero carry.
+ *  hbp_add_carry    g_all[l] += carry [N][d] for l = 0..steps: applies the true carry to a scan that was started from
+ *                   zero.  Only for gates that are all one (then every state depends on the carry with coefficient one);
+ *                   HBP_ERR_UNSUPPORTED otherwise.
+ *  hbp_param_grads  Section 4.2: the parameter gradients from the estimate in g_all. */
+hbp_status hbp_iterate(hbp_ctx* ctx, const hbp_params* params, const void* delta, const void* x_all, const void* inputs,
+                       void* g_all, void* cuda_stream);
+hbp_status hbp_add_carry(hbp_ctx* ctx, const void* carry, void* g_all, void* cuda_stream);
+hbp_status hbp_param_grads(hbp_ctx* ctx, const hbp_params* params, const void* x_all, const void* inputs,
+                           const void* g_all, const hbp_grads* grads, void* cuda_stream);
+
 /* Eq. 9 / Eq. 12 on its own: g[L] = delta_L and g[l] = delta_l + a_l (.) g[l+1] + u[l] for l = L-1..0,
  * i.e. the reverse CumSumProd with diagonal K.  u [L][rows][d] (NULL = zeros), delta as in hbp_loss
  * (`loss`), a as in hbp_gate (`gate`), g [L+1][rows][d].  `scratch` is device memory of at least

@@ -22,7 +22,8 @@ LOSS_FINAL, LOSS_EVERY_STEP = 0, 1
 EXPORTS = ["hbp_workspace_bytes", "hbp_create", "hbp_forward", "hbp_backward", "hbp_exact",
            "hbp_cumsumprod_scratch_bytes", "hbp_cumsumprod", "hbp_sync_status", "hbp_launch_count",
            "hbp_profile_enable", "hbp_profile_read", "hbp_cumsumprod_static", "hbp_cumsumprod_static_max_bytes",
-           "hbp_compare_scratch_bytes", "hbp_compare", "hbp_status_string", "hbp_destroy"]
+           "hbp_compare_scratch_bytes", "hbp_compare", "hbp_iterate", "hbp_add_carry", "hbp_param_grads",
+           "hbp_status_string", "hbp_destroy"]
 
 
 class HbpError(RuntimeError):
@@ -61,6 +62,9 @@ def _load():
     lib.hbp_cumsumprod.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.hbp_cumsumprod_static.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp]
     lib.hbp_cumsumprod_static_max_bytes.argtypes = []
+    lib.hbp_iterate.argtypes = [vp, C.POINTER(hbp_params), vp, vp, vp, vp, vp]
+    lib.hbp_add_carry.argtypes = [vp, vp, vp, vp]
+    lib.hbp_param_grads.argtypes = [vp, C.POINTER(hbp_params), vp, vp, vp, C.POINTER(hbp_grads), vp]
     lib.hbp_compare_scratch_bytes.argtypes = [i32]
     lib.hbp_compare.argtypes = [i32, i32, i64, vp, vp, vp, vp, sz, vp]
     lib.hbp_sync_status.argtypes = [vp, vp]
@@ -217,6 +221,24 @@ class Context:
         _check(lib.hbp_exact(self._h, C.byref(p), _ptr(delta), _ptr(x_all), _ptr(inputs), _ptr(g_all),
                              self._grads(grads), _stream()), "hbp_exact")
         return g_all
+
+    # -- the pieces of backward, for callers that run the iterations themselves ----------------
+    def iterate(self, params, delta, x_all, g_all, inputs=None):
+        """One Highway-BP iteration in place on g_all (its last state is read as given, then set to delta_L)."""
+        p = self._params(params)
+        _check(lib.hbp_iterate(self._h, C.byref(p), _ptr(delta), _ptr(x_all), _ptr(inputs), _ptr(g_all), _stream()),
+               "hbp_iterate")
+        return g_all
+
+    def add_carry(self, carry, g_all):
+        _check(lib.hbp_add_carry(self._h, _ptr(carry), _ptr(g_all), _stream()), "hbp_add_carry")
+        return g_all
+
+    def param_grads(self, params, x_all, g_all, grads, inputs=None):
+        p = self._params(params)
+        _check(lib.hbp_param_grads(self._h, C.byref(p), _ptr(x_all), _ptr(inputs), _ptr(g_all), self._grads(grads),
+                                   _stream()), "hbp_param_grads")
+        return grads
 
     def sync_status(self):
         _check(lib.hbp_sync_status(self._h, _stream()), "hbp_sync_status")

@@ -467,6 +467,36 @@ struct Run {
     }
   }
 
+  // ---- all kinds: Eq. 8 for every step at once, and the parameter pass of Section 4.2 ---------------------------
+  void vjp_all() {
+    const int layers = c->layers, grp = c->group;
+    switch (c->cfg.block) {
+      case HBP_BLOCK_RNN_TANH: rnn_vjp_all(); break;
+      case HBP_BLOCK_GRU: gru_vjp_all(); break;
+      default:
+        for (int b0 = 0; b0 < layers; b0 += grp) mlp_vjp(b0, b0 + grp < layers ? b0 + grp : layers, true);
+        if (c->cfg.block == HBP_BLOCK_PRELN_TRANSFORMER) attn_vjp(0, layers, true);
+    }
+  }
+  void wgrad_all(const hbp_grads* gr) {
+    const int layers = c->layers, grp = c->group;
+    switch (c->cfg.block) {
+      case HBP_BLOCK_RNN_TANH: rnn_wgrad(gr); break;
+      case HBP_BLOCK_GRU: gru_wgrad(gr); break;
+      default:
+        for (int b0 = 0; b0 < layers; b0 += grp) {
+          const int b1 = b0 + grp < layers ? b0 + grp : layers;
+          mlp_vjp(b0, b1, false);
+          mlp_wgrad(b0, b1, gr);
+        }
+        if (c->cfg.block == HBP_BLOCK_PRELN_TRANSFORMER) {
+          attn_vjp(0, layers, false);
+          attn_wgrad(0, layers, gr);
+        }
+    }
+    gate_grads(gr);
+  }
+
   void gate_grads(const hbp_grads* gr) {
     if (!gr->da || c->cfg.gate == HBP_GATE_ONE) return;
     if (c->cfg.gate == HBP_GATE_CHANNEL_SHARED) {
@@ -821,36 +851,14 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
     for (int it = 0; it < iters; ++it) {
       {
         PhaseScope ph(r, HBP_PHASE_VJP);
-        if (rnn) {
-          r.rnn_vjp_all();
-        } else if (gru) {
-          r.gru_vjp_all();
-        } else {
-          for (int b0 = 0; b0 < layers; b0 += grp) r.mlp_vjp(b0, b0 + grp < layers ? b0 + grp : layers, true);
-          if (tr) r.attn_vjp(0, layers, true);
-        }
+        r.vjp_all();
       }
       PhaseScope ph(r, HBP_PHASE_SCAN);
       r.scan_with_u(0, steps);
     }
     if (grads) {  // Section 4.2: parameter gradients from the final estimate
       PhaseScope ph(r, HBP_PHASE_WGRAD);
-      if (rnn) {
-        r.rnn_wgrad(grads);
-      } else if (gru) {
-        r.gru_wgrad(grads);
-      } else {
-        for (int b0 = 0; b0 < layers; b0 += grp) {
-          const int b1 = b0 + grp < layers ? b0 + grp : layers;
-          r.mlp_vjp(b0, b1, false);
-          r.mlp_wgrad(b0, b1, grads);
-        }
-        if (tr) {
-          r.attn_vjp(0, layers, false);
-          r.attn_wgrad(0, layers, grads);
-        }
-      }
-      r.gate_grads(grads);
+      r.wgrad_all(grads);
     }
   } else {
     // Section 2.2: g_l = delta_l + a_l g_{l+1} + J_l^T g_{l+1}, one step at a time
@@ -904,6 +912,58 @@ hbp_status hbp_backward(hbp_ctx* ctx, const hbp_params* params, int32_t k, const
 hbp_status hbp_exact(hbp_ctx* ctx, const hbp_params* params, const void* delta, const void* x_all, const void* inputs,
                      void* g_all, const hbp_grads* grads, void* cuda_stream) {
   return backward_common(ctx, params, 0, true, delta, x_all, inputs, g_all, grads, cuda_stream);
+}
+
+hbp_status hbp_iterate(hbp_ctx* ctx, const hbp_params* params, const void* delta, const void* x_all, const void* inputs,
+                       void* g_all, void* cuda_stream) {
+  hbp_status st = check_call(ctx, params, true);
+  if (st != HBP_OK) return st;
+  if (!delta || !x_all || !g_all) return HBP_ERR_INVALID_ARG;
+  if (misaligned(delta) || misaligned(x_all) || misaligned(g_all)) return HBP_ERR_SHAPE;
+  Run r(ctx, params, cuda_stream);
+  r.x_all = (const char*)x_all;
+  r.inputs = (const char*)inputs;
+  r.g = (char*)g_all;
+  r.delta = (const char*)delta;
+  r.shifted = ctx->cfg.gamma != 0.0f;
+  {
+    PhaseScope ph(r, HBP_PHASE_VJP);
+    r.vjp_all();  // from the iterate as given, g_all[steps] included
+  }
+  PhaseScope ph(r, HBP_PHASE_SCAN);
+  r.set_last_state();
+  r.scan_with_u(0, ctx->steps);
+  return r.result();
+}
+
+hbp_status hbp_param_grads(hbp_ctx* ctx, const hbp_params* params, const void* x_all, const void* inputs, const void* g_all,
+                           const hbp_grads* grads, void* cuda_stream) {
+  hbp_status st = check_call(ctx, params, true);
+  if (st != HBP_OK) return st;
+  if (!x_all || !g_all || !grads) return HBP_ERR_INVALID_ARG;
+  if (misaligned(x_all) || misaligned(g_all)) return HBP_ERR_SHAPE;
+  st = check_grads(ctx, grads);
+  if (st != HBP_OK) return st;
+  const hbp_config& f = ctx->cfg;
+  if ((f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU) && !inputs) return HBP_ERR_INVALID_ARG;
+  Run r(ctx, params, cuda_stream);
+  r.x_all = (const char*)x_all;
+  r.inputs = (const char*)inputs;
+  r.g = (char*)const_cast<void*>(g_all);  // read only by the parameter pass
+  PhaseScope ph(r, HBP_PHASE_WGRAD);
+  r.wgrad_all(grads);
+  return r.result();
+}
+
+hbp_status hbp_add_carry(hbp_ctx* ctx, const void* carry, void* g_all, void* cuda_stream) {
+  if (!ctx || !carry || !g_all) return HBP_ERR_INVALID_ARG;
+  if (misaligned(carry) || misaligned(g_all)) return HBP_ERR_SHAPE;
+  if (ctx->cfg.gate != HBP_GATE_ONE || ctx->cfg.gamma != 0.0f || ctx->cfg.block == HBP_BLOCK_GRU) return HBP_ERR_UNSUPPORTED;
+  Launcher lc;
+  lc.stream = (cudaStream_t)cuda_stream;
+  lc.launches = &ctx->launches;
+  add_to_states(lc, ctx->cfg.dtype, g_all, carry, ctx->steps + 1, (int64_t)ctx->cfg.tokens * ctx->cfg.d);
+  return lc.err == cudaSuccess ? HBP_OK : HBP_ERR_CUDA;
 }
 
 size_t hbp_compare_scratch_bytes(int32_t segments) { return segments > 0 ? compare_scratch_bytes(segments) : 0; }

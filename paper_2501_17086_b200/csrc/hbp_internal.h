@@ -128,6 +128,8 @@ bool scan_ring(Launcher& lc, const ScanArgs& s);
 void ln_stats_finish(Launcher& lc, const float2* stats, int slots, const float* rstd, float4* lnstat, int64_t count,
                      int d);
 void copy_state(Launcher& lc, int dtype, void* dst, const void* src, int64_t elems);
+// states[s][e] += carry[e] for s in [0, count)
+void add_to_states(Launcher& lc, int dtype, void* states, const void* carry, int count, int64_t elems);
 // LayerNorm forward of one state: x (float master or dtype) -> xhat (dtype), rstd (float).
 void layernorm_fwd(Launcher& lc, int dtype, const void* x, bool x_is_f32, void* xhat, float* rstd, int64_t rows,
                    int d, float eps);

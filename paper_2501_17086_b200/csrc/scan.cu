@@ -394,6 +394,23 @@ __global__ void copy_kernel(T* __restrict__ dst, const T* __restrict__ src, int6
   if (v < nvec) stv<T>(dst + v * Vec<T>::N, ldv<T>(src + v * Vec<T>::N));
 }
 
+// states[s] += carry for every state s (the carry of a scan whose gates are all one, applied after the fact)
+template <typename T>
+__global__ void add_to_states_kernel(T* __restrict__ states, const T* __restrict__ carry, int64_t elems) {
+  constexpr int V = Vec<T>::N;
+  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v * V >= elems) return;
+  T* p = states + (int64_t)blockIdx.y * elems + v * V;
+  float a[V], c[V];
+  ldv<T>(p).get(a);
+  ldv<T>(carry + v * V).get(c);
+#pragma unroll
+  for (int i = 0; i < V; ++i) a[i] += c[i];
+  Vec<T> out;
+  out.set(a);
+  stv<T>(p, out);
+}
+
 template <typename T>
 __global__ void to_f32_kernel(const T* __restrict__ src, float* __restrict__ dst, int64_t n) {
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -599,6 +616,15 @@ void copy_state(Launcher& lc, int dtype, void* dst, const void* src, int64_t ele
     copy_kernel<float><<<(unsigned)((elems / 4 + 255) / 256), 256, 0, lc.stream>>>((float*)dst, (const float*)src, elems / 4);
   else
     copy_kernel<bf16><<<(unsigned)((elems / 8 + 255) / 256), 256, 0, lc.stream>>>((bf16*)dst, (const bf16*)src, elems / 8);
+  lc.count();
+  lc.check();
+}
+
+void add_to_states(Launcher& lc, int dtype, void* states, const void* carry, int count, int64_t elems) {
+  const int V = dtype == HBP_F32 ? 4 : 8;
+  dim3 grid((unsigned)((elems / V + 255) / 256), (unsigned)count);
+  if (dtype == HBP_F32) add_to_states_kernel<float><<<grid, 256, 0, lc.stream>>>((float*)states, (const float*)carry, elems);
+  else add_to_states_kernel<bf16><<<grid, 256, 0, lc.stream>>>((bf16*)states, (const bf16*)carry, elems);
   lc.count();
   lc.check();
 }

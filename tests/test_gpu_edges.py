@@ -224,3 +224,30 @@ def test_compare_matches_the_definition(dtype):
     with pytest.raises(B.HbpError):
         B.lib.hbp_compare.restype = C.c_int
         B._check(B.lib.hbp_compare(0, 0, 10, None, None, None, None, 0, None), "hbp_compare")
+
+
+@pytest.mark.parametrize("name,world,k", [("c2_twin", 2, 2), ("c2_twin", 3, 4), ("c2_twin_f32", 3, 3), ("c2_twin_f32", 5, 5),
+                                          ("c4_twin", 2, 2), ("c1", 4, 3)])
+def test_layer_parallel_shards_match_the_single_context_and_the_oracle(name, world, k):
+    """Layer-parallel Highway-BP with all shards in this process (one GPU): contexts over layer ranges, the scan's
+    carry handed over between them.  Must agree with the oracle like the single-context path does."""
+    from oracle import run as orun
+    from paper_2501_17086_b200 import harness, layer_parallel as LP
+    from paper_2501_17086_b200.workloads import WORKLOADS, make_inputs
+    from test_gpu_parity import TOL
+    w = WORKLOADS[name]
+    inp = make_inputs(w, "cuda")
+    shards = [LP.Shard(w, r, world, inp) for r in range(world)]
+    out = LP.run(shards, inp["x0"], k, lambda x_last: harness.loss_delta(w, x_last.unsqueeze(0), inp))
+    for s in shards:
+        s.ctx.sync_status()
+    ref = orun.run(w, inp, ks=(k,), exact=False, grads_for=(k,))
+    tol = TOL[w.dtype]
+    per_step = w.steps // w.L
+    for s, (g_all, grads) in zip(shards, out):
+        for j in range(g_all.shape[0]):
+            l = s.lo * per_step + j
+            assert rel(np64(g_all[j]), ref["hbp"][k][l]) < tol, f"rank {s.rank} state {l}"
+        for n, t in grads.items():
+            want = ref["grads"][k][n[1:]][s.lo:s.hi]
+            assert rel(np64(t), want) < tol, f"rank {s.rank} {n}"
