@@ -104,25 +104,37 @@ def dist_exchange(firsts):
     return out
 
 
-def run(shards, x0, k, loss_delta, exchange=local_exchange, pipe=None):
+def dist_pipe(x, src, dst):
+    """Moves a boundary state from rank src to rank dst (one shard per process): the sender passes x, the receiver
+    passes a tensor of the right shape to fill and gets it back."""
+    import torch.distributed as dist
+    if dist.get_rank() == src:
+        dist.send(x.contiguous(), dst)
+        return x
+    dist.recv(x, src)
+    return x
+
+
+def run(shards, x0, k, loss_delta, exchange=local_exchange, pipe=None, carries=carries_over_ranks):
     """Forward through the pipeline, then Highway-BP(k) and the parameter gradients.  `shards` are this process's
     shards in rank order (all of them, or one); `loss_delta(x_last)` gives delta_L on the rank that holds the last
-    layer; `pipe(x, src, dst)` moves a boundary state between processes (None when all shards are local).
+    layer; `pipe(x, src, dst)` moves a boundary state between processes (None when all shards are local);
+    `carries` turns the gathered first-layer values into the per-rank carries.
     Returns the per-shard (g_all, grads)."""
     x = x0
     for s in shards:
         if pipe is not None and s.rank > 0:
-            x = pipe(None, s.rank - 1, s.rank)
+            x = pipe(torch.empty_like(x0), s.rank - 1, s.rank)
         x = s.forward(x)
         if pipe is not None and not s.last:
             pipe(x, s.rank, s.rank + 1)
     delta_last = loss_delta(x) if shards[-1].last else None
 
     def scan_step(firsts):
-        carries = carries_over_ranks(exchange(firsts))
+        carry = carries(exchange(firsts))
         for s in shards:
             if not s.last:
-                s.apply_carry(carries[s.rank + 1])
+                s.apply_carry(carry[s.rank + 1])
 
     scan_step([s.start(delta_last).clone() for s in shards])
     for _ in range(min(k, shards[0].w.steps)):
