@@ -75,7 +75,7 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // tile load of a pair: the destination is this CTA's shared memory, the barrier may be the peer's (a
-// shared::cluster address).  No multicast: each CTA fetches its own half.
+// shared::cluster address).  Each CTA fetches its own half; nothing is broadcast across the pair.
 __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar_cluster, int c0, int c1,
                                                  int c2) {
   asm volatile(
@@ -83,11 +83,12 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
       ::"r"(dst), "l"(tm), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
-// arrives on the barrier at the same offset in both CTAs of the pair once the MMAs issued so far have completed
+// arrives on the barrier at the same offset in both CTAs of the pair once the MMAs issued so far have completed:
+// one commit per CTA, each naming that CTA's barrier by its cluster address
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
-               "h"((uint16_t)3)
-               : "memory");
+  const uint32_t own = map_to_cta(bar, 0), peer = map_to_cta(bar, 1);
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(own) : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(peer) : "memory");
 }
 __device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
   asm volatile(
