@@ -229,6 +229,51 @@ class GRUStep:
         return {"W": rec.T @ c["h"], "U": pre.T @ _f64(self.x_t)}
 
 
+class LSTMStep:
+    """One LSTM cell as a layer on the state x = [c, h] (Table 1, row "LSTM": f(x) = [a(x) * x_c + b(x), c(x)],
+    r(x, z) = [z1 * x_c + z2, z3]).  With [i, f, g, o] = [sigmoid, sigmoid, tanh, sigmoid](U x_t + W h):
+    c' = f * c + i * g,  h' = o * tanh(c').  The residual Jacobian is K = diag([f, 0]): only the cell state has a
+    linear path; everything else, including the path from c to h' through tanh(c'), belongs to J.
+    W [4u, u] and U [4u, in] stack the i, f, g, o rows (u = units; the state is 2u wide)."""
+
+    def __init__(self, W, U, x_t):
+        self.W, self.U, self.x_t = W, U, x_t
+
+    def forward(self, x):
+        W, U = _f64(self.W), _f64(self.U)
+        u = x.shape[-1] // 2
+        c, h = x[..., :u], x[..., u:]
+        pre = _f64(self.x_t) @ U.T + h @ W.T
+        i, f, o = _sigmoid(pre[..., :u]), _sigmoid(pre[..., u:2 * u]), _sigmoid(pre[..., 3 * u:])
+        g = np.tanh(pre[..., 2 * u:3 * u])
+        c_new = f * c + i * g
+        tc = np.tanh(c_new)
+        h_new = o * tc
+        block = np.concatenate([i * g, h_new], axis=-1)          # what r adds to the gated state
+        return block, dict(c=c, h=h, i=i, f=f, g=g, o=o, tc=tc)
+
+    def gate(self, cache):
+        return np.concatenate([cache["f"], np.zeros_like(cache["f"])], axis=-1)
+
+    def _pre_grads(self, k, g):
+        u = k["f"].shape[-1]
+        gc, gh = g[..., :u], g[..., u:]
+        through_h = gh * k["o"] * (1.0 - k["tc"] ** 2)           # dLoss/dc' that arrives through h' = o tanh(c')
+        dct = gc + through_h
+        pre = np.concatenate([dct * k["g"] * k["i"] * (1.0 - k["i"]), dct * k["c"] * k["f"] * (1.0 - k["f"]),
+                              dct * k["i"] * (1.0 - k["g"] ** 2), gh * k["tc"] * k["o"] * (1.0 - k["o"])], axis=-1)
+        return pre, through_h
+
+    def vjp(self, k, g):
+        pre, through_h = self._pre_grads(k, g)
+        # the cell state's share of J: f * (what came through h'); f * g_c itself is K's
+        return np.concatenate([k["f"] * through_h, pre @ _f64(self.W)], axis=-1)
+
+    def param_vjp(self, k, g):
+        pre, _ = self._pre_grads(k, g)
+        return {"W": pre.T @ k["h"], "U": pre.T @ _f64(self.x_t)}
+
+
 class ShiftedStep:
     """The gamma-shifted split of a residual layer x + Block(x) (Appendix C.3, Eq. 17): the block becomes
     g(x) = Block(x) + gamma x and the residual function r(x, z) = (1 - gamma) x + z, so the layer itself is
@@ -292,6 +337,11 @@ def gru_stack(W, U, X):
     """GRU over time; X is [T, B, in]."""
     T = len(X)
     return Stack([GRUStep(W, U, _Lazy(X, t)) for t in range(T)])
+
+
+def lstm_stack(W, U, X):
+    """LSTM over time on the state [c, h]; X is [T, B, in]."""
+    return Stack([LSTMStep(W, U, _Lazy(X, t)) for t in range(len(X))])
 
 
 def rnn_stack(W, U, a, X):

@@ -567,3 +567,65 @@ def test_agreement_sums_on_known_vectors():
     assert abs(s[3] - (s[1] + s[2] - 2 * s[0])) < 1e-12
     t = O.agreement(a, a)
     assert t[0] == t[1] == t[2] and t[3] == 0.0
+
+
+# ---------------------------------------------- 13. LSTM: state [c, h], gate on the cell state only (Table 1)
+def test_lstm_matches_the_library_cell_and_autograd():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(51)
+    T, u, nin, B = 5, 4, 3, 2
+    W = rng.normal(size=(4 * u, u)) * 0.6
+    U = rng.normal(size=(4 * u, nin)) * 0.6
+    X = rng.normal(size=(T, B, nin))
+    st = O.lstm_stack(W, U, X)
+    x0 = rng.normal(size=(B, 2 * u))
+    xs, caches = O.forward(st, x0)
+    cell = torch.nn.LSTMCell(nin, u, bias=False).double()
+    with torch.no_grad():
+        cell.weight_ih.copy_(torch.tensor(U))
+        cell.weight_hh.copy_(torch.tensor(W))
+    x0t = torch.tensor(x0, requires_grad=True)
+    c, h = x0t[:, :u], x0t[:, u:]
+    states = []
+    for t in range(T):
+        h, c = cell(torch.tensor(X[t]), (h, c))
+        states.append(torch.cat([c, h], dim=1))
+    for t in range(T):
+        np.testing.assert_allclose(xs[t + 1], states[t].detach().numpy(), rtol=1e-12, atol=1e-13)
+    Y = rng.normal(size=(T, B, 2 * u))
+    loss = sum(0.5 * ((states[t] - torch.tensor(Y[t])) ** 2).sum() for t in range(T))
+    loss.backward()
+    deltas = [np.zeros_like(x0)] + [xs[t + 1] - Y[t] for t in range(T)]
+    g = O.exact_bp(st, caches, deltas)
+    np.testing.assert_allclose(g[0], x0t.grad.numpy(), rtol=1e-10, atol=1e-12)
+    grads = O.param_grads(st, caches, xs, g, [("", None)] * T)
+    np.testing.assert_allclose(grads["W"], cell.weight_hh.grad.numpy(), rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(grads["U"], cell.weight_ih.grad.numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_lstm_path_sums_and_exactness():
+    rng = np.random.default_rng(52)
+    T, u = 4, 2
+    W = rng.normal(size=(4 * u, u)) * 0.7
+    U = rng.normal(size=(4 * u, 2)) * 0.7
+    X = rng.normal(size=(T, 1, 2))
+    st = O.lstm_stack(W, U, X)
+    xs, caches = O.forward(st, rng.normal(size=(1, 2 * u)))
+    deltas = random_deltas(xs, every=True, rng=rng)
+    J, K = [None], [None]
+    for l in range(T):
+        def cell(xflat, l=l):
+            blk, c = st.steps[l].forward(xflat.reshape(1, 2 * u))
+            return (st.steps[l].gate(c) * xflat.reshape(1, 2 * u) + blk).reshape(-1)
+        full = O.finite_difference_jacobian(cell, xs[l].reshape(-1), h=1e-5)
+        Km = np.diag(st.steps[l].gate(caches[l]).reshape(-1))
+        K.append(Km)
+        J.append(full - Km)
+    flat = [x.reshape(-1) for x in deltas]
+    for k in range(T + 1):
+        w = O.highway_bp(st, caches, deltas, k)
+        for i in range(T + 1):
+            np.testing.assert_allclose(w[i].reshape(-1), O.path_sum(flat, J, K, i, k), rtol=1e-6, atol=1e-8)
+    g = O.exact_bp(st, caches, deltas)
+    for a, b in zip(O.highway_bp(st, caches, deltas, T), g):
+        np.testing.assert_allclose(a, b, rtol=1e-11, atol=1e-12)
