@@ -98,6 +98,9 @@ def algorithmic_flops(w, k):
     if w.block == "gru":
         rows = w.L * w.batch
         return 6 * w.d * w.d * rows, 6 * w.d * (w.d + w.in_dim) * rows
+    if w.block == "lstm":
+        rows, u = w.L * w.batch, w.hidden
+        return 8 * u * u * rows, 8 * u * (u + w.in_dim) * rows
     if w.block == "preln_transformer":
         n, d, s = w.tokens, w.d, w.seq
         blk = 8 * d * d * n + 5 * s * d * n + 16 * d * d * n
@@ -128,7 +131,7 @@ def oracle_timing(w, k, sample, steps, warmup):
         inp64 = {n: (t.double() if n in weights else t) for n, t in inp.items()}
     else:  # too large to hold in float64 at once: converted layer by layer inside the timed calls
         inp64 = inp
-    units = {"preln_transformer": w.batch, "rnn_tanh": w.batch, "gru": w.batch}.get(w.block, w.tokens)
+    units = {"preln_transformer": w.batch, "rnn_tanh": w.batch, "gru": w.batch, "lstm": w.batch}.get(w.block, w.tokens)
     sample = min(sample, units)
     times = []
     for it in range(warmup + steps):
@@ -316,7 +319,7 @@ def run_ours(args):
                     "fp32_alu_peak_tflops": 148 * 128 * 2 * 1.965e9 / 1e12,
                     "peak_source": "of measured bf16 x nominal tf32/bf16 ratio" if peaks else "of fallback", "traffic": None}
     # scan: read u (+ xhat when the LayerNorm finish is fused, + the per-element gate of a GRU), write g
-    tensors = 2 + (1 if w.block in ("preln_mlp", "preln_transformer", "gru") else 0)  # per-step delta is added by the VJP GEMM epilogue
+    tensors = 2 + (1 if w.block in ("preln_mlp", "preln_transformer", "gru", "lstm") else 0)  # per-step delta is added by the VJP GEMM epilogue
     scan_bytes = tensors * w.steps * w.tokens * w.d * es
     hbm = peaks.get("hbm_gbs", 6650.0)
     scan_iter_ms = None
@@ -348,7 +351,7 @@ def run_ours(args):
             "phases_ms_per_step": {"vjp": vjp_ms / args.steps, "scan": scan_ms / args.steps, "wgrad": wg_ms / args.steps},
             "tflops": {"vjp": vjp_flops * kk / (vjp_ms / args.steps * 1e-3) / 1e12 if vjp_ms else None,
                        "wgrad": wgrad_flops / (wg_ms / args.steps * 1e-3) / 1e12 if wg_ms else None},
-            "replicas_tokens_per_s": world * w.tokens * (w.L if w.block in ("rnn_tanh", "gru") else 1) / (ms_step * 1e-3)}
+            "replicas_tokens_per_s": world * w.tokens * (w.L if w.block in ("rnn_tanh", "gru", "lstm") else 1) / (ms_step * 1e-3)}
 
     if not args.no_detail and rank == 0:
         detail = {}

@@ -69,9 +69,14 @@ typedef enum {
  *                    z = sigmoid(U_z x_t + W_z h), n = tanh(U_n x_t + r (.) W_n h), no biases, weights shared over
  *                    t.  The residual gate is the update gate z_t itself, K = diag(z_t): it depends on the state,
  *                    is produced by hbp_forward and kept in the workspace; cfg.gate must be HBP_GATE_ONE (there is
- *                    no further constant gate) and cfg.gamma 0. */
+ *                    no further constant gate) and cfg.gamma 0.
+ *  LSTM              Table 1, row "LSTM": the state is [c, h] (d = 2 * hidden wide); [i, f, g, o] = [sigmoid, sigmoid,
+ *                    tanh, sigmoid](U x_t + W h), c' = f (.) c + i (.) g, h' = o (.) tanh(c'), no biases.  The residual
+ *                    gate is [f_t, 0] (only the cell state has a linear path), produced by hbp_forward like the GRU's;
+ *                    cfg.gate must be HBP_GATE_ONE, cfg.gamma 0, cfg.hidden = d / 2 = the number of units. */
 typedef enum {
-  HBP_BLOCK_MLP = 0, HBP_BLOCK_PRELN_MLP = 1, HBP_BLOCK_RNN_TANH = 2, HBP_BLOCK_PRELN_TRANSFORMER = 3, HBP_BLOCK_GRU = 4
+  HBP_BLOCK_MLP = 0, HBP_BLOCK_PRELN_MLP = 1, HBP_BLOCK_RNN_TANH = 2, HBP_BLOCK_PRELN_TRANSFORMER = 3, HBP_BLOCK_GRU = 4,
+  HBP_BLOCK_LSTM = 5
 } hbp_block;
 typedef enum { HBP_F32 = 0, HBP_BF16 = 1 } hbp_dtype;
 /* Residual gate a_l, the diagonal of K (Eq. 2): all ones, one vector a[d] for every step, or a[steps][d]. */
@@ -87,8 +92,8 @@ typedef struct {
   int32_t loss;     /* hbp_loss  */
   int32_t L;        /* residual steps (MLP kinds), time steps (RNN), decoder blocks (Transformer) */
   int32_t d;        /* state width */
-  int32_t hidden;   /* MLP hidden width (MLP kinds, Transformer) */
-  int32_t in_dim;   /* RNN / GRU input width */
+  int32_t hidden;   /* MLP hidden width (MLP kinds, Transformer); LSTM: units */
+  int32_t in_dim;   /* RNN / GRU / LSTM input width */
   int32_t n_heads;  /* Transformer: n_heads * head_dim == d */
   int32_t head_dim;
   int32_t seq;      /* Transformer: tokens == batch * seq */
@@ -102,6 +107,7 @@ typedef struct {
  *  MLP kinds:    W1 [L][hidden][d], W2 [L][d][hidden]
  *  RNN:          W [d][d], U [d][in_dim]
  *  GRU:          W [3d][d], U [3d][in_dim]: the rows of the r, z and n parts stacked in that order
+ *  LSTM:         W [4u][u], U [4u][in_dim], u = hidden: the rows of the i, f, g and o parts stacked in that order
  *  Transformer:  Wq, Wk, Wv, Wo [L][d][d], W1 [L][hidden][d], W2 [L][d][hidden]
  *  gate:         a [d] or [steps][d] when cfg.gate != HBP_GATE_ONE (steps = 2L for the Transformer) */
 typedef struct {
@@ -131,7 +137,7 @@ hbp_status hbp_create(const hbp_config* cfg, void* workspace, size_t workspace_b
 
 /* Section 3, h_i = f_i(h_{i-1}): runs the steps from x0 [N][d] and stores every state in
  * x_all [steps+1][N][d] (x_all[0] = x0) plus, in the workspace, what the block VJPs need.
- * `inputs` is the RNN's or GRU's x [L][batch][in_dim] (NULL otherwise). */
+ * `inputs` is the recurrent kinds' x [L][batch][in_dim] (NULL otherwise). */
 hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, const void* inputs,
                        void* x_all, void* cuda_stream);
 

@@ -53,6 +53,11 @@ def build_stack(cfg, inputs, rows=None):
         stack = O.gru_stack(_np(inputs["W"]), _np(inputs["U"]), F64Items(X))
         x0 = _np(inputs["x0"] if rows is None else inputs["x0"][rows])
         groups = [("", None)] * cfg.L
+    elif cfg.block == "lstm":
+        X = inputs["X"] if rows is None else inputs["X"][:, rows]
+        stack = O.lstm_stack(_np(inputs["W"]), _np(inputs["U"]), F64Items(X))
+        x0 = _np(inputs["x0"] if rows is None else inputs["x0"][rows])
+        groups = [("", None)] * cfg.L
     elif cfg.block == "preln_transformer":
         stack = O.transformer_stack(*(F64Items(inputs[n]) for n in ("Wq", "Wk", "Wv", "Wo", "W1", "W2")),
                                     cfg.n_heads, cfg.ln_eps)

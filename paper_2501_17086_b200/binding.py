@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhbp.so")
 
 HBP_F32, HBP_BF16 = 0, 1
-BLOCKS = {"mlp": 0, "preln_mlp": 1, "rnn_tanh": 2, "preln_transformer": 3, "gru": 4}
+BLOCKS = {"mlp": 0, "preln_mlp": 1, "rnn_tanh": 2, "preln_transformer": 3, "gru": 4, "lstm": 5}
 GATE_ONE, GATE_CHANNEL_SHARED, GATE_CHANNEL_PER_STEP = 0, 1, 2
 LOSS_FINAL, LOSS_EVERY_STEP = 0, 1
 
@@ -136,6 +136,7 @@ _GRAD_SHAPES = {
     "mlp": lambda c: {"dW1": (c.L, c.hidden, c.d), "dW2": (c.L, c.d, c.hidden)},
     "rnn_tanh": lambda c: {"dW": (c.d, c.d), "dU": (c.d, c.in_dim)},
     "gru": lambda c: {"dW": (3 * c.d, c.d), "dU": (3 * c.d, c.in_dim)},
+    "lstm": lambda c: {"dW": (4 * c.hidden, c.hidden), "dU": (4 * c.hidden, c.in_dim)},
     "preln_transformer": lambda c: {"dW1": (c.L, c.hidden, c.d), "dW2": (c.L, c.d, c.hidden),
                                     **{n: (c.L, c.d, c.d) for n in ("dWq", "dWk", "dWv", "dWo")}},
 }

@@ -63,6 +63,8 @@ struct hbp_ctx {
   // GRU: the update gate z_t [T][B][d] (the diagonal of K), the VJP coefficients [T*B][4d] = [c_r|c_z|c_nr|c_n]
   // and, for the GEMMs that do not take the tf32 splits, g times those coefficients [T*B][4d]
   char *Zc = nullptr, *C4 = nullptr, *A4 = nullptr;
+  // LSTM (u = d / 2 units): the scan's gate [T][B][2u] = [f | 0], the VJP coefficients [T*B][5u] (A4 is [T*B][4u])
+  char *Fg = nullptr, *C5 = nullptr;
   char* scan_scratch = nullptr;
   size_t scan_scratch_bytes = 0;
   float* partial = nullptr;  // split-K / gate-gradient partial sums
@@ -89,7 +91,7 @@ inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 hbp_status check_config(const hbp_config* c) {
   if (!c) return HBP_ERR_INVALID_ARG;
   if (c->dtype != HBP_F32 && c->dtype != HBP_BF16) return HBP_ERR_DTYPE;
-  if (c->block < 0 || c->block > HBP_BLOCK_GRU) return HBP_ERR_UNSUPPORTED;
+  if (c->block < 0 || c->block > HBP_BLOCK_LSTM) return HBP_ERR_UNSUPPORTED;
   if (c->gate < 0 || c->gate > HBP_GATE_CHANNEL_PER_STEP) return HBP_ERR_UNSUPPORTED;
   if (c->loss != HBP_LOSS_FINAL && c->loss != HBP_LOSS_EVERY_STEP) return HBP_ERR_UNSUPPORTED;
   const int v = c->dtype == HBP_F32 ? 4 : 8;
@@ -98,8 +100,10 @@ hbp_status check_config(const hbp_config* c) {
   if (c->gamma != 0.0f && (c->gate != HBP_GATE_ONE || c->block == HBP_BLOCK_RNN_TANH)) return HBP_ERR_UNSUPPORTED;
   if (c->d % v) return HBP_ERR_SHAPE;
   if (c->d / v > 1024) return HBP_ERR_SHAPE;  // one block per row in the LayerNorm kernels
-  if (c->block == HBP_BLOCK_GRU && (c->gate != HBP_GATE_ONE || c->gamma != 0.0f)) return HBP_ERR_UNSUPPORTED;
-  if (c->block == HBP_BLOCK_RNN_TANH || c->block == HBP_BLOCK_GRU) {
+  const bool gated_cell = c->block == HBP_BLOCK_GRU || c->block == HBP_BLOCK_LSTM;
+  if (gated_cell && (c->gate != HBP_GATE_ONE || c->gamma != 0.0f)) return HBP_ERR_UNSUPPORTED;
+  if (c->block == HBP_BLOCK_LSTM && (c->hidden <= 0 || c->hidden % v || 2 * c->hidden != c->d)) return HBP_ERR_SHAPE;
+  if (c->block == HBP_BLOCK_RNN_TANH || gated_cell) {
     if (c->in_dim <= 0 || c->in_dim % v) return HBP_ERR_SHAPE;
     if (c->batch != c->tokens) return HBP_ERR_SHAPE;
   } else {
@@ -132,10 +136,26 @@ size_t carve(hbp_ctx* c, char* base) {
   const size_t steps = (size_t)c->steps;
   c->status = (int*)take(256);
   c->U = take(steps * N * d * es);
-  const bool recurrent = f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU;
+  const bool recurrent = f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU || f.block == HBP_BLOCK_LSTM;
   if (f.dtype == HBP_BF16 && !recurrent) c->xres = (float*)take(N * d * 4);
   c->partial_floats = (size_t)kGateBlocks * d;
-  if (f.block == HBP_BLOCK_GRU) {
+  if (f.block == HBP_BLOCK_LSTM) {
+    const size_t in = (size_t)f.in_dim, u = d / 2, rows = steps * N;
+    c->Fg = take(rows * d * es);
+    c->C5 = take(rows * 5 * u * es);
+    c->A4 = take(rows * 4 * u * es);
+    c->hres = (double*)take(2 * N * d * 8);
+    if (f.dtype == HBP_F32) {
+      c->Ahi = (float*)take(rows * 4 * u * 4); c->Alo = (float*)take(rows * 4 * u * 4);
+      c->Hhi = (float*)take(rows * u * 4); c->Hlo = (float*)take(rows * u * 4);
+      c->Xhi = (float*)take(rows * in * 4); c->Xlo = (float*)take(rows * in * 4);
+      c->Whi = (float*)take(4 * u * u * 4); c->Wlo = (float*)take(4 * u * u * 4);
+    }
+    c->scan_scratch_bytes = scan_scratch_bytes(f.dtype, f.L, f.tokens, f.d);
+    c->scan_scratch = take(c->scan_scratch_bytes);
+    const size_t wmax = 4 * u * (u > in ? u : in);
+    if ((size_t)kMaxSplit * wmax > c->partial_floats) c->partial_floats = (size_t)kMaxSplit * wmax;
+  } else if (f.block == HBP_BLOCK_GRU) {
     const size_t in = (size_t)f.in_dim;
     c->Zc = take(steps * N * d * es);
     c->C4 = take(steps * N * 4 * d * es);
@@ -467,12 +487,77 @@ struct Run {
     }
   }
 
+  // ---- LSTM (u = d / 2 units; rows of g, U and the states are 2u wide) ------------------------------------
+  // u_h = [t c_i | t c_f | t c_g | g_h c_o] W for every t at once (one GEMM, K = 4u); u_c elementwise beside it
+  void lstm_vjp_all() {
+    const int T = c->cfg.L;
+    const int64_t rows = (int64_t)T * N, u = d / 2;
+    const bool every = c->cfg.loss == HBP_LOSS_EVERY_STEP;
+    GemmArgs a = base_args();
+    a.M = (int)rows; a.N = (int)u; a.K = (int)(4 * u);
+    a.A = c->A4; a.a_sm = 4 * u; a.a_sk = 1;
+    a.B = p->W; a.b_sn = 1; a.b_sk = u;
+    a.epi = EPI_STORE; a.D = at(c->U, u); a.ldd = d;
+    if (every) {  // u_t + delta_t on both halves: the GEMM epilogue adds the h half, the operand kernels the c half
+      a.epi = EPI_ADD; a.E = at(delta, u); a.lde = d;
+      u_has_delta = true;
+    }
+    const void* dl = every ? delta : nullptr;
+    bool tc = false;
+    if (c->Ahi && !g_force_simt) {
+      lstm_split(lc, (const float*)at(g, state), (const float*)c->C5, (const float*)c->Fg, (const float*)dl, c->Ahi, c->Alo,
+                 (float*)c->U, rows, (int)u);
+      a.A_hi = c->Ahi; a.A_lo = c->Alo; a.hl_a_sm = 4 * u; a.hl_a_sk = 1;
+      a.B_hi = c->Whi; a.B_lo = c->Wlo; a.hl_b_sn = 4 * u; a.hl_b_sk = 1;
+      tc = gemm_tc(lc, a, c->status);
+    }
+    if (!tc) {
+      lstm_operand(lc, c->cfg.dtype, at(g, state), c->C5, c->Fg, dl, c->A4, c->U, rows, (int)u);
+      a.A_hi = a.A_lo = a.B_hi = a.B_lo = nullptr;
+      run_gemm(a);
+    }
+  }
+  // dW = [..]^T H (H = the h half of states 0..T-1), dU = [..]^T X with the same four-block operand
+  void lstm_wgrad(const hbp_grads* gr) {
+    const int T = c->cfg.L;
+    const int64_t rows = (int64_t)T * N, in = c->cfg.in_dim, u = d / 2;
+    int split = (int)(rows / (c->Ahi ? 512 : 2048));
+    if (split < 1) split = 1;
+    if (split > kMaxSplit) split = kMaxSplit;
+    const bool try_tc = c->Ahi && !g_force_simt;
+    if (try_tc) lstm_split_transposed(lc, (const float*)at(g, state), (const float*)c->C5, c->Ahi, c->Alo, rows, (int)u);
+    bool have_a4 = false;
+    for (int w = 0; w < 2; ++w) {
+      const int64_t n = w == 0 ? u : in;
+      GemmArgs a = base_args();
+      a.M = (int)(4 * u); a.N = (int)n; a.K = (int)rows;
+      a.A = c->A4; a.a_sm = 1; a.a_sk = 4 * u;
+      a.B = w == 0 ? at(x_all, u) : inputs; a.b_sn = 1; a.b_sk = w == 0 ? d : in;
+      a.epi = EPI_STORE; a.d_f32 = true;
+      a.D = w == 0 ? gr->dW : gr->dU; a.ldd = n;
+      if (split > 1) { a.splitk = split; a.partial = c->partial; }
+      bool tc = false;
+      if (try_tc) {
+        a.A_hi = c->Ahi; a.A_lo = c->Alo; a.hl_a_sm = rows; a.hl_a_sk = 1;
+        a.B_hi = w == 0 ? c->Hhi : c->Xhi; a.B_lo = w == 0 ? c->Hlo : c->Xlo; a.hl_b_sn = rows; a.hl_b_sk = 1;
+        tc = gemm_tc(lc, a, c->status);
+      }
+      if (!tc) {
+        if (!have_a4) lstm_operand(lc, c->cfg.dtype, at(g, state), c->C5, c->Fg, nullptr, c->A4, nullptr, rows, (int)u);
+        have_a4 = true;
+        a.A_hi = a.A_lo = a.B_hi = a.B_lo = nullptr;
+        run_gemm(a);
+      }
+    }
+  }
+
   // ---- all kinds: Eq. 8 for every step at once, and the parameter pass of Section 4.2 ---------------------------
   void vjp_all() {
     const int layers = c->layers, grp = c->group;
     switch (c->cfg.block) {
       case HBP_BLOCK_RNN_TANH: rnn_vjp_all(); break;
       case HBP_BLOCK_GRU: gru_vjp_all(); break;
+      case HBP_BLOCK_LSTM: lstm_vjp_all(); break;
       default:
         for (int b0 = 0; b0 < layers; b0 += grp) mlp_vjp(b0, b0 + grp < layers ? b0 + grp : layers, true);
         if (c->cfg.block == HBP_BLOCK_PRELN_TRANSFORMER) attn_vjp(0, layers, true);
@@ -483,6 +568,7 @@ struct Run {
     switch (c->cfg.block) {
       case HBP_BLOCK_RNN_TANH: rnn_wgrad(gr); break;
       case HBP_BLOCK_GRU: gru_wgrad(gr); break;
+      case HBP_BLOCK_LSTM: lstm_wgrad(gr); break;
       default:
         for (int b0 = 0; b0 < layers; b0 += grp) {
           const int b1 = b0 + grp < layers ? b0 + grp : layers;
@@ -528,6 +614,7 @@ struct Run {
     s.delta = delta; s.loss = c->cfg.loss;
     s.a = p->a; s.gate = c->cfg.gate;
     if (c->cfg.block == HBP_BLOCK_GRU) { s.a = c->Zc; s.gate = kGateElement; }
+    if (c->cfg.block == HBP_BLOCK_LSTM) { s.a = c->Fg; s.gate = kGateElement; }
     s.g = g;
     if (with_u && c->preln) {
       s.xhat = c->Y; s.rstd = c->rstd;
@@ -574,7 +661,7 @@ hbp_status check_call(hbp_ctx* ctx, const hbp_params* p, bool need_forward) {
   if (!ctx || !p) return HBP_ERR_INVALID_ARG;
   if (need_forward && !ctx->forward_done) return HBP_ERR_STATE;
   const hbp_config& f = ctx->cfg;
-  if (f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU) {
+  if (f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU || f.block == HBP_BLOCK_LSTM) {
     if (!p->W || !p->U) return HBP_ERR_INVALID_ARG;
   } else {
     if (!p->W1 || !p->W2) return HBP_ERR_INVALID_ARG;
@@ -587,7 +674,7 @@ hbp_status check_call(hbp_ctx* ctx, const hbp_params* p, bool need_forward) {
 hbp_status check_grads(const hbp_ctx* ctx, const hbp_grads* g) {
   if (!g) return HBP_OK;
   const hbp_config& f = ctx->cfg;
-  if (f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU) return (g->dW && g->dU) ? HBP_OK : HBP_ERR_INVALID_ARG;
+  if (f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU || f.block == HBP_BLOCK_LSTM) return (g->dW && g->dU) ? HBP_OK : HBP_ERR_INVALID_ARG;
   if (!g->dW1 || !g->dW2) return HBP_ERR_INVALID_ARG;
   if (f.block == HBP_BLOCK_PRELN_TRANSFORMER && (!g->dWq || !g->dWk || !g->dWv || !g->dWo)) return HBP_ERR_INVALID_ARG;
   return HBP_OK;
@@ -708,7 +795,7 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
   if (!x0 || !x_all) return HBP_ERR_INVALID_ARG;
   if (misaligned(x0) || misaligned(x_all)) return HBP_ERR_SHAPE;
   const hbp_config& f = ctx->cfg;
-  if ((f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU) && !inputs) return HBP_ERR_INVALID_ARG;
+  if ((f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU || f.block == HBP_BLOCK_LSTM) && !inputs) return HBP_ERR_INVALID_ARG;
   Run r(ctx, params, cuda_stream);
   r.x_all = (const char*)x_all;
   char* xa = (char*)x_all;
@@ -716,7 +803,23 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
   copy_state(r.lc, f.dtype, xa, x0, state);
   if (ctx->xres) convert_to_f32(r.lc, f.dtype, x0, ctx->xres, state);
 
-  if (f.block == HBP_BLOCK_GRU) {
+  if (f.block == HBP_BLOCK_LSTM) {
+    const int T = f.L;
+    const int64_t u = d / 2;
+    convert_to_f64(r.lc, f.dtype, x0, ctx->hres, state);
+    for (int t = 0; t < T; ++t) {
+      const double* sin = ctx->hres + (int64_t)(t & 1) * state;
+      double* sout = ctx->hres + (int64_t)((t + 1) & 1) * state;
+      lstm_forward_step(r.lc, f.dtype, params->W, params->U, r.at(inputs, (int64_t)t * N * f.in_dim), sin, sout,
+                        r.at(ctx->Fg, (int64_t)t * state), r.at(ctx->C5, (int64_t)t * N * 5 * u),
+                        r.at(xa, (int64_t)(t + 1) * state), (int)N, (int)u, f.in_dim);
+    }
+    if (ctx->Ahi) {
+      split_tf32_transposed(r.lc, (const float*)xa + u, nullptr, ctx->Hhi, ctx->Hlo, (int64_t)T * N, (int)u, d);
+      split_tf32_transposed(r.lc, (const float*)inputs, nullptr, ctx->Xhi, ctx->Xlo, (int64_t)T * N, f.in_dim);
+      split_tf32_transposed(r.lc, (const float*)params->W, nullptr, ctx->Whi, ctx->Wlo, 4 * u, (int)u);  // -> [u][4u]
+    }
+  } else if (f.block == HBP_BLOCK_GRU) {
     const int T = f.L;
     convert_to_f64(r.lc, f.dtype, x0, ctx->hres, state);
     for (int t = 0; t < T; ++t) {
@@ -826,7 +929,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
   st = check_grads(ctx, grads);
   if (st != HBP_OK) return st;
   const hbp_config& f = ctx->cfg;
-  if ((f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU) && grads && !inputs) return HBP_ERR_INVALID_ARG;
+  if ((f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU || f.block == HBP_BLOCK_LSTM) && grads && !inputs) return HBP_ERR_INVALID_ARG;
   Run r(ctx, params, cuda_stream);
   r.x_all = (const char*)x_all;
   r.inputs = (const char*)inputs;
@@ -885,6 +988,17 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
                           r.at(r.g, (int64_t)t * r.state), (int)r.N, (int)r.d);
       }
       if (grads) r.gru_wgrad(grads);
+    } else if (f.block == HBP_BLOCK_LSTM) {
+      convert_to_f64(r.lc, f.dtype, r.at(r.g, (int64_t)steps * r.state), ctx->hres, r.state);
+      for (int t = steps - 1; t >= 0; --t) {
+        const double* gin = ctx->hres + (int64_t)((steps - 1 - t) & 1) * r.state;
+        double* gout = ctx->hres + (int64_t)((steps - t) & 1) * r.state;
+        lstm_backward_step(r.lc, f.dtype, params->W, r.at(ctx->Fg, (int64_t)t * r.state),
+                           r.at(ctx->C5, (int64_t)t * r.N * 5 * (r.d / 2)),
+                           f.loss == HBP_LOSS_EVERY_STEP ? r.at(r.delta, (int64_t)t * r.state) : nullptr, gin, gout,
+                           r.at(r.g, (int64_t)t * r.state), (int)r.N, (int)(r.d / 2));
+      }
+      if (grads) r.lstm_wgrad(grads);
     } else {
       for (int l = steps - 1; l >= 0; --l) {
         const int b = tr ? l / 2 : l;
@@ -945,7 +1059,7 @@ hbp_status hbp_param_grads(hbp_ctx* ctx, const hbp_params* params, const void* x
   st = check_grads(ctx, grads);
   if (st != HBP_OK) return st;
   const hbp_config& f = ctx->cfg;
-  if ((f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU) && !inputs) return HBP_ERR_INVALID_ARG;
+  if ((f.block == HBP_BLOCK_RNN_TANH || f.block == HBP_BLOCK_GRU || f.block == HBP_BLOCK_LSTM) && !inputs) return HBP_ERR_INVALID_ARG;
   Run r(ctx, params, cuda_stream);
   r.x_all = (const char*)x_all;
   r.inputs = (const char*)inputs;
@@ -958,7 +1072,9 @@ hbp_status hbp_param_grads(hbp_ctx* ctx, const hbp_params* params, const void* x
 hbp_status hbp_add_carry(hbp_ctx* ctx, const void* carry, void* g_all, void* cuda_stream) {
   if (!ctx || !carry || !g_all) return HBP_ERR_INVALID_ARG;
   if (misaligned(carry) || misaligned(g_all)) return HBP_ERR_SHAPE;
-  if (ctx->cfg.gate != HBP_GATE_ONE || ctx->cfg.gamma != 0.0f || ctx->cfg.block == HBP_BLOCK_GRU) return HBP_ERR_UNSUPPORTED;
+  if (ctx->cfg.gate != HBP_GATE_ONE || ctx->cfg.gamma != 0.0f || ctx->cfg.block == HBP_BLOCK_GRU ||
+      ctx->cfg.block == HBP_BLOCK_LSTM)
+    return HBP_ERR_UNSUPPORTED;
   Launcher lc;
   lc.stream = (cudaStream_t)cuda_stream;
   lc.launches = &ctx->launches;

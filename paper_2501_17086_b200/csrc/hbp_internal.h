@@ -141,7 +141,9 @@ void reduce_splitk(Launcher& lc, const float* partial, float* out, int splits, i
 // hi = tf32-exact part of v, lo = tf32 rounding of (v - hi), with v = a[i] * (b ? b[i] : 1).
 void split_tf32(Launcher& lc, const float* a, const float* b, float* hi, float* lo, int64_t elems);
 // The same for a [rows][cols] matrix, written transposed: hiT, loT are [cols][rows].
-void split_tf32_transposed(Launcher& lc, const float* a, const float* b, float* hiT, float* loT, int64_t rows, int cols);
+// (ld = elements between rows of a and b; 0 = cols)
+void split_tf32_transposed(Launcher& lc, const float* a, const float* b, float* hiT, float* loT, int64_t rows, int cols,
+                           int64_t ld = 0);
 
 // ---------------------------------------------------------------- RNN forward step (rnn.cu)
 // z = W h + U x_t in double from the double master state h_in; writes h_out (double), the cached
@@ -173,6 +175,23 @@ void gru_operand(Launcher& lc, int dtype, const void* g, const void* c4, void* a
 // tf32 high/low split of g * c4: columns [0, 3d) as [rows][3d], or all of it transposed as [4d][rows].
 void gru_split(Launcher& lc, const float* g, const float* c4, float* hi, float* lo, int64_t rows, int d);
 void gru_split_transposed(Launcher& lc, const float* g, const float* c4, float* hiT, float* loT, int64_t rows, int d);
+
+// ---------------------------------------------------------------- LSTM (lstm.cu); u units, state [c | h] 2u wide
+// One forward step in double from the double master state; writes the new master, the stored state, the scan's
+// gate fg [B][2u] = [f | 0] and the VJP coefficients c5 [B][5u] = [c_i | c_f | c_g | c_o | c_h].
+void lstm_forward_step(Launcher& lc, int dtype, const void* W, const void* U, const void* x_t, const double* s_in,
+                       double* s_out, void* fg, void* c5, void* state_out, int B, int u, int in_dim);
+// exact backpropagation through one step in double from the double master g_in
+void lstm_backward_step(Launcher& lc, int dtype, const void* W, const void* fg, const void* c5, const void* delta,
+                        const double* g_in, double* g_out, void* g_store, int B, int u);
+// a4 [rows][4u] = [t c_i | t c_f | t c_g | g_h c_o], t = g_c + g_h c_h, from g [rows][2u]; if uo is given also the
+// cell-state half of the block VJP, uo[row][0..u) = f g_h c_h (+ delta), rows of uo 2u wide
+void lstm_operand(Launcher& lc, int dtype, const void* g, const void* c5, const void* fg, const void* delta, void* a4,
+                  void* uo, int64_t rows, int u);
+// the same operand as tf32 high/low parts: [rows][4u] (with the optional uo), or transposed [4u][rows]
+void lstm_split(Launcher& lc, const float* g, const float* c5, const float* fg, const float* delta, float* hi, float* lo,
+                float* uo, int64_t rows, int u);
+void lstm_split_transposed(Launcher& lc, const float* g, const float* c5, float* hiT, float* loT, int64_t rows, int u);
 
 // ---------------------------------------------------------------- attention (attention.cu)
 struct AttnArgs {

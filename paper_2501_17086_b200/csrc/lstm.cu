@@ -1,0 +1,290 @@
+// LSTM cell as a residual step on the state x = [c, h] (Table 1, row "LSTM"), u units, state width 2u:
+//     [i, f, g, o] = [sigmoid, sigmoid, tanh, sigmoid](U x_t + W h),   c' = f * c + i * g,   h' = o * tanh(c').
+// K = diag([f, 0]) is the cheap Jacobian (only the cell state has a linear path).  With the upstream gradient
+// [g_c, g_h], t = g_c + g_h * c_h is what reaches c' (c_h = o (1 - tanh(c')^2)), and the block VJP is
+//     u_c = f * g_h * c_h,     u_h = [t c_i | t c_f | t c_g | g_h c_o] W
+// with the per-element coefficients c_i = g i (1 - i), c_f = c f (1 - f), c_g = i (1 - g^2), c_o = tanh(c') o (1 - o),
+// computed once, in double, by the forward step and stored as C5 = [c_i | c_f | c_g | c_o | c_h] per row.  The
+// parameter gradients contract the same four-block operand with h and with x_t.  As for the other recurrent cells,
+// the recurrence itself and exact backpropagation through time are carried in double beside the stored values.
+#include "hbp_internal.h"
+
+namespace hbp {
+
+namespace {
+
+constexpr int kTile = 32;
+
+// acc[q][j] += sum_k src[m_j][k] * Wm[q * u + n][k] over k in [0, kdim); src rows are src_ld apart
+template <typename T, bool kSrcDouble>
+__device__ __forceinline__ void lstm_accumulate(const void* __restrict__ src, int64_t src_ld, const T* __restrict__ Wm,
+                                                int kdim, int B, int u, int m0, int n0, double (*Hs)[kTile + 1],
+                                                float (*Ws)[kTile][kTile + 1], double acc[4][4]) {
+  const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
+  for (int k0 = 0; k0 < kdim; k0 += kTile) {
+    for (int i = ty; i < kTile; i += 8) {
+      const int k = k0 + tx, m = m0 + i, n = n0 + i;
+      double hv = 0.0;
+      if (k < kdim && m < B)
+        hv = kSrcDouble ? ((const double*)src)[(int64_t)m * src_ld + k] : (double)to_f(((const T*)src)[(int64_t)m * src_ld + k]);
+      Hs[i][tx] = hv;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) Ws[q][i][tx] = (k < kdim && n < u) ? to_f(Wm[((int64_t)q * u + n) * kdim + k]) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int kk = 0; kk < kTile; ++kk) {
+      double w[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) w[q] = (double)Ws[q][tx][kk];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const double hv = Hs[ty + 8 * j][kk];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[q][j] = fma(hv, w[q], acc[q][j]);
+      }
+    }
+    __syncthreads();
+  }
+}
+
+__device__ __forceinline__ double sigmoid_d(double v) { return 1.0 / (1.0 + exp(-v)); }
+// tanh(v) and 1 - tanh(v)^2 = 4e / (1 + e)^2 with e = exp(-2|v|): no cancellation near saturation
+__device__ __forceinline__ void tanh_and_slope(double v, double& t, double& s) {
+  const double e = exp(-2.0 * fabs(v));
+  t = copysign((1.0 - e) / (1.0 + e), v);
+  s = 4.0 * e / ((1.0 + e) * (1.0 + e));
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) lstm_step_kernel(const T* __restrict__ W, const T* __restrict__ U,
+                                                        const T* __restrict__ x_t, const double* __restrict__ s_in,
+                                                        double* __restrict__ s_out, T* __restrict__ fg,
+                                                        T* __restrict__ c5, T* __restrict__ state_out, int B, int u,
+                                                        int in_dim) {
+  __shared__ double Hs[kTile][kTile + 1];
+  __shared__ float Ws[4][kTile][kTile + 1];
+  const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
+  const int n0 = blockIdx.x * kTile, m0 = blockIdx.y * kTile;
+  double acc[4][4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[q][j] = 0.0;
+  lstm_accumulate<T, true>(s_in + u, 2 * u, W, u, B, u, m0, n0, Hs, Ws, acc);   // W h: h is the second half of the state
+  lstm_accumulate<T, false>(x_t, in_dim, U, in_dim, B, u, m0, n0, Hs, Ws, acc);  // + U x_t
+  const int n = n0 + tx;
+  if (n >= u) return;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int m = m0 + ty + 8 * j;
+    if (m >= B) continue;
+    const double i = sigmoid_d(acc[0][j]), i1 = sigmoid_d(-acc[0][j]);
+    const double f = sigmoid_d(acc[1][j]), f1 = sigmoid_d(-acc[1][j]);
+    const double o = sigmoid_d(acc[3][j]), o1 = sigmoid_d(-acc[3][j]);
+    double g, dg, tc, dtc;
+    tanh_and_slope(acc[2][j], g, dg);
+    const double c = s_in[(int64_t)m * 2 * u + n];
+    const double cn = f * c + i * g;
+    tanh_and_slope(cn, tc, dtc);
+    const double hn = o * tc;
+    const int64_t so = (int64_t)m * 2 * u + n;
+    s_out[so] = cn;
+    s_out[so + u] = hn;
+    state_out[so] = from_f<T>((float)cn);
+    state_out[so + u] = from_f<T>((float)hn);
+    fg[so] = from_f<T>((float)f);
+    fg[so + u] = from_f<T>(0.0f);
+    T* k = c5 + (int64_t)m * 5 * u + n;
+    k[0] = from_f<T>((float)(g * i * i1));
+    k[u] = from_f<T>((float)(c * f * f1));
+    k[2 * u] = from_f<T>((float)(i * dg));
+    k[3 * u] = from_f<T>((float)(tc * o * o1));
+    k[4 * u] = from_f<T>((float)(o * dtc));
+  }
+}
+
+__device__ __forceinline__ double as_d(double v) { return v; }
+__device__ __forceinline__ double as_d(float v) { return (double)v; }
+__device__ __forceinline__ double as_d(bf16 v) { return (double)to_f(v); }
+
+// element (row, column k of the [4u] operand) from the upstream gradient [g_c | g_h] and the coefficients
+template <typename T, typename G>
+__device__ __forceinline__ double operand_value(const G* __restrict__ g_row, const T* __restrict__ c5_row, int u, int k) {
+  const int q = k / u, n = k - q * u;
+  const double gh = as_d(g_row[u + n]);
+  if (q == 3) return gh * (double)to_f(c5_row[3 * u + n]);
+  const double t = as_d(g_row[n]) + gh * (double)to_f(c5_row[4 * u + n]);
+  return t * (double)to_f(c5_row[q * u + n]);
+}
+
+// Exact backpropagation through one step in double: g_t = delta_t + [f * g_c, 0] + [u_c, u_h].
+template <typename T>
+__global__ void __launch_bounds__(256) lstm_bwd_step_kernel(const T* __restrict__ W, const T* __restrict__ fg,
+                                                            const T* __restrict__ c5, const T* __restrict__ delta,
+                                                            const double* __restrict__ g_in, double* __restrict__ g_out,
+                                                            T* __restrict__ g_store, int B, int u) {
+  __shared__ double Hs[kTile][kTile + 1];
+  __shared__ float Ws[kTile][kTile + 1];
+  const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
+  const int n0 = blockIdx.x * kTile, m0 = blockIdx.y * kTile;
+  double acc[4] = {0.0, 0.0, 0.0, 0.0};
+  for (int k0 = 0; k0 < 4 * u; k0 += kTile) {  // u is a multiple of 4, not of the tile: blocks may straddle gates
+    for (int i = ty; i < kTile; i += 8) {
+      const int m = m0 + i, k = k0 + tx;
+      Hs[i][tx] = (m < B && k < 4 * u) ? operand_value<T, double>(g_in + (int64_t)m * 2 * u, c5 + (int64_t)m * 5 * u, u, k) : 0.0;
+      const int kk = k0 + i, n = n0 + tx;  // W[k][n]: contiguous in n
+      Ws[tx][i] = (kk < 4 * u && n < u) ? to_f(W[(int64_t)kk * u + n]) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < kTile; ++kk) {
+      const double w = (double)Ws[tx][kk];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[j] = fma(Hs[ty + 8 * j][kk], w, acc[j]);
+    }
+    __syncthreads();
+  }
+  const int n = n0 + tx;
+  if (n >= u) return;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int m = m0 + ty + 8 * j;
+    if (m >= B) continue;
+    const int64_t so = (int64_t)m * 2 * u + n;
+    const double f = (double)to_f(fg[so]), ch = (double)to_f(c5[(int64_t)m * 5 * u + 4 * u + n]);
+    const double gc = g_in[so], gh = g_in[so + u];
+    const double vc = (delta ? (double)to_f(delta[so]) : 0.0) + f * (gc + gh * ch);
+    const double vh = (delta ? (double)to_f(delta[so + u]) : 0.0) + acc[j];
+    g_out[so] = vc;
+    g_out[so + u] = vh;
+    g_store[so] = from_f<T>((float)vc);
+    g_store[so + u] = from_f<T>((float)vh);
+  }
+}
+
+// The cell-state half of the block VJP (+ delta when given): uo[row][n] = f g_h c_h, n < u.  uo rows are 2u wide.
+template <typename T>
+__device__ __forceinline__ void write_uc(const T* g_row, const T* c5_row, const T* fg_row, const T* delta_row, T* uo_row,
+                                         int u, int n) {
+  float v = to_f(fg_row[n]) * to_f(g_row[u + n]) * to_f(c5_row[4 * u + n]);
+  if (delta_row) v += to_f(delta_row[n]);
+  uo_row[n] = from_f<T>(v);
+}
+
+// a4[row][k] = operand (in dtype) for the GEMMs that do not take the tf32 splits; optionally the u_c half
+template <typename T>
+__global__ void lstm_operand_kernel(const T* __restrict__ g, const T* __restrict__ c5, const T* __restrict__ fg,
+                                    const T* __restrict__ delta, T* __restrict__ a4, T* __restrict__ uo, int64_t rows,
+                                    int u) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= rows * 4 * u) return;
+  const int64_t row = i / (4 * u);
+  const int k = (int)(i - row * 4 * u);
+  const T* g_row = g + row * 2 * u;
+  a4[i] = from_f<T>((float)operand_value<T, T>(g_row, c5 + row * 5 * u, u, k));
+  if (uo && k < u) write_uc<T>(g_row, c5 + row * 5 * u, fg + row * 2 * u, delta ? delta + row * 2 * u : nullptr, uo + row * 2 * u, u, k);
+}
+
+// tf32 split of the operand as [rows][4u]; optionally the u_c half (float data)
+__global__ void lstm_split_kernel(const float* __restrict__ g, const float* __restrict__ c5, const float* __restrict__ fg,
+                                  const float* __restrict__ delta, float* __restrict__ hi, float* __restrict__ lo,
+                                  float* __restrict__ uo, int64_t rows, int u) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= rows * 4 * u) return;
+  const int64_t row = i / (4 * u);
+  const int k = (int)(i - row * 4 * u);
+  const float* g_row = g + row * 2 * u;
+  const float v = (float)operand_value<float, float>(g_row, c5 + row * 5 * u, u, k);
+  const float h = round_tf32(v);
+  hi[i] = h;
+  lo[i] = round_tf32(v - h);
+  if (uo && k < u) write_uc<float>(g_row, c5 + row * 5 * u, fg + row * 2 * u, delta ? delta + row * 2 * u : nullptr, uo + row * 2 * u, u, k);
+}
+
+// the same operand written transposed, [4u][rows] (the weight-gradient GEMMs contract over rows)
+__global__ void __launch_bounds__(256) lstm_split_transposed_kernel(const float* __restrict__ g, const float* __restrict__ c5,
+                                                                    float* __restrict__ hiT, float* __restrict__ loT,
+                                                                    int64_t rows, int u) {
+  __shared__ float th[32][33], tl[32][33];
+  const int64_t r0 = (int64_t)blockIdx.x * 32;
+  const int c0 = blockIdx.y * 32;
+  const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
+  for (int i = ty; i < 32; i += 8) {
+    const int64_t r = r0 + i;
+    const int c = c0 + tx;
+    float v = 0.0f;
+    if (r < rows && c < 4 * u) v = (float)operand_value<float, float>(g + r * 2 * u, c5 + r * 5 * u, u, c);
+    const float h = round_tf32(v);
+    th[i][tx] = h;
+    tl[i][tx] = round_tf32(v - h);
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int c = c0 + i;
+    const int64_t r = r0 + tx;
+    if (c < 4 * u && r < rows) {
+      hiT[(int64_t)c * rows + r] = th[tx][i];
+      loT[(int64_t)c * rows + r] = tl[tx][i];
+    }
+  }
+}
+
+}  // namespace
+
+void lstm_forward_step(Launcher& lc, int dtype, const void* W, const void* U, const void* x_t, const double* s_in,
+                       double* s_out, void* fg, void* c5, void* state_out, int B, int u, int in_dim) {
+  dim3 grid((u + kTile - 1) / kTile, (B + kTile - 1) / kTile);
+  if (dtype == HBP_F32)
+    lstm_step_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)U, (const float*)x_t, s_in, s_out,
+                                                         (float*)fg, (float*)c5, (float*)state_out, B, u, in_dim);
+  else
+    lstm_step_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)U, (const bf16*)x_t, s_in, s_out,
+                                                        (bf16*)fg, (bf16*)c5, (bf16*)state_out, B, u, in_dim);
+  lc.count();
+  lc.check();
+}
+
+void lstm_backward_step(Launcher& lc, int dtype, const void* W, const void* fg, const void* c5, const void* delta,
+                        const double* g_in, double* g_out, void* g_store, int B, int u) {
+  dim3 grid((u + kTile - 1) / kTile, (B + kTile - 1) / kTile);
+  if (dtype == HBP_F32)
+    lstm_bwd_step_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)fg, (const float*)c5,
+                                                             (const float*)delta, g_in, g_out, (float*)g_store, B, u);
+  else
+    lstm_bwd_step_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)fg, (const bf16*)c5,
+                                                            (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, u);
+  lc.count();
+  lc.check();
+}
+
+void lstm_operand(Launcher& lc, int dtype, const void* g, const void* c5, const void* fg, const void* delta, void* a4,
+                  void* uo, int64_t rows, int u) {
+  const int64_t n = rows * 4 * u;
+  const unsigned grid = (unsigned)((n + 255) / 256);
+  if (dtype == HBP_F32)
+    lstm_operand_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)g, (const float*)c5, (const float*)fg,
+                                                            (const float*)delta, (float*)a4, (float*)uo, rows, u);
+  else
+    lstm_operand_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)g, (const bf16*)c5, (const bf16*)fg,
+                                                           (const bf16*)delta, (bf16*)a4, (bf16*)uo, rows, u);
+  lc.count();
+  lc.check();
+}
+
+void lstm_split(Launcher& lc, const float* g, const float* c5, const float* fg, const float* delta, float* hi, float* lo,
+                float* uo, int64_t rows, int u) {
+  const int64_t n = rows * 4 * u;
+  lstm_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, lc.stream>>>(g, c5, fg, delta, hi, lo, uo, rows, u);
+  lc.count();
+  lc.check();
+}
+
+void lstm_split_transposed(Launcher& lc, const float* g, const float* c5, float* hiT, float* loT, int64_t rows, int u) {
+  dim3 grid((unsigned)((rows + 31) / 32), (unsigned)((4 * u + 31) / 32));
+  lstm_split_transposed_kernel<<<grid, 256, 0, lc.stream>>>(g, c5, hiT, loT, rows, u);
+  lc.count();
+  lc.check();
+}
+
+}  // namespace hbp

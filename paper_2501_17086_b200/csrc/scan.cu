@@ -495,7 +495,7 @@ __global__ void split_tf32_kernel(const float4* __restrict__ a, const float4* __
 }
 __global__ void __launch_bounds__(256) split_tf32_transposed_kernel(const float* __restrict__ a, const float* __restrict__ b,
                                                                     float* __restrict__ hiT, float* __restrict__ loT,
-                                                                    int64_t rows, int cols) {
+                                                                    int64_t rows, int cols, int64_t ld) {
   __shared__ float th[32][33], tl[32][33];
   const int64_t r0 = (int64_t)blockIdx.x * 32;
   const int c0 = blockIdx.y * 32;
@@ -505,8 +505,8 @@ __global__ void __launch_bounds__(256) split_tf32_transposed_kernel(const float*
     const int c = c0 + tx;
     float v = 0.0f;
     if (r < rows && c < cols) {
-      v = a[r * cols + c];
-      if (b) v *= b[r * cols + c];
+      v = a[r * ld + c];
+      if (b) v *= b[r * ld + c];
     }
     const float h = round_tf32(v);
     th[i][tx] = h;
@@ -659,9 +659,10 @@ void split_tf32(Launcher& lc, const float* a, const float* b, float* hi, float* 
   lc.check();
 }
 
-void split_tf32_transposed(Launcher& lc, const float* a, const float* b, float* hiT, float* loT, int64_t rows, int cols) {
+void split_tf32_transposed(Launcher& lc, const float* a, const float* b, float* hiT, float* loT, int64_t rows, int cols,
+                           int64_t ld) {
   dim3 grid((unsigned)((rows + 31) / 32), (unsigned)((cols + 31) / 32));
-  split_tf32_transposed_kernel<<<grid, 256, 0, lc.stream>>>(a, b, hiT, loT, rows, cols);
+  split_tf32_transposed_kernel<<<grid, 256, 0, lc.stream>>>(a, b, hiT, loT, rows, cols, ld > 0 ? ld : cols);
   lc.count();
   lc.check();
 }

@@ -11,14 +11,14 @@ from .workloads import Workload
 def params_for(w: Workload, inputs: dict) -> dict:
     if w.block == "rnn_tanh":
         return {"W": inputs["W"], "U": inputs["U"], "a": inputs["a"]}
-    if w.block == "gru":
+    if w.block in ("gru", "lstm"):
         return {"W": inputs["W"], "U": inputs["U"]}
     names = ("W1", "W2") if w.block != "preln_transformer" else ("Wq", "Wk", "Wv", "Wo", "W1", "W2")
     return {n: inputs[n] for n in names}
 
 
 def rnn_inputs(w: Workload, inputs: dict):
-    return inputs["X"] if w.block in ("rnn_tanh", "gru") else None
+    return inputs["X"] if w.block in ("rnn_tanh", "gru", "lstm") else None
 
 
 def loss_delta(w: Workload, x_all: torch.Tensor, inputs: dict) -> torch.Tensor:

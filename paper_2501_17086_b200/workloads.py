@@ -24,7 +24,7 @@ import torch
 @dataclasses.dataclass(frozen=True)
 class Workload:
     name: str
-    block: str            # "mlp" | "preln_mlp" | "rnn_tanh" | "preln_transformer" | "gru"
+    block: str            # "mlp" | "preln_mlp" | "rnn_tanh" | "preln_transformer" | "gru" | "lstm"
     dtype: str            # "f32" | "bf16"
     L: int                # residual steps (mlp), time steps (rnn), decoder blocks (transformer)
     d: int
@@ -62,6 +62,8 @@ WORKLOADS = {
     # pixels); the input widths 210 and 3 are rounded up to multiples of 4 for 128-bit access
     "g1": Workload("g1", "gru", "f32", L=256, d=512, in_dim=212, batch=128, tokens=128, seed=1006, loss="every_mse"),
     "g2": Workload("g2", "gru", "f32", L=1024, d=64, in_dim=4, batch=128, tokens=128, seed=1007, loss="every_mse"),
+    # LSTM in the shape of the paper's character-level experiment: 256 steps, 512 units (state [c, h] 1024 wide)
+    "l1": Workload("l1", "lstm", "f32", L=256, d=1024, hidden=512, in_dim=212, batch=128, tokens=128, seed=1008, loss="every_mse"),
     # c2 with 8 layers: same per-launch tile shapes, small enough for multi-pass profiler captures
     "c2_small": Workload("c2_small", "preln_mlp", "bf16", L=8, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1012),
     # c4 with 4 decoder blocks: same per-launch shapes, small enough for multi-pass profiler captures
@@ -77,6 +79,11 @@ WORKLOADS = {
                               loss="every_mse"),
     "gru_twin_bf16": Workload("gru_twin_bf16", "gru", "bf16", L=24, d=64, in_dim=16, batch=6, tokens=6, seed=2026,
                               loss="every_mse"),
+    "lstm_twin": Workload("lstm_twin", "lstm", "f32", L=40, d=72, hidden=36, in_dim=12, batch=5, tokens=5, seed=2007, loss="every_mse"),
+    "lstm_twin_long": Workload("lstm_twin_long", "lstm", "f32", L=300, d=64, hidden=32, in_dim=4, batch=12, tokens=12, seed=2017,
+                               loss="every_mse"),
+    "lstm_twin_bf16": Workload("lstm_twin_bf16", "lstm", "bf16", L=24, d=64, hidden=32, in_dim=16, batch=6, tokens=6, seed=2027,
+                               loss="every_mse"),
     "c4_twin": Workload("c4_twin", "preln_transformer", "bf16", L=2, d=128, hidden=512, n_heads=2, head_dim=64,
                         seq=200, batch=2, tokens=400, seed=2004),
     "c4_twin_f32": Workload("c4_twin_f32", "preln_transformer", "f32", L=2, d=64, hidden=128, n_heads=2, head_dim=32,
@@ -95,6 +102,8 @@ def make_inputs(cfg: Workload, device="cpu"):
     Keys: mlp / preln_mlp: W1 [L,h,d], W2 [L,d,h], x0 [N,d], y [N,d].
     rnn_tanh: a [d], W [d,d], U [d,in], X [T,B,in], Y [T,B,d], x0 [B,d] (zeros).
     gru: W [3d,d] (variance 1/d), U [3d,in] (variance 1/in), X, Y, x0 as for rnn_tanh.
+    lstm: W [4u,u] (variance 1/u), U [4u,in] (variance 1/in) with u = hidden units, d = 2u; X [T,B,in], Y [T,B,2u],
+    x0 [B,2u] (zeros).
     preln_transformer: Wq, Wk, Wv, Wo [L,d,d], W1 [L,h,d], W2 [L,d,h], x0 [N,d], y [N,d].
     Standard deviations: 0.02 for Transformer-style inputs weights and
     0.02 / sqrt(2 * steps) for the weights that write into the residual stream;
@@ -133,6 +142,13 @@ def make_inputs(cfg: Workload, device="cpu"):
         T, d, B, nin = cfg.L, cfg.d, cfg.batch, cfg.in_dim
         out["W"] = _randn(gen, (3 * d, d), 1.0 / math.sqrt(d), dev).to(dt)
         out["U"] = _randn(gen, (3 * d, nin), 1.0 / math.sqrt(nin), dev).to(dt)
+        out["X"] = _randn(gen, (T, B, nin), 1.0, dev).to(dt)
+        out["Y"] = _randn(gen, (T, B, d), 1.0, dev).to(dt)
+        out["x0"] = torch.zeros((B, d), device=dev, dtype=dt)
+    elif cfg.block == "lstm":
+        T, d, u, B, nin = cfg.L, cfg.d, cfg.hidden, cfg.batch, cfg.in_dim
+        out["W"] = _randn(gen, (4 * u, u), 1.0 / math.sqrt(u), dev).to(dt)
+        out["U"] = _randn(gen, (4 * u, nin), 1.0 / math.sqrt(nin), dev).to(dt)
         out["X"] = _randn(gen, (T, B, nin), 1.0, dev).to(dt)
         out["Y"] = _randn(gen, (T, B, d), 1.0, dev).to(dt)
         out["x0"] = torch.zeros((B, d), device=dev, dtype=dt)

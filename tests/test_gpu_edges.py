@@ -173,7 +173,7 @@ def test_gamma_shifted_split_matches_oracle(name, gamma):
         assert rel(np64(grads["d" + n]), v) < tol, n
 
 
-@pytest.mark.parametrize("name,ks", [("gru_twin", (1, 3)), ("c3_twin", (2,)), ("c2_twin", (2,)), ("c4_twin", (2,))])
+@pytest.mark.parametrize("name,ks", [("gru_twin", (1, 3)), ("lstm_twin", (1, 3)), ("c3_twin", (2,)), ("c2_twin", (2,)), ("c4_twin", (2,))])
 def test_cuda_core_fallback_matches_oracle(name, ks, monkeypatch):
     """HBP_FORCE_SIMT=1 (read when a context is made) keeps every GEMM and the attention backward off the
     tensor cores: the fallback kernels must meet the same bar."""

@@ -72,6 +72,9 @@ def compare(w, gpu, ref, ks, grads_for):
     ("gru_twin", (0, 1, 2, 4, 8, 40)),
     ("gru_twin_long", (0, 1, 3)),
     ("gru_twin_bf16", (1, 2, 4)),
+    ("lstm_twin", (0, 1, 2, 4, 8, 40)),
+    ("lstm_twin_long", (0, 1, 3)),
+    ("lstm_twin_bf16", (1, 2, 4)),
 ])
 def test_twin_matches_oracle_in_full(name, ks):
     w = WORKLOADS[name]
