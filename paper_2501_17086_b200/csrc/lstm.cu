@@ -109,13 +109,25 @@ __device__ __forceinline__ double as_d(float v) { return (double)v; }
 __device__ __forceinline__ double as_d(bf16 v) { return (double)to_f(v); }
 
 // element (row, column k of the [4u] operand) from the upstream gradient [g_c | g_h] and the coefficients
-template <typename T, typename G>
-__device__ __forceinline__ double operand_value(const G* __restrict__ g_row, const T* __restrict__ c5_row, int u, int k) {
+// (C = the type to compute in: double for exact backpropagation, float for GEMM operands)
+template <typename C, typename T, typename G>
+__device__ __forceinline__ C operand_value(const G* __restrict__ g_row, const T* __restrict__ c5_row, int u, int k) {
   const int q = k / u, n = k - q * u;
-  const double gh = as_d(g_row[u + n]);
-  if (q == 3) return gh * (double)to_f(c5_row[3 * u + n]);
-  const double t = as_d(g_row[n]) + gh * (double)to_f(c5_row[4 * u + n]);
-  return t * (double)to_f(c5_row[q * u + n]);
+  const C gh = (C)as_d(g_row[u + n]);
+  if (q == 3) return gh * (C)to_f(c5_row[3 * u + n]);
+  const C t = (C)as_d(g_row[n]) + gh * (C)to_f(c5_row[4 * u + n]);
+  return t * (C)to_f(c5_row[q * u + n]);
+}
+
+// the four operand values of (row, unit n) at once
+template <typename T>
+__device__ __forceinline__ void operand_quad(const T* __restrict__ g_row, const T* __restrict__ c5_row, int u, int n, float* v) {
+  const float gh = to_f(g_row[u + n]);
+  const float t = to_f(g_row[n]) + gh * to_f(c5_row[4 * u + n]);
+  v[0] = t * to_f(c5_row[n]);
+  v[1] = t * to_f(c5_row[u + n]);
+  v[2] = t * to_f(c5_row[2 * u + n]);
+  v[3] = gh * to_f(c5_row[3 * u + n]);
 }
 
 // Exact backpropagation through one step in double: g_t = delta_t + [f * g_c, 0] + [u_c, u_h].
@@ -132,7 +144,7 @@ __global__ void __launch_bounds__(256) lstm_bwd_step_kernel(const T* __restrict_
   for (int k0 = 0; k0 < 4 * u; k0 += kTile) {  // u is a multiple of 4, not of the tile: blocks may straddle gates
     for (int i = ty; i < kTile; i += 8) {
       const int m = m0 + i, k = k0 + tx;
-      Hs[i][tx] = (m < B && k < 4 * u) ? operand_value<T, double>(g_in + (int64_t)m * 2 * u, c5 + (int64_t)m * 5 * u, u, k) : 0.0;
+      Hs[i][tx] = (m < B && k < 4 * u) ? operand_value<double, T, double>(g_in + (int64_t)m * 2 * u, c5 + (int64_t)m * 5 * u, u, k) : 0.0;
       const int kk = k0 + i, n = n0 + tx;  // W[k][n]: contiguous in n
       Ws[tx][i] = (kk < 4 * u && n < u) ? to_f(W[(int64_t)kk * u + n]) : 0.0f;
     }
@@ -172,34 +184,41 @@ __device__ __forceinline__ void write_uc(const T* g_row, const T* c5_row, const 
   uo_row[n] = from_f<T>(v);
 }
 
-// a4[row][k] = operand (in dtype) for the GEMMs that do not take the tf32 splits; optionally the u_c half
+// a4[row][k] = operand (in dtype) for the GEMMs that do not take the tf32 splits; optionally the u_c half.
+// One block row per row of the operand, one thread per unit (its four columns are u apart).
 template <typename T>
-__global__ void lstm_operand_kernel(const T* __restrict__ g, const T* __restrict__ c5, const T* __restrict__ fg,
-                                    const T* __restrict__ delta, T* __restrict__ a4, T* __restrict__ uo, int64_t rows,
-                                    int u) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= rows * 4 * u) return;
-  const int64_t row = i / (4 * u);
-  const int k = (int)(i - row * 4 * u);
+__global__ void __launch_bounds__(256) lstm_operand_kernel(const T* __restrict__ g, const T* __restrict__ c5,
+                                                           const T* __restrict__ fg, const T* __restrict__ delta,
+                                                           T* __restrict__ a4, T* __restrict__ uo, int u) {
+  const int64_t row = blockIdx.x;
+  const int n = blockIdx.y * blockDim.x + threadIdx.x;
+  if (n >= u) return;
   const T* g_row = g + row * 2 * u;
-  a4[i] = from_f<T>((float)operand_value<T, T>(g_row, c5 + row * 5 * u, u, k));
-  if (uo && k < u) write_uc<T>(g_row, c5 + row * 5 * u, fg + row * 2 * u, delta ? delta + row * 2 * u : nullptr, uo + row * 2 * u, u, k);
+  float v[4];
+  operand_quad<T>(g_row, c5 + row * 5 * u, u, n, v);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) a4[row * 4 * u + q * u + n] = from_f<T>(v[q]);
+  if (uo) write_uc<T>(g_row, c5 + row * 5 * u, fg + row * 2 * u, delta ? delta + row * 2 * u : nullptr, uo + row * 2 * u, u, n);
 }
 
 // tf32 split of the operand as [rows][4u]; optionally the u_c half (float data)
-__global__ void lstm_split_kernel(const float* __restrict__ g, const float* __restrict__ c5, const float* __restrict__ fg,
-                                  const float* __restrict__ delta, float* __restrict__ hi, float* __restrict__ lo,
-                                  float* __restrict__ uo, int64_t rows, int u) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= rows * 4 * u) return;
-  const int64_t row = i / (4 * u);
-  const int k = (int)(i - row * 4 * u);
+__global__ void __launch_bounds__(256) lstm_split_kernel(const float* __restrict__ g, const float* __restrict__ c5,
+                                                         const float* __restrict__ fg, const float* __restrict__ delta,
+                                                         float* __restrict__ hi, float* __restrict__ lo,
+                                                         float* __restrict__ uo, int u) {
+  const int64_t row = blockIdx.x;
+  const int n = blockIdx.y * blockDim.x + threadIdx.x;
+  if (n >= u) return;
   const float* g_row = g + row * 2 * u;
-  const float v = (float)operand_value<float, float>(g_row, c5 + row * 5 * u, u, k);
-  const float h = round_tf32(v);
-  hi[i] = h;
-  lo[i] = round_tf32(v - h);
-  if (uo && k < u) write_uc<float>(g_row, c5 + row * 5 * u, fg + row * 2 * u, delta ? delta + row * 2 * u : nullptr, uo + row * 2 * u, u, k);
+  float v[4];
+  operand_quad<float>(g_row, c5 + row * 5 * u, u, n, v);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float h = round_tf32(v[q]);
+    hi[row * 4 * u + q * u + n] = h;
+    lo[row * 4 * u + q * u + n] = round_tf32(v[q] - h);
+  }
+  if (uo) write_uc<float>(g_row, c5 + row * 5 * u, fg + row * 2 * u, delta ? delta + row * 2 * u : nullptr, uo + row * 2 * u, u, n);
 }
 
 // the same operand written transposed, [4u][rows] (the weight-gradient GEMMs contract over rows)
@@ -214,7 +233,7 @@ __global__ void __launch_bounds__(256) lstm_split_transposed_kernel(const float*
     const int64_t r = r0 + i;
     const int c = c0 + tx;
     float v = 0.0f;
-    if (r < rows && c < 4 * u) v = (float)operand_value<float, float>(g + r * 2 * u, c5 + r * 5 * u, u, c);
+    if (r < rows && c < 4 * u) v = operand_value<float, float, float>(g + r * 2 * u, c5 + r * 5 * u, u, c);
     const float h = round_tf32(v);
     th[i][tx] = h;
     tl[i][tx] = round_tf32(v - h);
@@ -260,22 +279,21 @@ void lstm_backward_step(Launcher& lc, int dtype, const void* W, const void* fg, 
 
 void lstm_operand(Launcher& lc, int dtype, const void* g, const void* c5, const void* fg, const void* delta, void* a4,
                   void* uo, int64_t rows, int u) {
-  const int64_t n = rows * 4 * u;
-  const unsigned grid = (unsigned)((n + 255) / 256);
+  dim3 grid((unsigned)rows, (unsigned)((u + 255) / 256));
   if (dtype == HBP_F32)
     lstm_operand_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)g, (const float*)c5, (const float*)fg,
-                                                            (const float*)delta, (float*)a4, (float*)uo, rows, u);
+                                                            (const float*)delta, (float*)a4, (float*)uo, u);
   else
     lstm_operand_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)g, (const bf16*)c5, (const bf16*)fg,
-                                                           (const bf16*)delta, (bf16*)a4, (bf16*)uo, rows, u);
+                                                           (const bf16*)delta, (bf16*)a4, (bf16*)uo, u);
   lc.count();
   lc.check();
 }
 
 void lstm_split(Launcher& lc, const float* g, const float* c5, const float* fg, const float* delta, float* hi, float* lo,
                 float* uo, int64_t rows, int u) {
-  const int64_t n = rows * 4 * u;
-  lstm_split_kernel<<<(unsigned)((n + 255) / 256), 256, 0, lc.stream>>>(g, c5, fg, delta, hi, lo, uo, rows, u);
+  dim3 grid((unsigned)rows, (unsigned)((u + 255) / 256));
+  lstm_split_kernel<<<grid, 256, 0, lc.stream>>>(g, c5, fg, delta, hi, lo, uo, u);
   lc.count();
   lc.check();
 }
