@@ -1,0 +1,49 @@
+"""Seeded random shapes through the C ABI against the oracle: widths, hidden sizes, token counts and depths that are
+not multiples of any tile (only of the 16-byte vector), for every block kind and both dtypes.  Each case is small
+enough for the oracle to run in full."""
+import dataclasses
+import random
+
+import pytest
+
+from oracle import run as orun
+from paper_2501_17086_b200.workloads import Workload, make_inputs
+from test_gpu_parity import compare, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(seed):
+    rnd = random.Random(seed)
+    dtype = rnd.choice(["f32", "bf16"])
+    v = 4 if dtype == "f32" else 8
+    block = rnd.choice(["mlp", "preln_mlp", "rnn_tanh", "gru", "lstm", "preln_transformer"])
+    mult = lambda lo, hi: v * rnd.randint(max(1, lo // v), hi // v)
+    if block in ("mlp", "preln_mlp"):
+        return Workload(f"rand{seed}", block, dtype, L=rnd.randint(1, 6), d=mult(8, 328), hidden=mult(8, 520),
+                        tokens=rnd.randint(1, 300), batch=1, seq=1, seed=5000 + seed,
+                        loss=rnd.choice(["final_mse", "final_half_sse"]))
+    if block == "preln_transformer":
+        heads, hd = rnd.randint(1, 3), rnd.choice([32, 64]) if dtype == "f32" else 64
+        batch, seq = rnd.randint(1, 3), rnd.randint(1, 210)
+        return Workload(f"rand{seed}", block, dtype, L=rnd.randint(1, 2), d=heads * hd, hidden=mult(8, 260), n_heads=heads,
+                        head_dim=hd, seq=seq, batch=batch, tokens=batch * seq, seed=5000 + seed)
+    T, B, nin = rnd.randint(1, 150), rnd.randint(1, 40), mult(8, 40)
+    if block == "lstm":
+        u = mult(8, 100)
+        return Workload(f"rand{seed}", block, dtype, L=T, d=2 * u, hidden=u, in_dim=nin, batch=B, tokens=B,
+                        seed=5000 + seed, loss="every_mse")
+    return Workload(f"rand{seed}", block, dtype, L=T, d=mult(8, 200), in_dim=nin, batch=B, tokens=B, seed=5000 + seed,
+                    loss="every_mse")
+
+
+@pytest.mark.parametrize("seed", range(36))
+def test_random_shape_matches_oracle(seed):
+    w = _case(seed)
+    rnd = random.Random(1000 + seed)
+    ks = tuple(sorted({0, rnd.randint(1, 3), rnd.randint(1, max(1, min(w.steps, 6)))}))
+    inp = make_inputs(w, "cuda")
+    gpu = run_gpu(w, inp, ks)
+    kmax = max(ks)
+    ref = orun.run(w, inp, ks=ks, grads_for=("exact", kmax))
+    compare(w, gpu, ref, ks, ("exact", kmax))
