@@ -274,6 +274,31 @@ class LSTMStep:
         return {"W": pre.T @ k["h"], "U": pre.T @ _f64(self.x_t)}
 
 
+class ReluResStep:
+    """ResNet-style layer f(x) = ReLU(x + Block(x)) (Table 1, row "ResNet": g = Block, r(x, z) = ReLU(x + z)).
+    dr/dx = dr/dz = diag(mask) with mask = [x + Block(x) > 0], so K = diag(mask) depends on the state and
+    J = diag(mask) J_Block.  `inner` is the block (an MLPStep)."""
+
+    def __init__(self, inner):
+        self.inner = inner
+
+    def forward(self, x):
+        z, cache = self.inner.forward(x)
+        mask = (x + z > 0.0).astype(np.float64)
+        cache = dict(cache)
+        cache["mask"] = mask
+        return mask * z, cache            # r(x, z) = mask * x + mask * z: the gate carries the first term
+
+    def gate(self, cache):
+        return cache["mask"]
+
+    def vjp(self, cache, g):
+        return self.inner.vjp(cache, cache["mask"] * g)
+
+    def param_vjp(self, cache, g):
+        return self.inner.param_vjp(cache, cache["mask"] * g)
+
+
 class ShiftedStep:
     """The gamma-shifted split of a residual layer x + Block(x) (Appendix C.3, Eq. 17): the block becomes
     g(x) = Block(x) + gamma x and the residual function r(x, z) = (1 - gamma) x + z, so the layer itself is
@@ -342,6 +367,11 @@ def gru_stack(W, U, X):
 def lstm_stack(W, U, X):
     """LSTM over time on the state [c, h]; X is [T, B, in]."""
     return Stack([LSTMStep(W, U, _Lazy(X, t)) for t in range(len(X))])
+
+
+def relu_mlp_stack(W1, W2):
+    """L layers x <- ReLU(x + W2 gelu(W1 x))."""
+    return Stack([ReluResStep(s) for s in mlp_stack(W1, W2, False, 0.0).steps])
 
 
 def rnn_stack(W, U, a, X):

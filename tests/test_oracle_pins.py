@@ -629,3 +629,45 @@ def test_lstm_path_sums_and_exactness():
     g = O.exact_bp(st, caches, deltas)
     for a, b in zip(O.highway_bp(st, caches, deltas, T), g):
         np.testing.assert_allclose(a, b, rtol=1e-11, atol=1e-12)
+
+
+# ---------------------------------------------- 14. ReLU(x + Block(x)): a 0/1 gate that depends on the state (Table 1)
+def test_relu_residual_matches_autograd_and_path_sums():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(61)
+    L, d, h, N = 4, 3, 5, 2
+    W1 = rng.normal(size=(L, h, d)) * 0.8
+    W2 = rng.normal(size=(L, d, h)) * 0.8
+    st = O.relu_mlp_stack(W1, W2)
+    x0 = rng.normal(size=(N, d))
+    xs, caches = O.forward(st, x0)
+    # the plain definition with the library's ops
+    xt = torch.tensor(x0, requires_grad=True)
+    x = xt
+    for l in range(L):
+        x = torch.relu(x + torch.nn.functional.gelu(x @ torch.tensor(W1[l]).T) @ torch.tensor(W2[l]).T)
+        np.testing.assert_allclose(xs[l + 1], x.detach().numpy(), rtol=1e-12, atol=1e-13)
+    assert 0.05 < np.mean([c["mask"].mean() for c in caches]) < 0.95      # both branches of the ReLU occur
+    y = rng.normal(size=(N, d))
+    (0.5 * ((x - torch.tensor(y)) ** 2).sum()).backward()
+    deltas = [np.zeros_like(x0) for _ in range(L)] + [xs[L] - y]
+    g = O.exact_bp(st, caches, deltas)
+    np.testing.assert_allclose(g[0], xt.grad.numpy(), rtol=1e-10, atol=1e-12)
+    for a, b in zip(O.highway_bp(st, caches, deltas, L), g):
+        np.testing.assert_allclose(a, b, rtol=1e-11, atol=1e-12)
+    # path sums with K = diag(mask), J = diag(mask) J_block (J_block by finite differences of the block alone)
+    one = O.relu_mlp_stack(W1, W2)
+    xs1, c1 = O.forward(one, x0[:1])
+    d1 = [rng.normal(size=(1, d)) for _ in range(L + 1)]
+    J, K = [None], [None]
+    for l in range(L):
+        blk = lambda v, l=l: one.steps[l].inner.forward(v.reshape(1, d))[0].reshape(-1)
+        Jb = O.finite_difference_jacobian(blk, xs1[l].reshape(-1), h=1e-5)
+        M = np.diag(c1[l]["mask"].reshape(-1))
+        K.append(M)
+        J.append(M @ Jb)
+    flat = [v.reshape(-1) for v in d1]
+    for k in range(L + 1):
+        w = O.highway_bp(one, c1, d1, k)
+        for i in range(L + 1):
+            np.testing.assert_allclose(w[i].reshape(-1), O.path_sum(flat, J, K, i, k), rtol=1e-6, atol=1e-8)
