@@ -31,6 +31,10 @@ __device__ __forceinline__ void epilogue_store(const GemmArgs& g, int b, int m, 
       float gate = g.gate ? to_f(((const T*)g.gate)[b * g.gate_sb + n]) : 1.0f;
       float r = g.R ? g.R[(int64_t)m * g.N + n] : to_f(((const T*)g.E)[b * g.e_sb + (int64_t)m * g.lde + n]);
       float v = gate * r + acc;
+      if (g.relu) {
+        ((T*)g.D2)[b * g.d2_sb + (int64_t)m * g.ldd2 + n] = from_f<T>(v > 0.0f ? 1.0f : 0.0f);
+        v = fmaxf(v, 0.0f);
+      }
       if (g.R) g.R[(int64_t)m * g.N + n] = v;
       ((T*)g.D)[b * g.d_sb + dn] = from_f<T>(v);
     } break;

@@ -13,7 +13,7 @@ bool g_force_simt = false;
 bool g_gemm_pair = false;
 
 bool gemm(Launcher& lc, const GemmArgs& g, int* status_word) {
-  if (!g_force_simt && gemm_tc(lc, g, status_word)) return true;
+  if (!g_force_simt && !g.relu && gemm_tc(lc, g, status_word)) return true;
   gemm_simt(lc, g);
   return false;
 }
@@ -65,6 +65,8 @@ struct hbp_ctx {
   char *Zc = nullptr, *C4 = nullptr, *A4 = nullptr;
   // LSTM (u = d / 2 units): the scan's gate [T][B][2u] = [f | 0], the VJP coefficients [T*B][5u] (A4 is [T*B][4u])
   char *Fg = nullptr, *C5 = nullptr;
+  // ReLU(x + Block(x)): the masks [L][N][d] (0/1 in dtype: the scan's gate) and mask * g_{l+1} [L][N][d]
+  char *MASK = nullptr, *GM = nullptr;
   char* scan_scratch = nullptr;
   size_t scan_scratch_bytes = 0;
   float* partial = nullptr;  // split-K / gate-gradient partial sums
@@ -91,7 +93,7 @@ inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 hbp_status check_config(const hbp_config* c) {
   if (!c) return HBP_ERR_INVALID_ARG;
   if (c->dtype != HBP_F32 && c->dtype != HBP_BF16) return HBP_ERR_DTYPE;
-  if (c->block < 0 || c->block > HBP_BLOCK_LSTM) return HBP_ERR_UNSUPPORTED;
+  if (c->block < 0 || c->block > HBP_BLOCK_RELU_MLP) return HBP_ERR_UNSUPPORTED;
   if (c->gate < 0 || c->gate > HBP_GATE_CHANNEL_PER_STEP) return HBP_ERR_UNSUPPORTED;
   if (c->loss != HBP_LOSS_FINAL && c->loss != HBP_LOSS_EVERY_STEP) return HBP_ERR_UNSUPPORTED;
   const int v = c->dtype == HBP_F32 ? 4 : 8;
@@ -101,7 +103,10 @@ hbp_status check_config(const hbp_config* c) {
   if (c->d % v) return HBP_ERR_SHAPE;
   if (c->d / v > 1024) return HBP_ERR_SHAPE;  // one block per row in the LayerNorm kernels
   const bool gated_cell = c->block == HBP_BLOCK_GRU || c->block == HBP_BLOCK_LSTM;
-  if (gated_cell && (c->gate != HBP_GATE_ONE || c->gamma != 0.0f)) return HBP_ERR_UNSUPPORTED;
+  if ((gated_cell || c->block == HBP_BLOCK_RELU_MLP) && (c->gate != HBP_GATE_ONE || c->gamma != 0.0f)) return HBP_ERR_UNSUPPORTED;
+  // the 0/1 mask is a sign decision: taken in bf16 arithmetic it differs from an exact evaluation on the elements
+  // that land near zero, and each such element changes its whole gradient path; float only
+  if (c->block == HBP_BLOCK_RELU_MLP && c->dtype != HBP_F32) return HBP_ERR_UNSUPPORTED;
   if (c->block == HBP_BLOCK_LSTM && (c->hidden <= 0 || c->hidden % v || 2 * c->hidden != c->d)) return HBP_ERR_SHAPE;
   if (c->block == HBP_BLOCK_RNN_TANH || gated_cell) {
     if (c->in_dim <= 0 || c->in_dim % v) return HBP_ERR_SHAPE;
@@ -194,6 +199,10 @@ size_t carve(hbp_ctx* c, char* base) {
         c->lnstat = (float4*)take(steps * N * sizeof(float4));
       }
     }
+    if (f.block == HBP_BLOCK_RELU_MLP) {
+      c->MASK = take(steps * N * d * es);
+      c->GM = take(steps * N * d * es);
+    }
     c->ACT = take((size_t)c->layers * N * h * es);
     c->DACT = take((size_t)c->layers * N * h * es);
     const size_t per_layer = N * h * es;
@@ -275,13 +284,25 @@ struct Run {
     b.stats_sb = (int64_t)ss * N * c->ln_slots;
   }
 
+  // What the MLP block of layer b0 is differentiated against: g_{l+1}, or mask_l * g_{l+1} for ReLU(x + Block(x))
+  // (mask_gradients fills GM first).
+  const char* upstream(int b0) const {
+    if (c->GM) return at(c->GM, (int64_t)b0 * state);
+    return at(g, (int64_t)(mlp_step(b0) + 1) * state);
+  }
+  void mask_gradients(int b0, int b1) {
+    if (!c->GM) return;
+    mul_elementwise(lc, c->cfg.dtype, at(c->GM, (int64_t)b0 * state), at(c->MASK, (int64_t)b0 * state),
+                    at(g, (int64_t)(b0 + 1) * state), (int64_t)(b1 - b0) * state);
+  }
+
   // ---- MLP block: u = J^T g for layers [b0, b1) (b1 - b0 <= group), from states g[step+1] -------
   // dA = G W2, dZ = dA * gelu'(Z) -> H1 (cached derivative);  dY = dZ W1 -> U[step].
   void mlp_vjp(int b0, int b1, bool want_dy) {
     const int nb = b1 - b0, ss = step_stride();
     GemmArgs a = base_args();
     a.M = (int)N; a.N = (int)h; a.K = (int)d; a.batch = nb;
-    a.A = at(g, (int64_t)(mlp_step(b0) + 1) * state); a.a_sm = d; a.a_sk = 1; a.a_sb = ss * state;
+    a.A = upstream(b0); a.a_sm = d; a.a_sk = 1; a.a_sb = ss * state;
     a.B = at(p->W2, (int64_t)b0 * d * h); a.b_sn = 1; a.b_sk = h; a.b_sb = d * h;
     a.epi = EPI_MUL;
     a.E = at(c->DACT, (int64_t)b0 * N * h); a.lde = h; a.e_sb = N * h;
@@ -303,7 +324,7 @@ struct Run {
     const int nb = b1 - b0, ss = step_stride();
     GemmArgs a = base_args();
     a.M = (int)d; a.N = (int)h; a.K = (int)N; a.batch = nb;
-    a.A = at(g, (int64_t)(mlp_step(b0) + 1) * state); a.a_sm = 1; a.a_sk = d; a.a_sb = ss * state;
+    a.A = upstream(b0); a.a_sm = 1; a.a_sk = d; a.a_sb = ss * state;
     a.B = at(c->ACT, (int64_t)b0 * N * h); a.b_sn = 1; a.b_sk = h; a.b_sb = N * h;
     a.epi = EPI_STORE; a.d_f32 = true;
     a.D = gr->dW2 + (int64_t)b0 * d * h; a.ldd = h; a.d_sb = d * h;
@@ -559,6 +580,7 @@ struct Run {
       case HBP_BLOCK_GRU: gru_vjp_all(); break;
       case HBP_BLOCK_LSTM: lstm_vjp_all(); break;
       default:
+        mask_gradients(0, layers);
         for (int b0 = 0; b0 < layers; b0 += grp) mlp_vjp(b0, b0 + grp < layers ? b0 + grp : layers, true);
         if (c->cfg.block == HBP_BLOCK_PRELN_TRANSFORMER) attn_vjp(0, layers, true);
     }
@@ -570,6 +592,7 @@ struct Run {
       case HBP_BLOCK_GRU: gru_wgrad(gr); break;
       case HBP_BLOCK_LSTM: lstm_wgrad(gr); break;
       default:
+        mask_gradients(0, layers);
         for (int b0 = 0; b0 < layers; b0 += grp) {
           const int b1 = b0 + grp < layers ? b0 + grp : layers;
           mlp_vjp(b0, b1, false);
@@ -615,6 +638,7 @@ struct Run {
     s.a = p->a; s.gate = c->cfg.gate;
     if (c->cfg.block == HBP_BLOCK_GRU) { s.a = c->Zc; s.gate = kGateElement; }
     if (c->cfg.block == HBP_BLOCK_LSTM) { s.a = c->Fg; s.gate = kGateElement; }
+    if (c->cfg.block == HBP_BLOCK_RELU_MLP) { s.a = c->MASK; s.gate = kGateElement; }
     s.g = g;
     if (with_u && c->preln) {
       s.xhat = c->Y; s.rstd = c->rstd;
@@ -867,6 +891,7 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
       if (ctx->xres) a.R = ctx->xres;
       else { a.E = r.at(xa, (int64_t)step * state); a.lde = d; }
       a.D = r.at(xa, (int64_t)(step + 1) * state); a.ldd = d;
+      if (ctx->MASK) { a.relu = true; a.D2 = r.at(ctx->MASK, (int64_t)step * state); a.ldd2 = d; }
     };
     auto ln_of = [&](int step) {
       const void* src = ctx->xres ? (const void*)ctx->xres : (const void*)r.at(xa, (int64_t)step * state);
@@ -1004,6 +1029,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
         const int b = tr ? l / 2 : l;
         const bool is_mlp = !tr || (l % 2 == 1);
         if (is_mlp) {
+          r.mask_gradients(b, b + 1);
           r.mlp_vjp(b, b + 1, true);
           if (grads) r.mlp_wgrad(b, b + 1, grads);
         } else {
@@ -1073,7 +1099,7 @@ hbp_status hbp_add_carry(hbp_ctx* ctx, const void* carry, void* g_all, void* cud
   if (!ctx || !carry || !g_all) return HBP_ERR_INVALID_ARG;
   if (misaligned(carry) || misaligned(g_all)) return HBP_ERR_SHAPE;
   if (ctx->cfg.gate != HBP_GATE_ONE || ctx->cfg.gamma != 0.0f || ctx->cfg.block == HBP_BLOCK_GRU ||
-      ctx->cfg.block == HBP_BLOCK_LSTM)
+      ctx->cfg.block == HBP_BLOCK_LSTM || ctx->cfg.block == HBP_BLOCK_RELU_MLP)
     return HBP_ERR_UNSUPPORTED;
   Launcher lc;
   lc.stream = (cudaStream_t)cuda_stream;

@@ -45,6 +45,7 @@ struct GemmArgs {
   const void* gate = nullptr;  // [N] per batch entry (stride gate_sb), nullptr = ones
   int64_t gate_sb = 0;
   float* R = nullptr;  // fp32 master copy of the residual stream [M][N], leading dim N
+  bool relu = false;   // EPI_RESID on the CUDA-core kernel only: v = max(v, 0) and D2[m,n] = (v > 0) as 0/1 (the mask that gates this step)
   float2* stats = nullptr;  // EPI_STORE_LN: [batch][M][stats_slots] partial sums; batch stride stats_sb (in float2)
   int64_t stats_sb = 0;
   // float operands for the tensor cores: each of A (after the A2 product) and B split into a tf32-exact
@@ -128,6 +129,8 @@ bool scan_ring(Launcher& lc, const ScanArgs& s);
 void ln_stats_finish(Launcher& lc, const float2* stats, int slots, const float* rstd, float4* lnstat, int64_t count,
                      int d);
 void copy_state(Launcher& lc, int dtype, void* dst, const void* src, int64_t elems);
+// dst[i] = a[i] * b[i] (dtype), elems a multiple of the 16-byte vector
+void mul_elementwise(Launcher& lc, int dtype, void* dst, const void* a, const void* b, int64_t elems);
 // states[s][e] += carry[e] for s in [0, count)
 void add_to_states(Launcher& lc, int dtype, void* states, const void* carry, int count, int64_t elems);
 // LayerNorm forward of one state: x (float master or dtype) -> xhat (dtype), rstd (float).

@@ -394,6 +394,21 @@ __global__ void copy_kernel(T* __restrict__ dst, const T* __restrict__ src, int6
   if (v < nvec) stv<T>(dst + v * Vec<T>::N, ldv<T>(src + v * Vec<T>::N));
 }
 
+template <typename T>
+__global__ void mul_kernel(T* __restrict__ dst, const T* __restrict__ a, const T* __restrict__ b, int64_t nvec) {
+  constexpr int V = Vec<T>::N;
+  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v >= nvec) return;
+  float x[V], y[V];
+  ldv_stream<T>(a + v * V).get(x);
+  ldv_stream<T>(b + v * V).get(y);
+#pragma unroll
+  for (int i = 0; i < V; ++i) x[i] *= y[i];
+  Vec<T> out;
+  out.set(x);
+  stv<T>(dst + v * V, out);
+}
+
 // states[s] += carry for every state s (the carry of a scan whose gates are all one, applied after the fact)
 template <typename T>
 __global__ void add_to_states_kernel(T* __restrict__ states, const T* __restrict__ carry, int64_t elems) {
@@ -616,6 +631,15 @@ void copy_state(Launcher& lc, int dtype, void* dst, const void* src, int64_t ele
     copy_kernel<float><<<(unsigned)((elems / 4 + 255) / 256), 256, 0, lc.stream>>>((float*)dst, (const float*)src, elems / 4);
   else
     copy_kernel<bf16><<<(unsigned)((elems / 8 + 255) / 256), 256, 0, lc.stream>>>((bf16*)dst, (const bf16*)src, elems / 8);
+  lc.count();
+  lc.check();
+}
+
+void mul_elementwise(Launcher& lc, int dtype, void* dst, const void* a, const void* b, int64_t elems) {
+  const int V = dtype == HBP_F32 ? 4 : 8;
+  const unsigned grid = (unsigned)((elems / V + 255) / 256);
+  if (dtype == HBP_F32) mul_kernel<float><<<grid, 256, 0, lc.stream>>>((float*)dst, (const float*)a, (const float*)b, elems / V);
+  else mul_kernel<bf16><<<grid, 256, 0, lc.stream>>>((bf16*)dst, (const bf16*)a, (const bf16*)b, elems / V);
   lc.count();
   lc.check();
 }

@@ -74,3 +74,11 @@ def test_argument_errors_before_any_cuda_call(B):
     assert lib.hbp_sync_status(None, None) == 1
     assert B.status_string(8) == "bounded device wait expired"
     assert B.cumsumprod_static_max_bytes() == 32 << 20
+
+
+def test_relu_residual_kind_is_float_only(B):
+    n = C.c_size_t()
+    ok = B.make_config("relu_mlp", "f32", 4, 64, 32, hidden=128)
+    bad = B.make_config("relu_mlp", "bf16", 4, 64, 32, hidden=128)
+    assert B.lib.hbp_workspace_bytes(C.byref(ok), C.byref(n)) == 0 and n.value > 0
+    assert B.lib.hbp_workspace_bytes(C.byref(bad), C.byref(n)) == 6
