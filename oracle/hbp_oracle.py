@@ -299,6 +299,36 @@ class ReluResStep:
         return self.inner.param_vjp(cache, cache["mask"] * g)
 
 
+class PostLNStep:
+    """Post-LayerNorm layer f(x) = LN(x + Block(x)) (Table 1, row "Transformer (Post-LN)": g = [a(x), b(x)],
+    r(x, z) = z1 * x + z2; Appendix C.3's derivation with alpha = 1, beta = 0): with y = x + Block(x),
+    a(x) = 1 / sigma(y) per row and b(x) = (Block(x) - mu(y)) / sigma(y).  K = diag(a) is a row-wise scalar gate that
+    depends on the state; J is the rest of the layer's Jacobian.  `inner` is the block (an MLPStep)."""
+
+    def __init__(self, inner, eps):
+        self.inner, self.eps = inner, eps
+
+    def forward(self, x):
+        z, cache = self.inner.forward(x)
+        out, rstd = layernorm(x + z, self.eps)
+        cache = dict(cache)
+        cache["out"], cache["rstd"] = out, rstd
+        return out - rstd * x, cache      # what r adds to a(x) * x
+
+    def gate(self, cache):
+        return cache["rstd"]              # [..., 1]: the same gate for every channel of a row
+
+    def _through_ln(self, cache, g):
+        return layernorm_vjp(cache["out"], cache["rstd"], g)
+
+    def vjp(self, cache, g):
+        t = self._through_ln(cache, g)    # dLoss/dy; the layer's full VJP is t + J_Block^T t
+        return t - cache["rstd"] * g + self.inner.vjp(cache, t)
+
+    def param_vjp(self, cache, g):
+        return self.inner.param_vjp(cache, self._through_ln(cache, g))
+
+
 class ShiftedStep:
     """The gamma-shifted split of a residual layer x + Block(x) (Appendix C.3, Eq. 17): the block becomes
     g(x) = Block(x) + gamma x and the residual function r(x, z) = (1 - gamma) x + z, so the layer itself is
@@ -372,6 +402,11 @@ def lstm_stack(W, U, X):
 def relu_mlp_stack(W1, W2):
     """L layers x <- ReLU(x + W2 gelu(W1 x))."""
     return Stack([ReluResStep(s) for s in mlp_stack(W1, W2, False, 0.0).steps])
+
+
+def postln_mlp_stack(W1, W2, eps=1e-5):
+    """L layers x <- LN(x + W2 gelu(W1 x)), LayerNorm without affine."""
+    return Stack([PostLNStep(s, eps) for s in mlp_stack(W1, W2, False, 0.0).steps])
 
 
 def rnn_stack(W, U, a, X):

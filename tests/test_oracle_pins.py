@@ -671,3 +671,46 @@ def test_relu_residual_matches_autograd_and_path_sums():
         w = O.highway_bp(one, c1, d1, k)
         for i in range(L + 1):
             np.testing.assert_allclose(w[i].reshape(-1), O.path_sum(flat, J, K, i, k), rtol=1e-6, atol=1e-8)
+
+
+# ---------------------------------------------- 15. post-LN layers: a row-wise gate 1 / sigma (Table 1, Appendix C.3)
+def test_postln_matches_autograd_and_path_sums():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(71)
+    L, d, h, N, eps = 4, 5, 6, 2, 1e-5
+    W1 = rng.normal(size=(L, h, d)) * 0.7
+    W2 = rng.normal(size=(L, d, h)) * 0.7
+    st = O.postln_mlp_stack(W1, W2, eps)
+    x0 = rng.normal(size=(N, d))
+    xs, caches = O.forward(st, x0)
+    xt = torch.tensor(x0, requires_grad=True)
+    x = xt
+    for l in range(L):
+        y = x + torch.nn.functional.gelu(x @ torch.tensor(W1[l]).T) @ torch.tensor(W2[l]).T
+        x = torch.nn.functional.layer_norm(y, (d,), eps=eps)
+        np.testing.assert_allclose(xs[l + 1], x.detach().numpy(), rtol=1e-11, atol=1e-12)
+    y_t = rng.normal(size=(N, d))
+    (0.5 * ((x - torch.tensor(y_t)) ** 2).sum()).backward()
+    deltas = [np.zeros_like(x0) for _ in range(L)] + [xs[L] - y_t]
+    g = O.exact_bp(st, caches, deltas)
+    np.testing.assert_allclose(g[0], xt.grad.numpy(), rtol=1e-9, atol=1e-11)
+    for a, b in zip(O.highway_bp(st, caches, deltas, L), g):
+        np.testing.assert_allclose(a, b, rtol=1e-10, atol=1e-12)
+    # path sums on one row: K = diag(rstd), J = (Jacobian of the whole layer, by finite differences) - K
+    one = O.postln_mlp_stack(W1, W2, eps)
+    xs1, c1 = O.forward(one, x0[:1])
+    d1 = [rng.normal(size=(1, d)) for _ in range(L + 1)]
+    J, K = [None], [None]
+    for l in range(L):
+        def layer(v, l=l):
+            blk, c = one.steps[l].forward(v.reshape(1, d))
+            return (one.steps[l].gate(c) * v.reshape(1, d) + blk).reshape(-1)
+        full = O.finite_difference_jacobian(layer, xs1[l].reshape(-1), h=1e-5)
+        Km = np.eye(d) * float(c1[l]["rstd"].reshape(-1)[0])
+        K.append(Km)
+        J.append(full - Km)
+    flat = [v.reshape(-1) for v in d1]
+    for k in range(L + 1):
+        w = O.highway_bp(one, c1, d1, k)
+        for i in range(L + 1):
+            np.testing.assert_allclose(w[i].reshape(-1), O.path_sum(flat, J, K, i, k), rtol=1e-5, atol=1e-7)
