@@ -89,7 +89,7 @@ def measured_traffic(key, w):
 
 def algorithmic_flops(w, k):
     """VJP flops per iteration and parameter-pass flops of the MLP stacks (4dh and 6dh per token-layer)."""
-    if w.block in ("mlp", "preln_mlp", "relu_mlp"):
+    if w.block in ("mlp", "preln_mlp", "relu_mlp", "postln_mlp"):
         per = w.d * w.hidden * w.tokens * w.L
         return 4 * per, 6 * per
     if w.block == "rnn_tanh":

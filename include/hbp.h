@@ -77,10 +77,14 @@ typedef enum {
  *  RELU_MLP          Table 1, row "ResNet": x' = ReLU(x + W2 gelu(W1 x)).  The residual gate is the ReLU's 0/1 mask
  *                    [x + Block(x) > 0], produced by hbp_forward and kept in the workspace; the block Jacobian is
  *                    the mask times the MLP's.  cfg.gate must be HBP_GATE_ONE, cfg.gamma 0, cfg.dtype HBP_F32 (a mask
- *                    decided in bf16 arithmetic flips on elements near zero; HBP_ERR_UNSUPPORTED). */
+ *                    decided in bf16 arithmetic flips on elements near zero; HBP_ERR_UNSUPPORTED).
+ *  POSTLN_MLP        Table 1, row "Transformer (Post-LN)" and Appendix C.3 with alpha = 1, beta = 0:
+ *                    x' = LN(x + W2 gelu(W1 x)) = a(x) (.) x + b(x) with the row-wise gate a = 1 / sigma(x + Block(x)),
+ *                    produced by hbp_forward; the block Jacobian is the rest of the layer's.  cfg.gate must be
+ *                    HBP_GATE_ONE, cfg.gamma 0. */
 typedef enum {
   HBP_BLOCK_MLP = 0, HBP_BLOCK_PRELN_MLP = 1, HBP_BLOCK_RNN_TANH = 2, HBP_BLOCK_PRELN_TRANSFORMER = 3, HBP_BLOCK_GRU = 4,
-  HBP_BLOCK_LSTM = 5, HBP_BLOCK_RELU_MLP = 6
+  HBP_BLOCK_LSTM = 5, HBP_BLOCK_RELU_MLP = 6, HBP_BLOCK_POSTLN_MLP = 7
 } hbp_block;
 typedef enum { HBP_F32 = 0, HBP_BF16 = 1 } hbp_dtype;
 /* Residual gate a_l, the diagonal of K (Eq. 2): all ones, one vector a[d] for every step, or a[steps][d]. */

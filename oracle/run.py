@@ -47,6 +47,10 @@ def build_stack(cfg, inputs, rows=None):
         stack = O.relu_mlp_stack(F64Items(inputs["W1"]), F64Items(inputs["W2"]))
         x0 = _np(inputs["x0"] if rows is None else inputs["x0"][rows])
         groups = [("", l) for l in range(cfg.L)]
+    elif cfg.block == "postln_mlp":
+        stack = O.postln_mlp_stack(F64Items(inputs["W1"]), F64Items(inputs["W2"]), cfg.ln_eps)
+        x0 = _np(inputs["x0"] if rows is None else inputs["x0"][rows])
+        groups = [("", l) for l in range(cfg.L)]
     elif cfg.block == "rnn_tanh":
         X = inputs["X"] if rows is None else inputs["X"][:, rows]
         stack = O.rnn_stack(_np(inputs["W"]), _np(inputs["U"]), _np(inputs["a"]), F64Items(X))

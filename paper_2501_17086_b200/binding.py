@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhbp.so")
 
 HBP_F32, HBP_BF16 = 0, 1
-BLOCKS = {"mlp": 0, "preln_mlp": 1, "rnn_tanh": 2, "preln_transformer": 3, "gru": 4, "lstm": 5, "relu_mlp": 6}
+BLOCKS = {"mlp": 0, "preln_mlp": 1, "rnn_tanh": 2, "preln_transformer": 3, "gru": 4, "lstm": 5, "relu_mlp": 6, "postln_mlp": 7}
 GATE_ONE, GATE_CHANNEL_SHARED, GATE_CHANNEL_PER_STEP = 0, 1, 2
 LOSS_FINAL, LOSS_EVERY_STEP = 0, 1
 
@@ -140,7 +140,7 @@ _GRAD_SHAPES = {
     "preln_transformer": lambda c: {"dW1": (c.L, c.hidden, c.d), "dW2": (c.L, c.d, c.hidden),
                                     **{n: (c.L, c.d, c.d) for n in ("dWq", "dWk", "dWv", "dWo")}},
 }
-_GRAD_SHAPES["preln_mlp"] = _GRAD_SHAPES["relu_mlp"] = _GRAD_SHAPES["mlp"]
+_GRAD_SHAPES["preln_mlp"] = _GRAD_SHAPES["relu_mlp"] = _GRAD_SHAPES["postln_mlp"] = _GRAD_SHAPES["mlp"]
 _BLOCK_NAMES = {v: k for k, v in BLOCKS.items()}
 
 

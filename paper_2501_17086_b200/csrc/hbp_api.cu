@@ -67,6 +67,9 @@ struct hbp_ctx {
   char *Fg = nullptr, *C5 = nullptr;
   // ReLU(x + Block(x)): the masks [L][N][d] (0/1 in dtype: the scan's gate) and mask * g_{l+1} [L][N][d]
   char *MASK = nullptr, *GM = nullptr;
+  // post-LN layers: GM holds LayerNorm-backward of g_{l+1} (what the block is differentiated against), CB the part of
+  // the layer's VJP that is not the block's, rstd [L][N] is the scan's row gate
+  char* CB = nullptr;
   char* scan_scratch = nullptr;
   size_t scan_scratch_bytes = 0;
   float* partial = nullptr;  // split-K / gate-gradient partial sums
@@ -93,7 +96,7 @@ inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 hbp_status check_config(const hbp_config* c) {
   if (!c) return HBP_ERR_INVALID_ARG;
   if (c->dtype != HBP_F32 && c->dtype != HBP_BF16) return HBP_ERR_DTYPE;
-  if (c->block < 0 || c->block > HBP_BLOCK_RELU_MLP) return HBP_ERR_UNSUPPORTED;
+  if (c->block < 0 || c->block > HBP_BLOCK_POSTLN_MLP) return HBP_ERR_UNSUPPORTED;
   if (c->gate < 0 || c->gate > HBP_GATE_CHANNEL_PER_STEP) return HBP_ERR_UNSUPPORTED;
   if (c->loss != HBP_LOSS_FINAL && c->loss != HBP_LOSS_EVERY_STEP) return HBP_ERR_UNSUPPORTED;
   const int v = c->dtype == HBP_F32 ? 4 : 8;
@@ -103,7 +106,9 @@ hbp_status check_config(const hbp_config* c) {
   if (c->d % v) return HBP_ERR_SHAPE;
   if (c->d / v > 1024) return HBP_ERR_SHAPE;  // one block per row in the LayerNorm kernels
   const bool gated_cell = c->block == HBP_BLOCK_GRU || c->block == HBP_BLOCK_LSTM;
-  if ((gated_cell || c->block == HBP_BLOCK_RELU_MLP) && (c->gate != HBP_GATE_ONE || c->gamma != 0.0f)) return HBP_ERR_UNSUPPORTED;
+  if ((gated_cell || c->block == HBP_BLOCK_RELU_MLP || c->block == HBP_BLOCK_POSTLN_MLP) &&
+      (c->gate != HBP_GATE_ONE || c->gamma != 0.0f))
+    return HBP_ERR_UNSUPPORTED;
   // the 0/1 mask is a sign decision: taken in bf16 arithmetic it differs from an exact evaluation on the elements
   // that land near zero, and each such element changes its whole gradient path; float only
   if (c->block == HBP_BLOCK_RELU_MLP && c->dtype != HBP_F32) return HBP_ERR_UNSUPPORTED;
@@ -203,6 +208,11 @@ size_t carve(hbp_ctx* c, char* base) {
       c->MASK = take(steps * N * d * es);
       c->GM = take(steps * N * d * es);
     }
+    if (f.block == HBP_BLOCK_POSTLN_MLP) {
+      c->GM = take(steps * N * d * es);
+      c->CB = take(steps * N * d * es);
+      c->rstd = (float*)take(steps * N * 4);
+    }
     c->ACT = take((size_t)c->layers * N * h * es);
     c->DACT = take((size_t)c->layers * N * h * es);
     const size_t per_layer = N * h * es;
@@ -292,6 +302,12 @@ struct Run {
   }
   void mask_gradients(int b0, int b1) {
     if (!c->GM) return;
+    if (c->CB) {  // post-LN: through the layer's LayerNorm first (its output is the next state)
+      postln_prepass(lc, c->cfg.dtype, at(g, (int64_t)(b0 + 1) * state), at(x_all, (int64_t)(b0 + 1) * state),
+                     c->rstd + (int64_t)b0 * N, at(c->GM, (int64_t)b0 * state), at(c->CB, (int64_t)b0 * state),
+                     (int64_t)(b1 - b0) * N, (int)d);
+      return;
+    }
     mul_elementwise(lc, c->cfg.dtype, at(c->GM, (int64_t)b0 * state), at(c->MASK, (int64_t)b0 * state),
                     at(g, (int64_t)(b0 + 1) * state), (int64_t)(b1 - b0) * state);
   }
@@ -639,6 +655,10 @@ struct Run {
     if (c->cfg.block == HBP_BLOCK_GRU) { s.a = c->Zc; s.gate = kGateElement; }
     if (c->cfg.block == HBP_BLOCK_LSTM) { s.a = c->Fg; s.gate = kGateElement; }
     if (c->cfg.block == HBP_BLOCK_RELU_MLP) { s.a = c->MASK; s.gate = kGateElement; }
+    if (c->cfg.block == HBP_BLOCK_POSTLN_MLP) {
+      s.gate = kGateRow; s.row_gate = c->rstd;
+      if (with_u) s.u2 = c->CB;
+    }
     s.g = g;
     if (with_u && c->preln) {
       s.xhat = c->Y; s.rstd = c->rstd;
@@ -938,6 +958,11 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
       c2.B = r.at(params->W2, (int64_t)b * d * h); c2.b_sn = h; c2.b_sk = 1;
       resid_epilogue(c2, step);
       r.run_gemm(c2);
+      if (f.block == HBP_BLOCK_POSTLN_MLP) {  // x_{l+1} = LN(x_l + Block(x_l)), normalised in place; 1/sigma is the gate
+        const void* src = ctx->xres ? (const void*)ctx->xres : (const void*)r.at(xa, (int64_t)(step + 1) * state);
+        layernorm_fwd(r.lc, f.dtype, src, ctx->xres != nullptr, r.at(xa, (int64_t)(step + 1) * state),
+                      ctx->rstd + (int64_t)step * N, N, (int)d, f.ln_eps, ctx->xres);
+      }
     }
   }
   ctx->forward_done = true;
@@ -1099,7 +1124,8 @@ hbp_status hbp_add_carry(hbp_ctx* ctx, const void* carry, void* g_all, void* cud
   if (!ctx || !carry || !g_all) return HBP_ERR_INVALID_ARG;
   if (misaligned(carry) || misaligned(g_all)) return HBP_ERR_SHAPE;
   if (ctx->cfg.gate != HBP_GATE_ONE || ctx->cfg.gamma != 0.0f || ctx->cfg.block == HBP_BLOCK_GRU ||
-      ctx->cfg.block == HBP_BLOCK_LSTM || ctx->cfg.block == HBP_BLOCK_RELU_MLP)
+      ctx->cfg.block == HBP_BLOCK_LSTM || ctx->cfg.block == HBP_BLOCK_RELU_MLP ||
+      ctx->cfg.block == HBP_BLOCK_POSTLN_MLP)
     return HBP_ERR_UNSUPPORTED;
   Launcher lc;
   lc.stream = (cudaStream_t)cuda_stream;

@@ -93,6 +93,8 @@ extern bool g_gemm_pair;
 // Internal gate kind beside the public hbp_gate values: a[L][rows][d], one gate per element and step (the
 // state-dependent gate of a GRU, produced by its forward pass).
 constexpr int kGateElement = 3;
+// ... and a[L][rows] in float, one gate per row and step (ScanArgs::row_gate; post-LN layers: 1 / sigma of the row)
+constexpr int kGateRow = 4;
 struct ScanArgs {
   int dtype = HBP_F32;
   int L = 0;               // number of steps in the buffers
@@ -106,6 +108,8 @@ struct ScanArgs {
   bool u_has_delta = false;     // u[l] already contains delta_l for l < L (added by the producing GEMM)
   const void* delta = nullptr;  // per hbp_loss
   int loss = HBP_LOSS_FINAL;
+  const float* row_gate = nullptr;  // kGateRow only
+  const void* u2 = nullptr;         // optional second additive tensor [L][rows][d] (serial depth scan only)
   const void* a = nullptr;  // gate
   int gate = HBP_GATE_ONE;  // an hbp_gate value, or kGateElement
   void* g = nullptr;  // [L+1][rows][d]
@@ -134,8 +138,12 @@ void mul_elementwise(Launcher& lc, int dtype, void* dst, const void* a, const vo
 // states[s][e] += carry[e] for s in [0, count)
 void add_to_states(Launcher& lc, int dtype, void* states, const void* carry, int count, int64_t elems);
 // LayerNorm forward of one state: x (float master or dtype) -> xhat (dtype), rstd (float).
+// (master, if given, receives the normalised values in float as well)
 void layernorm_fwd(Launcher& lc, int dtype, const void* x, bool x_is_f32, void* xhat, float* rstd, int64_t rows,
-                   int d, float eps);
+                   int d, float eps, float* master = nullptr);
+// t = rstd (g - mean g - xo mean(g xo)) and c = t - rstd g per row (post-LN layers; xo = the layer's output state)
+void postln_prepass(Launcher& lc, int dtype, const void* g, const void* xo, const float* rstd, void* t_out, void* c_out,
+                    int64_t rows, int d);
 void convert_to_f32(Launcher& lc, int dtype, const void* src, float* dst, int64_t elems);
 // da[c] = sum over rows of g[r][c] * x[r][c] (deterministic two-stage reduction; partial holds blocks*d floats).
 void gate_grad(Launcher& lc, int dtype, const void* g, const void* x, int64_t rows_total, int d, float* da,

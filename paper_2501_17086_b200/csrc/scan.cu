@@ -78,7 +78,7 @@ __device__ __forceinline__ const T* delta_at(const ScanArgs& s, int l, int64_t s
 // gate vector of step l for the 16-byte group at element `off` of the state, channel `ch` (nullptr = ones)
 template <typename T>
 __device__ __forceinline__ const T* gate_at(const ScanArgs& s, int l, int64_t state_elems, int64_t off, int ch) {
-  if (s.gate == HBP_GATE_ONE || !s.a) return nullptr;
+  if (s.gate == HBP_GATE_ONE || s.gate == kGateRow || !s.a) return nullptr;
   if (s.gate == kGateElement) return (const T*)s.a + (int64_t)l * state_elems + off;
   return (const T*)s.a + (s.gate == HBP_GATE_CHANNEL_PER_STEP ? (int64_t)l * s.d : 0) + ch;
 }
@@ -89,7 +89,11 @@ __device__ __forceinline__ void scan_step(const ScanArgs& s, int l, int64_t stat
                                           const typename Acc<T>::type* carry, typename Acc<T>::type* val) {
   constexpr int V = Vec<T>::N;
   const T* gp = gate_at<T>(s, l, state_elems, off, ch);
-  if (gp) {
+  if (s.gate == kGateRow) {  // one gate value per row and step (a float table [L][rows])
+    const float a = __ldg(s.row_gate + (int64_t)l * s.rows + off / s.d);
+#pragma unroll
+    for (int i = 0; i < V; ++i) val[i] = a * carry[i];
+  } else if (gp) {
     float a[V];
     ldv<T>(gp).get(a);
 #pragma unroll
@@ -97,6 +101,12 @@ __device__ __forceinline__ void scan_step(const ScanArgs& s, int l, int64_t stat
   } else {
 #pragma unroll
     for (int i = 0; i < V; ++i) val[i] = s.keep * carry[i];
+  }
+  if (s.u2) {
+    float w[V];
+    ldv_stream<T>((const T*)s.u2 + (int64_t)l * state_elems + off).get(w);
+#pragma unroll
+    for (int i = 0; i < V; ++i) val[i] += w[i];
   }
   if (s.u) {
     float u[V];
@@ -435,7 +445,8 @@ __global__ void to_f32_kernel(const T* __restrict__ src, float* __restrict__ dst
 // xhat = (x - mean) * rstd over the last axis, biased variance; one block per row, two passes in registers.
 template <typename T, typename X>
 __global__ void __launch_bounds__(1024) layernorm_fwd_kernel(const X* __restrict__ x, T* __restrict__ xhat,
-                                                             float* __restrict__ rstd, int d, float eps) {
+                                                             float* __restrict__ rstd, int d, float eps,
+                                                             float* __restrict__ master) {
   constexpr int V = Vec<T>::N;
   __shared__ float red[2][32];
   const int64_t row = blockIdx.x;
@@ -475,7 +486,66 @@ __global__ void __launch_bounds__(1024) layernorm_fwd_kernel(const X* __restrict
     Vec<T> out;
     out.set(o);
     stv<T>(xhat + row * d + threadIdx.x * V, out);
+    if (master) {  // the float copy of the residual stream continues from the normalised values (post-LN layers)
+#pragma unroll
+      for (int i = 0; i < V; ++i) master[row * d + threadIdx.x * V + i] = o[i];
+    }
   }
+}
+
+// Post-LN layers: per row, t = LayerNorm-backward of g through the layer's own output xo (the normalised state):
+// t = rstd (g - mean g - xo mean(g xo)), and c = t - rstd g, the part of the layer's VJP that is not the block's.
+template <typename T>
+__global__ void __launch_bounds__(1024) postln_prepass_kernel(const T* __restrict__ g, const T* __restrict__ xo,
+                                                              const float* __restrict__ rstd, T* __restrict__ t_out,
+                                                              T* __restrict__ c_out, int d) {
+  constexpr int V = Vec<T>::N;
+  __shared__ float red[2][32];
+  const int64_t row = blockIdx.x;
+  const bool active = (int)threadIdx.x * V < d;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
+  const int64_t off = row * d + (int64_t)threadIdx.x * V;
+  float gv[V], xv[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) gv[i] = xv[i] = 0.0f;
+  if (active) {
+    ldv<T>(g + off).get(gv);
+    ldv<T>(xo + off).get(xv);
+  }
+  float s1 = 0.0f, s2 = 0.0f;
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    s1 += gv[i];
+    s2 = fmaf(gv[i], xv[i], s2);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+    s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+  }
+  if (lane == 0) {
+    red[0][warp] = s1;
+    red[1][warp] = s2;
+  }
+  __syncthreads();
+  float t1 = 0.0f, t2 = 0.0f;
+  for (int w = 0; w < nwarps; ++w) {
+    t1 += red[0][w];
+    t2 += red[1][w];
+  }
+  if (!active) return;
+  const float m1 = t1 / (float)d, m2 = t2 / (float)d, r = rstd[row];
+  float tv[V], cv[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    cv[i] = r * (-m1 - xv[i] * m2);
+    tv[i] = fmaf(r, gv[i], cv[i]);
+  }
+  Vec<T> a, b;
+  a.set(tv);
+  b.set(cv);
+  stv<T>(t_out + off, a);
+  stv<T>(c_out + off, b);
 }
 
 // partial[b][c] = sum over the block's rows of g[r][c] * x[r][c]
@@ -583,8 +653,9 @@ void scan_reverse(Launcher& lc, const ScanArgs& s) {
   const size_t need = scan_scratch_bytes(s.dtype, steps, s.rows, s.d);
   // few channels, many steps: one serial pass in time behind a ring of TMA loads reads and writes every byte
   // once; the three-phase form below remains for what that kernel does not take (a gate table per step)
-  if (need > 0 && scan_ring(lc, s)) return;
-  if (need > 0 && s.scratch && s.scratch_bytes >= need && s.keep == 1.0f && s.gamma == 0.0f) {
+  const bool depth_only = s.u2 || s.gate == kGateRow;  // forms only the serial depth scan takes
+  if (need > 0 && !depth_only && scan_ring(lc, s)) return;
+  if (need > 0 && !depth_only && s.scratch && s.scratch_bytes >= need && s.keep == 1.0f && s.gamma == 0.0f) {
     const int nchunks = (steps + kChunk - 1) / kChunk;
     dim3 grid((unsigned)((nvec + 127) / 128), nchunks);
     const unsigned cgrid = (unsigned)((s.rows * s.d + 127) / 128);
@@ -635,6 +706,20 @@ void copy_state(Launcher& lc, int dtype, void* dst, const void* src, int64_t ele
   lc.check();
 }
 
+void postln_prepass(Launcher& lc, int dtype, const void* g, const void* xo, const float* rstd, void* t_out, void* c_out,
+                    int64_t rows, int d) {
+  const int V = dtype == HBP_F32 ? 4 : 8;
+  const int threads = row_block_threads(d, V);
+  if (dtype == HBP_F32)
+    postln_prepass_kernel<float><<<(unsigned)rows, threads, 0, lc.stream>>>((const float*)g, (const float*)xo, rstd,
+                                                                           (float*)t_out, (float*)c_out, d);
+  else
+    postln_prepass_kernel<bf16><<<(unsigned)rows, threads, 0, lc.stream>>>((const bf16*)g, (const bf16*)xo, rstd,
+                                                                          (bf16*)t_out, (bf16*)c_out, d);
+  lc.count();
+  lc.check();
+}
+
 void mul_elementwise(Launcher& lc, int dtype, void* dst, const void* a, const void* b, int64_t elems) {
   const int V = dtype == HBP_F32 ? 4 : 8;
   const unsigned grid = (unsigned)((elems / V + 255) / 256);
@@ -662,15 +747,15 @@ void convert_to_f32(Launcher& lc, int dtype, const void* src, float* dst, int64_
 }
 
 void layernorm_fwd(Launcher& lc, int dtype, const void* x, bool x_is_f32, void* xhat, float* rstd, int64_t rows,
-                   int d, float eps) {
+                   int d, float eps, float* master) {
   const int V = dtype == HBP_F32 ? 4 : 8;
   const int threads = row_block_threads(d, V);
   if (dtype == HBP_F32)
-    layernorm_fwd_kernel<float, float><<<(unsigned)rows, threads, 0, lc.stream>>>((const float*)x, (float*)xhat, rstd, d, eps);
+    layernorm_fwd_kernel<float, float><<<(unsigned)rows, threads, 0, lc.stream>>>((const float*)x, (float*)xhat, rstd, d, eps, master);
   else if (x_is_f32)
-    layernorm_fwd_kernel<bf16, float><<<(unsigned)rows, threads, 0, lc.stream>>>((const float*)x, (bf16*)xhat, rstd, d, eps);
+    layernorm_fwd_kernel<bf16, float><<<(unsigned)rows, threads, 0, lc.stream>>>((const float*)x, (bf16*)xhat, rstd, d, eps, master);
   else
-    layernorm_fwd_kernel<bf16, bf16><<<(unsigned)rows, threads, 0, lc.stream>>>((const bf16*)x, (bf16*)xhat, rstd, d, eps);
+    layernorm_fwd_kernel<bf16, bf16><<<(unsigned)rows, threads, 0, lc.stream>>>((const bf16*)x, (bf16*)xhat, rstd, d, eps, master);
   lc.count();
   lc.check();
 }

@@ -24,7 +24,7 @@ import torch
 @dataclasses.dataclass(frozen=True)
 class Workload:
     name: str
-    block: str            # "mlp" | "preln_mlp" | "rnn_tanh" | "preln_transformer" | "gru" | "lstm" | "relu_mlp"
+    block: str            # "mlp" | "preln_mlp" | "rnn_tanh" | "preln_transformer" | "gru" | "lstm" | "relu_mlp" | "postln_mlp"
     dtype: str            # "f32" | "bf16"
     L: int                # residual steps (mlp), time steps (rnn), decoder blocks (transformer)
     d: int
@@ -64,6 +64,8 @@ WORKLOADS = {
     "g2": Workload("g2", "gru", "f32", L=1024, d=64, in_dim=4, batch=128, tokens=128, seed=1007, loss="every_mse"),
     # LSTM in the shape of the paper's character-level experiment: 256 steps, 512 units (state [c, h] 1024 wide)
     "l1": Workload("l1", "lstm", "f32", L=256, d=1024, hidden=512, in_dim=212, batch=128, tokens=128, seed=1008, loss="every_mse"),
+    # c2's shape with post-LN layers x <- LN(x + MLP(x)) (the RoBERTa-style row of Table 1)
+    "p2": Workload("p2", "postln_mlp", "bf16", L=64, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1009),
     # c2 with 8 layers: same per-launch tile shapes, small enough for multi-pass profiler captures
     "c2_small": Workload("c2_small", "preln_mlp", "bf16", L=8, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1012),
     # c4 with 4 decoder blocks: same per-launch shapes, small enough for multi-pass profiler captures
@@ -85,6 +87,9 @@ WORKLOADS = {
     "lstm_twin_bf16": Workload("lstm_twin_bf16", "lstm", "bf16", L=24, d=64, hidden=32, in_dim=16, batch=6, tokens=6, seed=2027,
                                loss="every_mse"),
     "relu_twin": Workload("relu_twin", "relu_mlp", "f32", L=5, d=96, hidden=200, batch=1, seq=77, tokens=77, seed=2008),
+    "postln_twin": Workload("postln_twin", "postln_mlp", "f32", L=5, d=96, hidden=200, batch=1, seq=77, tokens=77, seed=2009),
+    "postln_twin_bf16": Workload("postln_twin_bf16", "postln_mlp", "bf16", L=5, d=256, hidden=1024, batch=1, seq=328,
+                                 tokens=328, seed=2019),
     "c4_twin": Workload("c4_twin", "preln_transformer", "bf16", L=2, d=128, hidden=512, n_heads=2, head_dim=64,
                         seq=200, batch=2, tokens=400, seed=2004),
     "c4_twin_f32": Workload("c4_twin_f32", "preln_transformer", "f32", L=2, d=64, hidden=128, n_heads=2, head_dim=32,
@@ -100,7 +105,7 @@ def _randn(gen, shape, std, device):
 def make_inputs(cfg: Workload, device="cpu"):
     """Returns a dict of tensors in ``cfg.dtype`` on ``device``.
 
-    Keys: mlp / preln_mlp / relu_mlp: W1 [L,h,d], W2 [L,d,h], x0 [N,d], y [N,d].
+    Keys: mlp / preln_mlp / relu_mlp / postln_mlp: W1 [L,h,d], W2 [L,d,h], x0 [N,d], y [N,d].
     rnn_tanh: a [d], W [d,d], U [d,in], X [T,B,in], Y [T,B,d], x0 [B,d] (zeros).
     gru: W [3d,d] (variance 1/d), U [3d,in] (variance 1/in), X, Y, x0 as for rnn_tanh.
     lstm: W [4u,u] (variance 1/u), U [4u,in] (variance 1/in) with u = hidden units, d = 2u; X [T,B,in], Y [T,B,2u],
@@ -115,9 +120,9 @@ def make_inputs(cfg: Workload, device="cpu"):
     gen.manual_seed(cfg.seed)
     dt = cfg.torch_dtype
     out = {}
-    if cfg.block in ("mlp", "preln_mlp", "relu_mlp"):
+    if cfg.block in ("mlp", "preln_mlp", "relu_mlp", "postln_mlp"):
         L, d, h, N = cfg.L, cfg.d, cfg.hidden, cfg.tokens
-        if cfg.block in ("mlp", "relu_mlp"):
+        if cfg.block in ("mlp", "relu_mlp", "postln_mlp"):
             s1, s2 = 1.0 / math.sqrt(d), 1.0 / math.sqrt(h)
         else:
             s1, s2 = 0.02, 0.02 / math.sqrt(2.0 * cfg.steps)

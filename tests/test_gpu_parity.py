@@ -76,6 +76,8 @@ def compare(w, gpu, ref, ks, grads_for):
     ("lstm_twin_long", (0, 1, 3)),
     ("lstm_twin_bf16", (1, 2, 4)),
     ("relu_twin", (0, 1, 2, 5)),
+    ("postln_twin", (0, 1, 2, 5)),
+    ("postln_twin_bf16", (1, 2, 5)),
 ])
 def test_twin_matches_oracle_in_full(name, ks):
     w = WORKLOADS[name]

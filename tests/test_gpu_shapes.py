@@ -18,10 +18,12 @@ def _case(seed):
     dtype = rnd.choice(["f32", "bf16"])
     v = 4 if dtype == "f32" else 8
     block = rnd.choice(["mlp", "preln_mlp", "rnn_tanh", "gru", "lstm", "preln_transformer"])
-    if seed >= 36:   # later seeds: the ReLU-residual kind (added after the first 36 cases were fixed)
+    if seed >= 42:   # the post-LN kind, both dtypes
+        block = "postln_mlp"
+    elif seed >= 36:   # later seeds: the ReLU-residual kind (added after the first 36 cases were fixed)
         block, dtype, v = "relu_mlp", "f32", 4
     mult = lambda lo, hi: v * rnd.randint(max(1, lo // v), hi // v)
-    if block in ("mlp", "preln_mlp", "relu_mlp"):
+    if block in ("mlp", "preln_mlp", "relu_mlp", "postln_mlp"):
         return Workload(f"rand{seed}", block, dtype, L=rnd.randint(1, 6), d=mult(8, 328), hidden=mult(8, 520),
                         tokens=rnd.randint(1, 300), batch=1, seq=1, seed=5000 + seed,
                         loss=rnd.choice(["final_mse", "final_half_sse"]))
@@ -39,7 +41,7 @@ def _case(seed):
                     loss="every_mse")
 
 
-@pytest.mark.parametrize("seed", range(42))
+@pytest.mark.parametrize("seed", range(50))
 def test_random_shape_matches_oracle(seed):
     w = _case(seed)
     rnd = random.Random(1000 + seed)
