@@ -303,27 +303,29 @@ class PostLNStep:
     """Post-LayerNorm layer f(x) = LN(x + Block(x)) (Table 1, row "Transformer (Post-LN)": g = [a(x), b(x)],
     r(x, z) = z1 * x + z2; Appendix C.3's derivation with alpha = 1, beta = 0): with y = x + Block(x),
     a(x) = 1 / sigma(y) per row and b(x) = (Block(x) - mu(y)) / sigma(y).  K = diag(a) is a row-wise scalar gate that
-    depends on the state; J is the rest of the layer's Jacobian.  `inner` is the block (an MLPStep)."""
+    depends on the state; J is the rest of the layer's Jacobian.  `inner` is the block (an MLPStep).
+    With the shift gamma of Appendix C.3 the split is g = [(1 - gamma) a, b + gamma x a]: K = (1 - gamma) diag(a), the
+    layer itself (and exact backpropagation) unchanged."""
 
-    def __init__(self, inner, eps):
-        self.inner, self.eps = inner, eps
+    def __init__(self, inner, eps, gamma=0.0):
+        self.inner, self.eps, self.gamma = inner, eps, float(gamma)
 
     def forward(self, x):
         z, cache = self.inner.forward(x)
         out, rstd = layernorm(x + z, self.eps)
         cache = dict(cache)
         cache["out"], cache["rstd"] = out, rstd
-        return out - rstd * x, cache      # what r adds to a(x) * x
+        return out - (1.0 - self.gamma) * rstd * x, cache      # what r adds to the gated state
 
     def gate(self, cache):
-        return cache["rstd"]              # [..., 1]: the same gate for every channel of a row
+        return (1.0 - self.gamma) * cache["rstd"]              # [..., 1]: the same gate for every channel of a row
 
     def _through_ln(self, cache, g):
         return layernorm_vjp(cache["out"], cache["rstd"], g)
 
     def vjp(self, cache, g):
         t = self._through_ln(cache, g)    # dLoss/dy; the layer's full VJP is t + J_Block^T t
-        return t - cache["rstd"] * g + self.inner.vjp(cache, t)
+        return t - (1.0 - self.gamma) * cache["rstd"] * g + self.inner.vjp(cache, t)
 
     def param_vjp(self, cache, g):
         return self.inner.param_vjp(cache, self._through_ln(cache, g))
@@ -404,9 +406,9 @@ def relu_mlp_stack(W1, W2):
     return Stack([ReluResStep(s) for s in mlp_stack(W1, W2, False, 0.0).steps])
 
 
-def postln_mlp_stack(W1, W2, eps=1e-5):
-    """L layers x <- LN(x + W2 gelu(W1 x)), LayerNorm without affine."""
-    return Stack([PostLNStep(s, eps) for s in mlp_stack(W1, W2, False, 0.0).steps])
+def postln_mlp_stack(W1, W2, eps=1e-5, gamma=0.0):
+    """L layers x <- LN(x + W2 gelu(W1 x)), LayerNorm without affine; gamma = the shift of the split."""
+    return Stack([PostLNStep(s, eps, gamma) for s in mlp_stack(W1, W2, False, 0.0).steps])
 
 
 def rnn_stack(W, U, a, X):

@@ -38,6 +38,8 @@ class Workload:
     seed: int = 0
     loss: str = "final_mse"   # "final_half_sse" | "final_mse" | "every_mse"
     ln_eps: float = 1e-5
+    init: str = ""        # MLP kinds: "fan_in" (variance 1/fan_in) or "small" (std 0.02, output weights 0.02/sqrt(2 steps));
+                          # "" = the kind's default (fan_in for mlp / relu_mlp / postln_mlp, small for preln_mlp)
 
     @property
     def steps(self) -> int:
@@ -65,7 +67,8 @@ WORKLOADS = {
     # LSTM in the shape of the paper's character-level experiment: 256 steps, 512 units (state [c, h] 1024 wide)
     "l1": Workload("l1", "lstm", "f32", L=256, d=1024, hidden=512, in_dim=212, batch=128, tokens=128, seed=1008, loss="every_mse"),
     # c2's shape with post-LN layers x <- LN(x + MLP(x)) (the RoBERTa-style row of Table 1)
-    "p2": Workload("p2", "postln_mlp", "bf16", L=64, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1009),
+    "p2": Workload("p2", "postln_mlp", "bf16", L=64, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1009,
+                   init="small"),
     # c2 with 8 layers: same per-launch tile shapes, small enough for multi-pass profiler captures
     "c2_small": Workload("c2_small", "preln_mlp", "bf16", L=8, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1012),
     # c4 with 4 decoder blocks: same per-launch shapes, small enough for multi-pass profiler captures
@@ -122,7 +125,8 @@ def make_inputs(cfg: Workload, device="cpu"):
     out = {}
     if cfg.block in ("mlp", "preln_mlp", "relu_mlp", "postln_mlp"):
         L, d, h, N = cfg.L, cfg.d, cfg.hidden, cfg.tokens
-        if cfg.block in ("mlp", "relu_mlp", "postln_mlp"):
+        init = cfg.init or ("small" if cfg.block == "preln_mlp" else "fan_in")
+        if init == "fan_in":
             s1, s2 = 1.0 / math.sqrt(d), 1.0 / math.sqrt(h)
         else:
             s1, s2 = 0.02, 0.02 / math.sqrt(2.0 * cfg.steps)

@@ -714,3 +714,31 @@ def test_postln_matches_autograd_and_path_sums():
         w = O.highway_bp(one, c1, d1, k)
         for i in range(L + 1):
             np.testing.assert_allclose(w[i].reshape(-1), O.path_sum(flat, J, K, i, k), rtol=1e-5, atol=1e-7)
+
+
+def test_postln_shift_leaves_the_network_and_exact_bp_unchanged():
+    rng = np.random.default_rng(72)
+    L, d, h, N = 5, 6, 7, 3
+    W1 = rng.normal(size=(L, h, d)) * 0.5
+    W2 = rng.normal(size=(L, d, h)) * 0.5
+    x0 = rng.normal(size=(N, d))
+    base = O.postln_mlp_stack(W1, W2)
+    xs0, c0 = O.forward(base, x0)
+    deltas = [np.zeros_like(x0) for _ in range(L)] + [rng.normal(size=(N, d))]
+    g0 = O.exact_bp(base, c0, deltas)
+    for gamma in (0.3, 0.8, 1.0):
+        st = O.postln_mlp_stack(W1, W2, gamma=gamma)
+        xs, c = O.forward(st, x0)
+        for a, b in zip(xs, xs0):
+            np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
+        for a, b in zip(O.exact_bp(st, c, deltas), g0):
+            np.testing.assert_allclose(a, b, rtol=1e-10, atol=1e-12)
+        for a, b in zip(O.highway_bp(st, c, deltas, L), g0):        # exact at k = L for every split
+            np.testing.assert_allclose(a, b, rtol=1e-9, atol=1e-11)
+        w1 = O.highway_bp(st, c, deltas, 1)
+        if gamma == 1.0:   # K = 0: one iteration reaches exactly one layer back (the fixed-point iteration)
+            assert all(np.all(w1[l] == 0.0) for l in range(L - 1))
+    # the shift changes the truncated estimates
+    a = O.highway_bp(O.postln_mlp_stack(W1, W2, gamma=0.8), c0, deltas, 2)[0]
+    b = O.highway_bp(base, c0, deltas, 2)[0]
+    assert np.linalg.norm(a - b) > 1e-3 * np.linalg.norm(b)
