@@ -81,7 +81,8 @@ typedef enum {
  *  POSTLN_MLP        Table 1, row "Transformer (Post-LN)" and Appendix C.3 with alpha = 1, beta = 0:
  *                    x' = LN(x + W2 gelu(W1 x)) = a(x) (.) x + b(x) with the row-wise gate a = 1 / sigma(x + Block(x)),
  *                    produced by hbp_forward; the block Jacobian is the rest of the layer's.  cfg.gate must be
- *                    HBP_GATE_ONE, cfg.gamma 0. */
+ *                    HBP_GATE_ONE.  cfg.gamma > 0 uses the shifted split of Appendix C.3, K = (1 - gamma) diag(a)
+ *                    (without a shift the truncated sums diverge on the directions LayerNorm removes). */
 typedef enum {
   HBP_BLOCK_MLP = 0, HBP_BLOCK_PRELN_MLP = 1, HBP_BLOCK_RNN_TANH = 2, HBP_BLOCK_PRELN_TRANSFORMER = 3, HBP_BLOCK_GRU = 4,
   HBP_BLOCK_LSTM = 5, HBP_BLOCK_RELU_MLP = 6, HBP_BLOCK_POSTLN_MLP = 7

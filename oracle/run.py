@@ -48,7 +48,7 @@ def build_stack(cfg, inputs, rows=None):
         x0 = _np(inputs["x0"] if rows is None else inputs["x0"][rows])
         groups = [("", l) for l in range(cfg.L)]
     elif cfg.block == "postln_mlp":
-        stack = O.postln_mlp_stack(F64Items(inputs["W1"]), F64Items(inputs["W2"]), cfg.ln_eps)
+        stack = O.postln_mlp_stack(F64Items(inputs["W1"]), F64Items(inputs["W2"]), cfg.ln_eps, cfg.gamma)
         x0 = _np(inputs["x0"] if rows is None else inputs["x0"][rows])
         groups = [("", l) for l in range(cfg.L)]
     elif cfg.block == "rnn_tanh":

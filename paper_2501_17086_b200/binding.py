@@ -123,7 +123,7 @@ def config_from_workload(w) -> hbp_config:
     gate = GATE_CHANNEL_SHARED if w.block == "rnn_tanh" else GATE_ONE
     loss = LOSS_EVERY_STEP if w.loss == "every_mse" else LOSS_FINAL
     return make_config(w.block, w.dtype, w.L, w.d, w.tokens, w.hidden, w.in_dim, w.n_heads, w.head_dim, w.seq,
-                       w.batch, gate, loss, w.ln_eps)
+                       w.batch, gate, loss, w.ln_eps, getattr(w, "gamma", 0.0))
 
 
 def workspace_bytes(cfg: hbp_config) -> int:

@@ -106,9 +106,8 @@ hbp_status check_config(const hbp_config* c) {
   if (c->d % v) return HBP_ERR_SHAPE;
   if (c->d / v > 1024) return HBP_ERR_SHAPE;  // one block per row in the LayerNorm kernels
   const bool gated_cell = c->block == HBP_BLOCK_GRU || c->block == HBP_BLOCK_LSTM;
-  if ((gated_cell || c->block == HBP_BLOCK_RELU_MLP || c->block == HBP_BLOCK_POSTLN_MLP) &&
-      (c->gate != HBP_GATE_ONE || c->gamma != 0.0f))
-    return HBP_ERR_UNSUPPORTED;
+  if ((gated_cell || c->block == HBP_BLOCK_RELU_MLP) && (c->gate != HBP_GATE_ONE || c->gamma != 0.0f)) return HBP_ERR_UNSUPPORTED;
+  if (c->block == HBP_BLOCK_POSTLN_MLP && c->gate != HBP_GATE_ONE) return HBP_ERR_UNSUPPORTED;
   // the 0/1 mask is a sign decision: taken in bf16 arithmetic it differs from an exact evaluation on the elements
   // that land near zero, and each such element changes its whole gradient path; float only
   if (c->block == HBP_BLOCK_RELU_MLP && c->dtype != HBP_F32) return HBP_ERR_UNSUPPORTED;

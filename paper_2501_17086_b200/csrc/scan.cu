@@ -90,7 +90,7 @@ __device__ __forceinline__ void scan_step(const ScanArgs& s, int l, int64_t stat
   constexpr int V = Vec<T>::N;
   const T* gp = gate_at<T>(s, l, state_elems, off, ch);
   if (s.gate == kGateRow) {  // one gate value per row and step (a float table [L][rows])
-    const float a = __ldg(s.row_gate + (int64_t)l * s.rows + off / s.d);
+    const float a = s.keep * __ldg(s.row_gate + (int64_t)l * s.rows + off / s.d);
 #pragma unroll
     for (int i = 0; i < V; ++i) val[i] = a * carry[i];
   } else if (gp) {
@@ -148,8 +148,10 @@ __global__ void __launch_bounds__(256) scan_depth_kernel(const ScanArgs s) {
     A val[V];
     scan_step<T>(s, l, state_elems, off, ch, carry, val);
     if (kShift) {
+      // the shifted part of the split acts on the previous iterate: gamma * a * g_{l+1} (a = 1 unless the gate is per row)
+      const float ga = s.gate == kGateRow ? s.gamma * __ldg(s.row_gate + (int64_t)l * s.rows + off / s.d) : s.gamma;
 #pragma unroll
-      for (int i = 0; i < V; ++i) val[i] += s.gamma * old_next[i];
+      for (int i = 0; i < V; ++i) val[i] += ga * old_next[i];
       ldv<T>(g + (int64_t)l * state_elems + off).get(old_next);  // before it is overwritten below
     }
     Vec<T> out;

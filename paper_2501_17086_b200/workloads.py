@@ -38,6 +38,7 @@ class Workload:
     seed: int = 0
     loss: str = "final_mse"   # "final_half_sse" | "final_mse" | "every_mse"
     ln_eps: float = 1e-5
+    gamma: float = 0.0    # shift of the residual split (post-LN workloads; Appendix C.3)
     init: str = ""        # MLP kinds: "fan_in" (variance 1/fan_in) or "small" (std 0.02, output weights 0.02/sqrt(2 steps));
                           # "" = the kind's default (fan_in for mlp / relu_mlp / postln_mlp, small for preln_mlp)
 
@@ -68,7 +69,7 @@ WORKLOADS = {
     "l1": Workload("l1", "lstm", "f32", L=256, d=1024, hidden=512, in_dim=212, batch=128, tokens=128, seed=1008, loss="every_mse"),
     # c2's shape with post-LN layers x <- LN(x + MLP(x)) (the RoBERTa-style row of Table 1)
     "p2": Workload("p2", "postln_mlp", "bf16", L=64, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1009,
-                   init="small"),
+                   init="small", gamma=0.8),
     # c2 with 8 layers: same per-launch tile shapes, small enough for multi-pass profiler captures
     "c2_small": Workload("c2_small", "preln_mlp", "bf16", L=8, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1012),
     # c4 with 4 decoder blocks: same per-launch shapes, small enough for multi-pass profiler captures
@@ -91,6 +92,10 @@ WORKLOADS = {
                                loss="every_mse"),
     "relu_twin": Workload("relu_twin", "relu_mlp", "f32", L=5, d=96, hidden=200, batch=1, seq=77, tokens=77, seed=2008),
     "postln_twin": Workload("postln_twin", "postln_mlp", "f32", L=5, d=96, hidden=200, batch=1, seq=77, tokens=77, seed=2009),
+    "postln_twin_shift": Workload("postln_twin_shift", "postln_mlp", "f32", L=5, d=96, hidden=200, batch=1, seq=77, tokens=77,
+                                  seed=2029, gamma=0.8),
+    "postln_twin_shift_bf16": Workload("postln_twin_shift_bf16", "postln_mlp", "bf16", L=6, d=128, hidden=512, batch=1, seq=200,
+                                       tokens=200, seed=2039, gamma=0.8),
     "postln_twin_bf16": Workload("postln_twin_bf16", "postln_mlp", "bf16", L=5, d=256, hidden=1024, batch=1, seq=328,
                                  tokens=328, seed=2019),
     "c4_twin": Workload("c4_twin", "preln_transformer", "bf16", L=2, d=128, hidden=512, n_heads=2, head_dim=64,

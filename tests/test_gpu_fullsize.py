@@ -74,8 +74,21 @@ def test_full_size_sampled_units(name, ks, rows):
 
     worst_x = max(rel(xs_gpu[l], ref["xs"][l]) for l in range(w.steps + 1))
     assert worst_x < tol, f"states: {worst_x:.3e}"
+
+    def worst_over_states(got_k, ref_k):
+        """Max per-state rel-L2; a state whose exact value lies below the range of float (a shifted split scales
+        each state by (1 - gamma) per step: 0.2^64 on p2) only has to be as small on the GPU."""
+        floor = 1e-30 * max(np.linalg.norm(r) for r in ref_k)
+        worst = 0.0
+        for l in range(w.steps + 1):
+            if np.linalg.norm(ref_k[l]) < floor:
+                assert np.linalg.norm(got_k[l]) <= floor, f"state {l} should have vanished"
+            else:
+                worst = max(worst, rel(got_k[l], ref_k[l]))
+        return worst
+
     for k in ks:
-        worst = max(rel(got[k][l], ref["hbp"][k][l]) for l in range(w.steps + 1))
+        worst = worst_over_states(got[k], ref["hbp"][k])
         assert worst < tol, f"k={k}: max rel-L2 {worst:.3e}"
     worst = max(rel(got["exact"][l], ref["exact"][l]) for l in range(w.steps + 1))
     tol_exact = TOL_EXACT_LONG_RNN if name == "c3" else tol

@@ -78,6 +78,8 @@ def compare(w, gpu, ref, ks, grads_for):
     ("relu_twin", (0, 1, 2, 5)),
     ("postln_twin", (0, 1, 2, 5)),
     ("postln_twin_bf16", (1, 2, 5)),
+    ("postln_twin_shift", (0, 1, 2, 5)),
+    ("postln_twin_shift_bf16", (1, 2, 6)),
 ])
 def test_twin_matches_oracle_in_full(name, ks):
     w = WORKLOADS[name]
