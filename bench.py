@@ -48,19 +48,19 @@ def config_of(w, k):
 # profiles/.  An entry is used only while the kernel's sources still hash to the value recorded with the capture and
 # the workload has the captured shapes; otherwise the bench line carries "traffic": null.
 TRAFFIC = {
-    # gemm_tc_kernel, VJP pair (dA + dY) on c2_small: 1243.126 MB + 894.741 MB for 8 layers x 8192 tokens
+    # gemm_tc_kernel, VJP pair (dA + dY) on c2_small: 1242.949 MB + 895.901 MB for 8 layers x 8192 tokens
     "gemm_vjp": {"sources": ("gemm_tc.cu", "tc_common.cuh"),
-                 "sha256": "c1bf7f31c6de2a40",
-                 "shape": ("preln_mlp", "bf16", 1024, 4096), "bytes_per_token_layer": (1243.126e6 + 894.741e6) / (8 * 8192),
+                 "sha256": "79b4e446ad5f9877",
+                 "shape": ("preln_mlp", "bf16", 1024, 4096), "bytes_per_token_layer": (1242.949e6 + 895.901e6) / (8 * 8192),
                  "profile": "profiles/gemm_tc_kernel_c2_small.md"},
-    # scan_depth_lnstat_kernel on c2_small: 286.272 MB read + 81.393 MB written for 8 steps x 8192 x 1024 elements
+    # scan_depth_lnstat_kernel on c2_small: 286.271 MB read + 80.891 MB written for 8 steps x 8192 x 1024 elements
     # (the writes still in L2 when that small launch ends are not in the counter)
-    "scan_lnstat": {"sources": ("scan.cu",), "sha256": "7f7fff07a1d164a0", "shape": ("preln_mlp", "bf16", 1024, 4096),
-                    "bytes_per_state_element_step": (286.272e6 + 81.393e6) / (8 * 8192 * 1024),
+    "scan_lnstat": {"sources": ("scan.cu",), "sha256": "08c908b07d964160", "shape": ("preln_mlp", "bf16", 1024, 4096),
+                    "bytes_per_state_element_step": (286.271e6 + 80.891e6) / (8 * 8192 * 1024),
                     "profile": "profiles/scan_depth_lnstat_kernel_c2_small.md"},
-    # scan_ring_kernel on c3: 268.520 MB read + 215.850 MB written per scan
-    "scan_ring": {"sources": ("scan_ring.cu", "tc_common.cuh"), "sha256": "ee364ca23032c441", "shape": ("rnn_tanh", "f32", 512, 0),
-                  "bytes_per_state_element_step": (268.520e6 + 215.850e6) / (4096 * 32 * 512),
+    # scan_ring_kernel on c3: 268.520 MB read + 217.638 MB written per scan
+    "scan_ring": {"sources": ("scan_ring.cu", "tc_common.cuh"), "sha256": "edb684e7b31e74f9", "shape": ("rnn_tanh", "f32", 512, 0),
+                  "bytes_per_state_element_step": (268.520e6 + 217.638e6) / (4096 * 32 * 512),
                   "profile": "profiles/scan_ring_kernel_c3.md"},
 }
 
