@@ -362,6 +362,22 @@ def run_ours(args):
         fn = lambda: ctx.exact(params, delta, x_all, xin, g_all=g_all, grads=grads)
         fn()
         detail["exact_bp_ms"] = timed_local(torch, fn, 3)
+        # the same step replayed from a CUDA graph (the calls only enqueue and never allocate): what launch overhead
+        # costs on the small workloads
+        try:
+            graph = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(graph, stream=side):
+                    ctx.backward(params, k, delta, x_all, xin, g_all=g_all, grads=grads)
+            torch.cuda.synchronize()
+            graph.replay()
+            detail["graph_replay_ms"] = timed_local(torch, graph.replay, 5)
+            del graph
+        except Exception as e:  # capture is a convenience of the host runtime: report, do not fail the bench
+            detail["graph_replay_ms"] = None
+            detail["graph_error"] = str(e)[:200]
         # Figure 5's quantity on this synthetic workload: cosine similarity of the k-iteration estimate with the
         # exact gradient, per state, computed on the device (hbp_compare); minimum and median over the states
         try:

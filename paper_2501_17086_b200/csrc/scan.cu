@@ -86,11 +86,12 @@ __device__ __forceinline__ const T* gate_at(const ScanArgs& s, int l, int64_t st
 // One step of the recurrence for a 16-byte channel group: val = a * carry + u + delta.
 template <typename T>
 __device__ __forceinline__ void scan_step(const ScanArgs& s, int l, int64_t state_elems, int64_t off, int ch,
-                                          const typename Acc<T>::type* carry, typename Acc<T>::type* val) {
+                                          const typename Acc<T>::type* carry, typename Acc<T>::type* val,
+                                          int64_t row = 0) {
   constexpr int V = Vec<T>::N;
   const T* gp = gate_at<T>(s, l, state_elems, off, ch);
   if (s.gate == kGateRow) {  // one gate value per row and step (a float table [L][rows])
-    const float a = s.keep * __ldg(s.row_gate + (int64_t)l * s.rows + off / s.d);
+    const float a = s.keep * __ldg(s.row_gate + (int64_t)l * s.rows + row);
 #pragma unroll
     for (int i = 0; i < V; ++i) val[i] = a * carry[i];
   } else if (gp) {
@@ -134,7 +135,8 @@ __global__ void __launch_bounds__(256) scan_depth_kernel(const ScanArgs s) {
   const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (v >= nvec) return;
   const int64_t off = v * V;
-  const int ch = (int)(off % s.d);
+  const int64_t row = off / s.d;  // once per thread: the per-row gate of post-LN layers is looked up by it
+  const int ch = (int)(off - row * s.d);
   T* g = (T*)s.g;
   typedef typename Acc<T>::type A;
   A carry[V];
@@ -146,10 +148,10 @@ __global__ void __launch_bounds__(256) scan_depth_kernel(const ScanArgs s) {
   }
   for (int l = s.l_hi - 1; l >= s.l_lo; --l) {
     A val[V];
-    scan_step<T>(s, l, state_elems, off, ch, carry, val);
+    scan_step<T>(s, l, state_elems, off, ch, carry, val, row);
     if (kShift) {
       // the shifted part of the split acts on the previous iterate: gamma * a * g_{l+1} (a = 1 unless the gate is per row)
-      const float ga = s.gate == kGateRow ? s.gamma * __ldg(s.row_gate + (int64_t)l * s.rows + off / s.d) : s.gamma;
+      const float ga = s.gate == kGateRow ? s.gamma * __ldg(s.row_gate + (int64_t)l * s.rows + row) : s.gamma;
 #pragma unroll
       for (int i = 0; i < V; ++i) val[i] += ga * old_next[i];
       ldv<T>(g + (int64_t)l * state_elems + off).get(old_next);  // before it is overwritten below

@@ -251,3 +251,44 @@ def test_layer_parallel_shards_match_the_single_context_and_the_oracle(name, wor
         for n, t in grads.items():
             want = ref["grads"][k][n[1:]][s.lo:s.hi]
             assert rel(np64(t), want) < tol, f"rank {s.rank} {n}"
+
+
+@pytest.mark.parametrize("name,k", [("gru_twin_long", 3), ("c2_twin", 2), ("c4_twin", 2)])
+def test_backward_replays_from_a_cuda_graph(name, k):
+    """The calls only enqueue work on the given stream and allocate nothing, so a backward (after one eager call
+    that does the one-time kernel attribute set-up) can be captured into a CUDA graph and replayed on new data in the
+    same buffers: the replay must reproduce the eager result bit for bit."""
+    from paper_2501_17086_b200 import harness
+    from paper_2501_17086_b200.workloads import WORKLOADS, make_inputs
+    w = WORKLOADS[name]
+    inp = make_inputs(w, "cuda")
+    ctx = harness.make_context(w)
+    params = harness.params_for(w, inp)
+    xin = harness.rnn_inputs(w, inp)
+    x_all = ctx.forward(params, inp["x0"], xin)
+    delta = harness.loss_delta(w, x_all, inp).contiguous()
+    g_all, grads = ctx.new_states(), ctx.new_grads()
+    ctx.backward(params, k, delta, x_all, xin, g_all=g_all, grads=grads)       # eager: also the one-time set-up
+    torch.cuda.synchronize()
+    want_g, want_w = g_all.clone(), {n: t.clone() for n, t in grads.items()}
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            ctx.backward(params, k, delta, x_all, xin, g_all=g_all, grads=grads)
+    g_all.zero_()
+    for t in grads.values():
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    ctx.sync_status()
+    assert torch.equal(g_all, want_g)
+    for n in grads:
+        assert torch.equal(grads[n], want_w[n]), n
+    delta2 = (delta.float() * 0.5).to(delta.dtype)
+    want2 = ctx.backward(params, k, delta2, x_all, xin).clone()
+    delta.copy_(delta2)                      # new data in the captured buffer
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(g_all, want2)
