@@ -381,7 +381,7 @@ def run_ours(args):
         # Figure 5's quantity on this synthetic workload: cosine similarity of the k-iteration estimate with the
         # exact gradient, per state, computed on the device (hbp_compare); minimum and median over the states
         try:
-            g_exact = g_all.clone()
+            g_exact = ctx.exact(params, delta, x_all, xin, g_all=g_all).clone()
             cos = {}
             for kx in (1, 2, 4, 8):
                 ctx.backward(params, kx, delta, x_all, xin, g_all=g_all, grads=None)
