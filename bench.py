@@ -53,10 +53,10 @@ TRAFFIC = {
                  "sha256": "79b4e446ad5f9877",
                  "shape": ("preln_mlp", "bf16", 1024, 4096), "bytes_per_token_layer": (1242.949e6 + 895.901e6) / (8 * 8192),
                  "profile": "profiles/gemm_tc_kernel_c2_small.md"},
-    # scan_depth_lnstat_kernel on c2_small: 286.271 MB read + 80.891 MB written for 8 steps x 8192 x 1024 elements
+    # scan_depth_lnstat_kernel on c2_small: 286.271 MB read + 80.401 MB written for 8 steps x 8192 x 1024 elements
     # (the writes still in L2 when that small launch ends are not in the counter)
-    "scan_lnstat": {"sources": ("scan.cu",), "sha256": "08c908b07d964160", "shape": ("preln_mlp", "bf16", 1024, 4096),
-                    "bytes_per_state_element_step": (286.271e6 + 80.891e6) / (8 * 8192 * 1024),
+    "scan_lnstat": {"sources": ("scan.cu",), "sha256": "5efee60609bc121d", "shape": ("preln_mlp", "bf16", 1024, 4096),
+                    "bytes_per_state_element_step": (286.271e6 + 80.401e6) / (8 * 8192 * 1024),
                     "profile": "profiles/scan_depth_lnstat_kernel_c2_small.md"},
     # scan_ring_kernel on c3: 268.520 MB read + 217.638 MB written per scan
     "scan_ring": {"sources": ("scan_ring.cu", "tc_common.cuh"), "sha256": "edb684e7b31e74f9", "shape": ("rnn_tanh", "f32", 512, 0),
@@ -320,6 +320,8 @@ def run_ours(args):
                     "peak_source": "of measured bf16 x nominal tf32/bf16 ratio" if peaks else "of fallback", "traffic": None}
     # scan: read u (+ xhat when the LayerNorm finish is fused, + the per-element gate of a GRU), write g
     tensors = 2 + (1 if w.block in ("preln_mlp", "preln_transformer", "gru", "lstm") else 0)  # per-step delta is added by the VJP GEMM epilogue
+    if w.block == "postln_mlp":  # u, the non-block part c, g written; + the previous iterate when the split is shifted
+        tensors = 3 + (1 if getattr(w, "gamma", 0.0) else 0)
     scan_bytes = tensors * w.steps * w.tokens * w.d * es
     hbm = peaks.get("hbm_gbs", 6650.0)
     scan_iter_ms = None
