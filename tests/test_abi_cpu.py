@@ -82,3 +82,23 @@ def test_relu_residual_kind_is_float_only(B):
     bad = B.make_config("relu_mlp", "bf16", 4, 64, 32, hidden=128)
     assert B.lib.hbp_workspace_bytes(C.byref(ok), C.byref(n)) == 0 and n.value > 0
     assert B.lib.hbp_workspace_bytes(C.byref(bad), C.byref(n)) == 6
+
+
+def test_new_entry_points_reject_bad_arguments_without_a_gpu(B):
+    lib = B.lib
+    assert lib.hbp_iterate(None, None, None, None, None, None, None) == 1
+    assert lib.hbp_param_grads(None, None, None, None, None, None, None) == 1
+    assert lib.hbp_add_carry(None, None, None, None) == 1
+    assert lib.hbp_compare(7, 1, 8, None, None, None, None, 0, None) == 3      # dtype
+    assert lib.hbp_compare(0, 0, 8, None, None, None, None, 0, None) == 2      # no segments
+    assert lib.hbp_compare(0, 1, 8, None, None, None, None, 0, None) == 1      # null tensors
+    assert lib.hbp_compare_scratch_bytes(3) == 3 * 64 * 4 * 8
+    n = C.c_size_t()
+    for block, kw in (("gru", dict(in_dim=8, batch=4)), ("lstm", dict(hidden=32, in_dim=8, batch=4)),
+                      ("postln_mlp", dict(hidden=128))):
+        cfg = B.make_config(block, "f32", 6, 64, 4, **kw)
+        assert lib.hbp_workspace_bytes(C.byref(cfg), C.byref(n)) == 0 and n.value > 0, block
+    bad = B.make_config("lstm", "f32", 6, 64, 4, hidden=20, in_dim=8, batch=4)   # hidden must be d / 2
+    assert lib.hbp_workspace_bytes(C.byref(bad), C.byref(n)) == 2
+    gated = B.make_config("gru", "f32", 6, 64, 4, in_dim=8, batch=4, gate=B.GATE_CHANNEL_SHARED)
+    assert lib.hbp_workspace_bytes(C.byref(gated), C.byref(n)) == 6              # the cell's gate is the only one
