@@ -984,7 +984,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
   r.inputs = (const char*)inputs;
   r.g = (char*)g_all;
   r.delta = (const char*)delta;
-  const int steps = ctx->steps, layers = ctx->layers, grp = ctx->group;
+  const int steps = ctx->steps;
   const bool tr = f.block == HBP_BLOCK_PRELN_TRANSFORMER, rnn = f.block == HBP_BLOCK_RNN_TANH;
   const bool gru = f.block == HBP_BLOCK_GRU;
   {
