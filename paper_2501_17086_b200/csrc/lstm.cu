@@ -106,7 +106,6 @@ __global__ void __launch_bounds__(256) lstm_step_kernel(const T* __restrict__ W,
 
 __device__ __forceinline__ double as_d(double v) { return v; }
 __device__ __forceinline__ double as_d(float v) { return (double)v; }
-__device__ __forceinline__ double as_d(bf16 v) { return (double)to_f(v); }
 
 // element (row, column k of the [4u] operand) from the upstream gradient [g_c | g_h] and the coefficients
 // (C = the type to compute in: double for exact backpropagation, float for GEMM operands)
