@@ -133,31 +133,18 @@ __device__ __forceinline__ double as_double(double v) { return v; }
 __device__ __forceinline__ double as_double(float v) { return (double)v; }
 __device__ __forceinline__ double as_double(bf16 v) { return (double)to_f(v); }
 
-// dst[r * lda + col0 + c] = src[(r0 + r) * ld + c] as double for r < nrows, c < ncols (zero where r0 + r >= rmax); eight
-// loads per thread are issued before the first store, so that a block has its whole tile in flight at once
-template <typename S>
+// dst[r * lda + col0 + c] = src[(r0 + r) * ld + c] as double for r < R, c < ncols (zero where r0 + r >= rmax).  A thread
+// walks columns and issues the loads of all R rows of a column before the first store: the block has its whole tile in
+// flight at once, and no index needs a division.
+template <int R, typename S>
 __device__ __forceinline__ void stage_tile(double* __restrict__ dst, int lda, int col0, const S* __restrict__ src, int64_t ld,
-                                           int r0, int rmax, int nrows, int ncols) {
-  const int total = nrows * ncols;
-  for (int base = threadIdx.x; base < total; base += 8 * blockDim.x) {
-    double v[8];
+                                           int r0, int rmax, int ncols) {
+  for (int c = threadIdx.x; c < ncols; c += blockDim.x) {
+    double v[R];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int idx = base + j * blockDim.x;
-      v[j] = 0.0;
-      if (idx < total) {
-        const int r = idx / ncols, c = idx - r * ncols;
-        if (r0 + r < rmax) v[j] = as_double(src[(int64_t)(r0 + r) * ld + c]);
-      }
-    }
+    for (int r = 0; r < R; ++r) v[r] = r0 + r < rmax ? as_double(src[(int64_t)(r0 + r) * ld + c]) : 0.0;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int idx = base + j * blockDim.x;
-      if (idx < total) {
-        const int r = idx / ncols, c = idx - r * ncols;
-        dst[r * lda + col0 + c] = v[j];
-      }
-    }
+    for (int r = 0; r < R; ++r) dst[r * lda + col0 + c] = v[r];
   }
 }
 
@@ -172,10 +159,10 @@ __global__ void __launch_bounds__(256) rnn_step_staged_kernel(const T* __restric
   double* As = sm;                     // [kSRows][lda]: h | x_t
   double* Ws = sm + kSRows * lda;      // [kSCols][lda]: W row | U row
   const int n0 = blockIdx.x * kSCols, m0 = blockIdx.y * kSRows;
-  stage_tile<double>(As, lda, 0, h_in, d, m0, B, kSRows, d);
-  stage_tile<T>(As, lda, d, x_t, in_dim, m0, B, kSRows, in_dim);
-  stage_tile<T>(Ws, lda, 0, W, d, n0, d, kSCols, d);
-  stage_tile<T>(Ws, lda, d, U, in_dim, n0, d, kSCols, in_dim);
+  stage_tile<kSRows, double>(As, lda, 0, h_in, d, m0, B, d);
+  stage_tile<kSRows, T>(As, lda, d, x_t, in_dim, m0, B, in_dim);
+  stage_tile<kSCols, T>(Ws, lda, 0, W, d, n0, d, d);
+  stage_tile<kSCols, T>(Ws, lda, d, U, in_dim, n0, d, in_dim);
   __syncthreads();
   const int o = threadIdx.x >> 1, half = threadIdx.x & 1, m = o / kSCols, c = o % kSCols;
   double z = dot_halves(As + m * lda, Ws + c * lda, ktot, half);
@@ -203,10 +190,17 @@ __global__ void __launch_bounds__(256) rnn_bwd_step_staged_kernel(const T* __res
   double* As = sm;                   // [kSRows][lda]: g_{t+1} * tanh'(z_t)
   double* Ws = sm + kSRows * lda;    // [kSCols][lda]: columns n0.. of W, one per row here
   const int n0 = blockIdx.x * kSCols, m0 = blockIdx.y * kSRows;
-#pragma unroll 8
-  for (int idx = threadIdx.x; idx < kSRows * d; idx += blockDim.x) {
-    const int m = idx / d, k = idx - m * d, gm = m0 + m;
-    As[m * lda + k] = gm < B ? g_in[(int64_t)gm * d + k] * (double)to_f(deriv[(int64_t)gm * d + k]) : 0.0;
+  for (int k = threadIdx.x; k < d; k += blockDim.x) {  // all rows of a column in flight before the first store
+    double gv[kSRows];
+    float dv[kSRows];
+#pragma unroll
+    for (int m = 0; m < kSRows; ++m) {
+      const bool okm = m0 + m < B;
+      gv[m] = okm ? g_in[(int64_t)(m0 + m) * d + k] : 0.0;
+      dv[m] = okm ? to_f(deriv[(int64_t)(m0 + m) * d + k]) : 0.0f;
+    }
+#pragma unroll
+    for (int m = 0; m < kSRows; ++m) As[m * lda + k] = gv[m] * (double)dv[m];
   }
 #pragma unroll 8
   for (int idx = threadIdx.x; idx < kSCols * d; idx += blockDim.x) {
