@@ -21,17 +21,34 @@ __device__ __forceinline__ void lstm_accumulate(const void* __restrict__ src, in
                                                 int kdim, int B, int u, int m0, int n0, double (*Hs)[kTile + 1],
                                                 float (*Ws)[kTile][kTile + 1], double acc[4][4]) {
   const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
-  for (int k0 = 0; k0 < kdim; k0 += kTile) {
-    for (int i = ty; i < kTile; i += 8) {
+  // The next tile's global loads are issued into registers before the current tile is multiplied, so the loop
+  // waits for memory once, not once per tile.
+  double hreg[4];
+  float wreg[4][4];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = ty + 8 * j;
       const int k = k0 + tx, m = m0 + i, n = n0 + i;
       double hv = 0.0;
       if (k < kdim && m < B)
         hv = kSrcDouble ? ((const double*)src)[(int64_t)m * src_ld + k] : (double)to_f(((const T*)src)[(int64_t)m * src_ld + k]);
-      Hs[i][tx] = hv;
+      hreg[j] = hv;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) Ws[q][i][tx] = (k < kdim && n < u) ? to_f(Wm[((int64_t)q * u + n) * kdim + k]) : 0.0f;
+      for (int q = 0; q < 4; ++q) wreg[q][j] = (k < kdim && n < u) ? to_f(Wm[((int64_t)q * u + n) * kdim + k]) : 0.0f;
+    }
+  };
+  fetch(0);
+  for (int k0 = 0; k0 < kdim; k0 += kTile) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = ty + 8 * j;
+      Hs[i][tx] = hreg[j];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) Ws[q][i][tx] = wreg[q][j];
     }
     __syncthreads();
+    if (k0 + kTile < kdim) fetch(k0 + kTile);
 #pragma unroll 8
     for (int kk = 0; kk < kTile; ++kk) {
       double w[4];
