@@ -128,15 +128,32 @@ __global__ void __launch_bounds__(256) gru_bwd_step_kernel(const T* __restrict__
   const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
   const int n0 = blockIdx.x * kTile, m0 = blockIdx.y * kTile;
   double acc[4] = {0.0, 0.0, 0.0, 0.0};
-  for (int q = 0; q < 3; ++q) {
-    for (int k0 = 0; k0 < d; k0 += kTile) {
-      for (int i = ty; i < kTile; i += 8) {
-        const int m = m0 + i, k = k0 + tx;
-        Hs[i][tx] = (m < B && k < d) ? g_in[(int64_t)m * d + k] * (double)to_f(c4[(int64_t)m * 4 * d + (int64_t)q * d + k]) : 0.0;
-        const int kk = k0 + i, n = n0 + tx;  // W[q*d + k][n]: contiguous in n
-        Ws[tx][i] = (kk < d && n < d) ? to_f(W[((int64_t)q * d + kk) * d + n]) : 0.0f;
+  // the next tile's operands are fetched into registers before the current tile is multiplied; tiles are numbered
+  // through the three gate blocks
+  const int tiles_per_gate = (d + kTile - 1) / kTile, ntiles = 3 * tiles_per_gate;
+  double hreg[4];
+  float wreg[4];
+  auto fetch = [&](int t) {
+    const int q = t / tiles_per_gate, k0 = (t - q * tiles_per_gate) * kTile;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = ty + 8 * j;
+      const int m = m0 + i, k = k0 + tx;
+      hreg[j] = (m < B && k < d) ? g_in[(int64_t)m * d + k] * (double)to_f(c4[(int64_t)m * 4 * d + (int64_t)q * d + k]) : 0.0;
+      const int kk = k0 + i, n = n0 + tx;  // W[q*d + k][n]: contiguous in n
+      wreg[j] = (kk < d && n < d) ? to_f(W[((int64_t)q * d + kk) * d + n]) : 0.0f;
+    }
+  };
+  fetch(0);
+  {
+    for (int t = 0; t < ntiles; ++t) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        Hs[ty + 8 * j][tx] = hreg[j];
+        Ws[tx][ty + 8 * j] = wreg[j];
       }
       __syncthreads();
+      if (t + 1 < ntiles) fetch(t + 1);
 #pragma unroll
       for (int kk = 0; kk < kTile; ++kk) {
         const double w = (double)Ws[tx][kk];

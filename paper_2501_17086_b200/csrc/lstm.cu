@@ -157,14 +157,28 @@ __global__ void __launch_bounds__(256) lstm_bwd_step_kernel(const T* __restrict_
   const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
   const int n0 = blockIdx.x * kTile, m0 = blockIdx.y * kTile;
   double acc[4] = {0.0, 0.0, 0.0, 0.0};
-  for (int k0 = 0; k0 < 4 * u; k0 += kTile) {  // u is a multiple of 4, not of the tile: blocks may straddle gates
-    for (int i = ty; i < kTile; i += 8) {
+  // the next tile's operands are fetched into registers before the current tile is multiplied
+  double hreg[4];
+  float wreg[4];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = ty + 8 * j;
       const int m = m0 + i, k = k0 + tx;
-      Hs[i][tx] = (m < B && k < 4 * u) ? operand_value<double, T, double>(g_in + (int64_t)m * 2 * u, c5 + (int64_t)m * 5 * u, u, k) : 0.0;
+      hreg[j] = (m < B && k < 4 * u) ? operand_value<double, T, double>(g_in + (int64_t)m * 2 * u, c5 + (int64_t)m * 5 * u, u, k) : 0.0;
       const int kk = k0 + i, n = n0 + tx;  // W[k][n]: contiguous in n
-      Ws[tx][i] = (kk < 4 * u && n < u) ? to_f(W[(int64_t)kk * u + n]) : 0.0f;
+      wreg[j] = (kk < 4 * u && n < u) ? to_f(W[(int64_t)kk * u + n]) : 0.0f;
+    }
+  };
+  fetch(0);
+  for (int k0 = 0; k0 < 4 * u; k0 += kTile) {  // u is a multiple of 4, not of the tile: blocks may straddle gates
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      Hs[ty + 8 * j][tx] = hreg[j];
+      Ws[tx][ty + 8 * j] = wreg[j];
     }
     __syncthreads();
+    if (k0 + kTile < 4 * u) fetch(k0 + kTile);
 #pragma unroll
     for (int kk = 0; kk < kTile; ++kk) {
       const double w = (double)Ws[tx][kk];
