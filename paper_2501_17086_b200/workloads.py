@@ -180,4 +180,6 @@ def make_inputs(cfg: Workload, device="cpu"):
         out["y"] = _randn(gen, (N, d), 1.0, dev).to(dt)
     else:
         raise ValueError(f"unknown block kind {cfg.block!r}")
+    if "Y" in out:
+        out["y"] = out["Y"][-1]  # target of the last state, for recurrent workloads with a loss on the last state only
     return out

@@ -49,10 +49,23 @@ def compare(w, gpu, ref, ks, grads_for):
     shape = ref["xs"][0].shape
     for l in range(steps + 1):
         assert rel_l2(to_np(gpu["x"][l]), ref["xs"][l]) < tol, f"state {l}"
+    def worst_over_states(got, want):
+        """Max per-state rel-L2.  A state whose exact value lies below the normal range of float (products of many
+        gates below one, with a loss on the last state only) cannot be held to a relative bound: it only has to be
+        as small on the GPU."""
+        floor = 1e-30 * max(np.linalg.norm(r) for r in want)
+        worst = 0.0
+        for l in range(steps + 1):
+            if np.linalg.norm(want[l]) < floor:
+                assert np.linalg.norm(to_np(got[l])) <= floor, f"state {l} should have vanished"
+            else:
+                worst = max(worst, rel_l2(to_np(got[l]), want[l]))
+        return worst
+
     for k in ks:
-        worst = max(rel_l2(to_np(gpu["hbp"][k][l]), ref["hbp"][k][l]) for l in range(steps + 1))
+        worst = worst_over_states(gpu["hbp"][k], ref["hbp"][k])
         assert worst < tol, f"k={k}: max rel-L2 {worst:.3e}"
-    worst = max(rel_l2(to_np(gpu["exact"][l]), ref["exact"][l]) for l in range(steps + 1))
+    worst = worst_over_states(gpu["exact"], ref["exact"])
     assert worst < tol, f"exact: max rel-L2 {worst:.3e}"
     for key in grads_for:
         for name, val in ref["grads"][key].items():

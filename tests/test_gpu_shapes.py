@@ -18,7 +18,10 @@ def _case(seed):
     dtype = rnd.choice(["f32", "bf16"])
     v = 4 if dtype == "f32" else 8
     block = rnd.choice(["mlp", "preln_mlp", "rnn_tanh", "gru", "lstm", "preln_transformer"])
-    if seed >= 42:   # the post-LN kind, both dtypes
+    if seed >= 50:   # recurrent kinds, loss on the last state only; float: with gates stored in bf16 the product of a
+        # hundred of them carries sqrt(100) * 2^-9 of relative error by itself, beyond the 2e-2 bar
+        block, dtype, v = ("rnn_tanh", "gru", "lstm")[seed % 3], "f32", 4
+    elif seed >= 42:   # the post-LN kind, both dtypes
         block = "postln_mlp"
     elif seed >= 36:   # later seeds: the ReLU-residual kind (added after the first 36 cases were fixed)
         block, dtype, v = "relu_mlp", "f32", 4
@@ -33,15 +36,18 @@ def _case(seed):
         return Workload(f"rand{seed}", block, dtype, L=rnd.randint(1, 2), d=heads * hd, hidden=mult(8, 260), n_heads=heads,
                         head_dim=hd, seq=seq, batch=batch, tokens=batch * seq, seed=5000 + seed)
     T, B, nin = rnd.randint(1, 150), rnd.randint(1, 40), mult(8, 40)
+    loss = "final_mse" if seed >= 50 else "every_mse"   # the last seeds: recurrent kinds with a loss on the last state only
+    if seed >= 50:
+        T = max(T, 70)                                   # long enough for the time scans
     if block == "lstm":
         u = mult(8, 100)
         return Workload(f"rand{seed}", block, dtype, L=T, d=2 * u, hidden=u, in_dim=nin, batch=B, tokens=B,
-                        seed=5000 + seed, loss="every_mse")
+                        seed=5000 + seed, loss=loss)
     return Workload(f"rand{seed}", block, dtype, L=T, d=mult(8, 200), in_dim=nin, batch=B, tokens=B, seed=5000 + seed,
-                    loss="every_mse")
+                    loss=loss)
 
 
-@pytest.mark.parametrize("seed", range(50))
+@pytest.mark.parametrize("seed", range(59))
 def test_random_shape_matches_oracle(seed):
     w = _case(seed)
     rnd = random.Random(1000 + seed)
