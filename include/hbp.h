@@ -184,11 +184,18 @@ hbp_status hbp_param_grads(hbp_ctx* ctx, const hbp_params* params, const void* x
 /* Eq. 9 / Eq. 12 on its own: g[L] = delta_L and g[l] = delta_l + a_l (.) g[l+1] + u[l] for l = L-1..0,
  * i.e. the reverse CumSumProd with diagonal K.  u [L][rows][d] (NULL = zeros), delta as in hbp_loss
  * (`loss`), a as in hbp_gate (`gate`), g [L+1][rows][d].  `scratch` is device memory of at least
- * hbp_cumsumprod_scratch_bytes(...) bytes (may be NULL when that is 0). */
+ * hbp_cumsumprod_scratch_bytes(...) bytes (may be NULL when that is 0).
+ * hbp_cumsumprod_status is the same call with a device status word: `status` (device, one int, 4-byte aligned) is
+ * where a kernel of the scan records HBP_ERR_TIMEOUT if one of its bounded waits gives up; the caller zeroes it
+ * beforehand and reads it once the stream has finished.  hbp_cumsumprod (and hbp_cumsumprod_static) have no such
+ * word: there a wait that gives up still ends the kernel, but goes unreported and leaves g partly unwritten. */
 hbp_status hbp_cumsumprod_scratch_bytes(int32_t dtype, int32_t L, int64_t rows, int32_t d, size_t* bytes);
 hbp_status hbp_cumsumprod(int32_t dtype, int32_t gate, int32_t loss, int32_t L, int64_t rows, int32_t d,
                           const void* u, const void* delta, const void* a, void* g,
                           void* scratch, size_t scratch_bytes, void* cuda_stream);
+hbp_status hbp_cumsumprod_status(int32_t dtype, int32_t gate, int32_t loss, int32_t L, int64_t rows, int32_t d,
+                                 const void* u, const void* delta, const void* a, void* g,
+                                 void* scratch, size_t scratch_bytes, int32_t* status, void* cuda_stream);
 
 /* The same scan for callers that cannot allocate device memory.  (The paper has no counterpart: this is a
  * packaging variant of hbp_cumsumprod, not a step of the method.)  Some hosts hand all device memory to
@@ -231,6 +238,13 @@ hbp_status hbp_profile_read(hbp_ctx* ctx, float* ms, int64_t* launches);
 
 /* Number of kernels this context has launched since creation (host counter). */
 int64_t hbp_launch_count(const hbp_ctx* ctx);
+
+/* Kernel-selection modes of a context, fixed when it was created from the environment of that moment:
+ * bit 0 = HBP_FORCE_SIMT=1 (every contraction on the CUDA-core kernels, a cross-check of the tensor-core ones),
+ * bit 1 = HBP_GEMM_PAIR=1 (the tensor-core GEMM pairs CTAs).  The modes belong to the context: contexts created
+ * under other settings, before or after, keep their own.  One-time kernel set-up is likewise remembered per
+ * device, so one process may hold contexts on several GPUs (each used with its device current). */
+int32_t hbp_context_modes(const hbp_ctx* ctx);
 
 const char* hbp_status_string(hbp_status s);
 void hbp_destroy(hbp_ctx* ctx);

@@ -114,8 +114,10 @@ def run(cfg, inputs, ks=(), rows=None, exact=True, grads_for=(), timing=None):
         if "exact" in grads_for:
             out["grads"]["exact"] = O.param_grads(stack, caches, xs, out["exact"], groups)
     t2 = time.perf_counter()
+    # one run to the largest k: iterate j of that run IS Highway-BP with k = j (each iteration starts from the previous one)
+    history = O.highway_bp(stack, caches, deltas, max(ks), return_all=True) if ks else []
     for k in ks:
-        out["hbp"][k] = O.highway_bp(stack, caches, deltas, k)
+        out["hbp"][k] = history[k]
         if k in grads_for:
             out["grads"][k] = O.param_grads(stack, caches, xs, out["hbp"][k], groups)
     t3 = time.perf_counter()

@@ -20,7 +20,8 @@ GATE_ONE, GATE_CHANNEL_SHARED, GATE_CHANNEL_PER_STEP = 0, 1, 2
 LOSS_FINAL, LOSS_EVERY_STEP = 0, 1
 
 EXPORTS = ["hbp_workspace_bytes", "hbp_create", "hbp_forward", "hbp_backward", "hbp_exact",
-           "hbp_cumsumprod_scratch_bytes", "hbp_cumsumprod", "hbp_sync_status", "hbp_launch_count",
+           "hbp_cumsumprod_scratch_bytes", "hbp_cumsumprod", "hbp_cumsumprod_status", "hbp_sync_status", "hbp_launch_count",
+           "hbp_context_modes",
            "hbp_profile_enable", "hbp_profile_read", "hbp_cumsumprod_static", "hbp_cumsumprod_static_max_bytes",
            "hbp_compare_scratch_bytes", "hbp_compare", "hbp_iterate", "hbp_add_carry", "hbp_param_grads",
            "hbp_status_string", "hbp_destroy"]
@@ -60,6 +61,9 @@ def _load():
     lib.hbp_exact.argtypes = [vp, C.POINTER(hbp_params), vp, vp, vp, vp, C.POINTER(hbp_grads), vp]
     lib.hbp_cumsumprod_scratch_bytes.argtypes = [i32, i32, i64, i32, C.POINTER(sz)]
     lib.hbp_cumsumprod.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.hbp_cumsumprod_status.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.hbp_context_modes.argtypes = [vp]
+    lib.hbp_context_modes.restype = i32
     lib.hbp_cumsumprod_static.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp]
     lib.hbp_cumsumprod_static_max_bytes.argtypes = []
     lib.hbp_iterate.argtypes = [vp, C.POINTER(hbp_params), vp, vp, vp, vp, vp]
@@ -79,7 +83,7 @@ def _load():
     for name in EXPORTS:
         if name in ("hbp_cumsumprod_static_max_bytes", "hbp_compare_scratch_bytes"):
             getattr(lib, name).restype = sz
-        elif name not in ("hbp_launch_count", "hbp_status_string", "hbp_destroy"):
+        elif name not in ("hbp_launch_count", "hbp_status_string", "hbp_destroy", "hbp_context_modes"):
             getattr(lib, name).restype = C.c_int
     return lib
 
@@ -160,6 +164,11 @@ class Context:
         _check(lib.hbp_create(C.byref(cfg), C.c_void_p(base), nbytes, C.byref(handle)), "hbp_create")
         self._h = handle
         self._keep = None
+
+    @property
+    def modes(self) -> int:
+        """Bit 0: CUDA-core kernels forced; bit 1: paired-CTA GEMM.  Fixed at creation, per context."""
+        return int(lib.hbp_context_modes(self._h))
 
     def close(self):
         if self._h is not None:
@@ -265,8 +274,9 @@ def cumsumprod_scratch_bytes(dtype, L, rows, d) -> int:
     return n.value
 
 
-def cumsumprod(u, delta, a=None, gate=None, loss=LOSS_FINAL, g=None, scratch=None):
-    """g[L] = delta_L, g[l] = delta_l + a_l * g[l+1] + u[l]; u is [L, rows, d] (or None with ``g`` given)."""
+def cumsumprod(u, delta, a=None, gate=None, loss=LOSS_FINAL, g=None, scratch=None, status=None):
+    """g[L] = delta_L, g[l] = delta_l + a_l * g[l+1] + u[l]; u is [L, rows, d] (or None with ``g`` given).
+    ``status``: an int32 device tensor (zeroed by the caller) that receives a kernel's error code, if any."""
     ref = u if u is not None else g
     L = ref.shape[0] - (0 if u is not None else 1)
     rows, d = ref.shape[1], ref.shape[2]
@@ -277,8 +287,13 @@ def cumsumprod(u, delta, a=None, gate=None, loss=LOSS_FINAL, g=None, scratch=Non
     need = cumsumprod_scratch_bytes(ref.dtype, L, rows, d)
     if scratch is None and need:
         scratch = torch.empty(need, dtype=torch.uint8, device=ref.device)
+    nbytes = 0 if scratch is None else scratch.numel()
+    if status is not None:
+        _check(lib.hbp_cumsumprod_status(_dtype_code(ref.dtype), gate, loss, L, rows, d, _ptr(u), _ptr(delta), _ptr(a),
+                                         _ptr(g), _ptr(scratch), nbytes, _ptr(status), _stream()), "hbp_cumsumprod_status")
+        return g
     _check(lib.hbp_cumsumprod(_dtype_code(ref.dtype), gate, loss, L, rows, d, _ptr(u), _ptr(delta), _ptr(a), _ptr(g),
-                              _ptr(scratch), 0 if scratch is None else scratch.numel(), _stream()), "hbp_cumsumprod")
+                              _ptr(scratch), nbytes, _stream()), "hbp_cumsumprod")
     return g
 
 

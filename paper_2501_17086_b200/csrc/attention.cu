@@ -242,13 +242,13 @@ void launch_fwd(Launcher& lc, const AttnArgs& a) {
 template <typename T, int DH>
 void launch_bwd(Launcher& lc, const AttnArgs& a) {
   dim3 grid((a.seq + kRows - 1) / kRows, a.heads, a.batch);
-  if (a.d_stats && !g_force_simt && attention_bwd_tc(lc, a, a.status)) return;  // row dots came with dO
+  if (a.d_stats && !lc.force_simt && attention_bwd_tc(lc, a, a.status)) return;  // row dots came with dO
   attn_rowdot_kernel<T, DH><<<grid, kThreads, 0, lc.stream>>>(a);
   lc.count();
   lc.check();
   AttnArgs plain = a;
   plain.d_stats = nullptr;
-  if (!g_force_simt && attention_bwd_tc(lc, plain, a.status)) return;  // bf16, head dimension 64: tensor cores
+  if (!lc.force_simt && attention_bwd_tc(lc, plain, a.status)) return;  // bf16, head dimension 64: tensor cores
   attn_bwd_dq_kernel<T, DH><<<grid, kThreads, 0, lc.stream>>>(a);
   attn_bwd_dkv_kernel<T, DH><<<grid, kThreads, 0, lc.stream>>>(a);
   lc.count(2);
@@ -269,7 +269,7 @@ void launch_bwd(Launcher& lc, const AttnArgs& a) {
   }
 
 void attention_fwd(Launcher& lc, const AttnArgs& a) {
-  if (!g_force_simt && attention_fwd_tc(lc, a, a.status)) return;  // bf16, head dimension 64: tensor cores
+  if (!lc.force_simt && attention_fwd_tc(lc, a, a.status)) return;  // bf16, head dimension 64: tensor cores
   HBP_ATTN_DISPATCH(launch_fwd)
 }
 void attention_bwd(Launcher& lc, const AttnArgs& a) { HBP_ATTN_DISPATCH(launch_bwd) }

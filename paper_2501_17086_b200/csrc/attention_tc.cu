@@ -565,7 +565,8 @@ bool attention_bwd_tc(Launcher& lc, const AttnArgs& a, int* status_word) {
             make_map4(&dq, dqkv, a.seq, a.heads, a.batch, ld3, BIG) && make_map4(&dk, dqkv + d, a.seq, a.heads, a.batch, ld3, BIG) &&
             make_map4(&dv, dqkv + 2 * d, a.seq, a.heads, a.batch, ld3, BIG);
   if (!ok) return false;
-  static bool attr_set = false;
+  static PerDevice<bool> attr_done;  // per-device kernel attribute
+  bool& attr_set = attr_done.here();
   if (!attr_set) {
     if (cudaFuncSetAttribute(attn_bwd_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
         cudaFuncSetAttribute(attn_bwd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
@@ -609,7 +610,8 @@ bool attention_fwd_tc(Launcher& lc, const AttnArgs& a, int* status_word) {
   if (!(make_map4(&q, qkv, a.seq, a.heads, a.batch, ld3, BIG) && make_map4(&k, qkv + d, a.seq, a.heads, a.batch, ld3, SMALL) &&
         make_map4(&v, qkv + 2 * d, a.seq, a.heads, a.batch, ld3, SMALL) && make_map4(&o, a.o, a.seq, a.heads, a.batch, d, BIG)))
     return false;
-  static bool attr_set = false;
+  static PerDevice<bool> attr_done;  // per-device kernel attribute
+  bool& attr_set = attr_done.here();
   if (!attr_set) {
     if (cudaFuncSetAttribute(attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD_SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();

@@ -517,11 +517,10 @@ EncodeTiledFn encode_fn() {
 }
 
 int sm_count() {
-  static int n = 0;
+  static PerDevice<int> count;
+  int& n = count.here();
   if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, current_device());
     if (n <= 0) n = 1;
   }
   return n;
@@ -576,7 +575,7 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   // pair mode halves the MMA thread's waits for operands but its MMAs run slower (about 200 cycles against
   // about 175 per 128 x 256 x 16 of work per SM), which nets out even
   const int sms = sm_count();
-  const bool pair = g_gemm_pair && sms >= 2 && g.M > BM;
+  const bool pair = lc.gemm_pair && sms >= 2 && g.M > BM;
   const int b_rows = pair ? Mode<true>::kBRows : Mode<false>::kBRows;
   CUtensorMap tmA, tmB;
   if (!make_map(&tmA, A0, g.M, g.K, g.batch, a_sm, a_sk, g.a_sb, a_mn, BM, f32)) return false;
@@ -611,7 +610,8 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
     if (g.epi == EPI_ADD && !make_map_epi(&tmE, g.E, true, g.M, g.N, g.batch, g.lde, g.e_sb)) return false;
   }
 
-  static bool attr_set = false;
+  static PerDevice<bool> attr_done;  // the shared-memory opt-in is a per-device attribute of the kernel
+  bool& attr_set = attr_done.here();
   if (!attr_set) {
     if (cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
         cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {

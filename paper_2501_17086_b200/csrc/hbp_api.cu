@@ -9,11 +9,8 @@
 #include "hbp_internal.h"
 
 namespace hbp {
-bool g_force_simt = false;
-bool g_gemm_pair = false;
-
 bool gemm(Launcher& lc, const GemmArgs& g, int* status_word) {
-  if (!g_force_simt && !g.relu && gemm_tc(lc, g, status_word)) return true;
+  if (!lc.force_simt && !g.relu && gemm_tc(lc, g, status_word)) return true;
   gemm_simt(lc, g);
   return false;
 }
@@ -29,6 +26,9 @@ struct ProfSeg {
 
 struct hbp_ctx {
   hbp_config cfg;
+  // kernel-selection modes, read from the environment (HBP_FORCE_SIMT=1, HBP_GEMM_PAIR=1) when THIS context is
+  // created and kept with it: another context created later under other settings does not change them
+  bool force_simt = false, gemm_pair = false;
   bool profiling = false;
   std::vector<ProfSeg> segs;       // recorded, not yet read
   std::vector<ProfSeg> free_segs;  // event pairs ready for reuse
@@ -251,6 +251,8 @@ struct Run {
   Run(hbp_ctx* ctx, const hbp_params* params, void* stream) : c(ctx), p(params) {
     lc.stream = (cudaStream_t)stream;
     lc.launches = &ctx->launches;
+    lc.force_simt = ctx->force_simt;
+    lc.gemm_pair = ctx->gemm_pair;
     N = ctx->cfg.tokens;
     d = ctx->cfg.d;
     h = ctx->cfg.hidden;
@@ -473,7 +475,7 @@ struct Run {
       u_has_delta = true;
     }
     bool tc = false;
-    if (c->Ahi && !g_force_simt) {
+    if (c->Ahi && !lc.force_simt) {
       gru_split(lc, (const float*)at(g, state), (const float*)c->C4, c->Ahi, c->Alo, rows, (int)d);
       a.A_hi = c->Ahi; a.A_lo = c->Alo; a.hl_a_sm = 3 * d; a.hl_a_sk = 1;
       a.B_hi = c->Whi; a.B_lo = c->Wlo; a.hl_b_sn = 3 * d; a.hl_b_sk = 1;
@@ -493,7 +495,7 @@ struct Run {
     int split = (int)(rows / (c->Ahi ? 512 : 2048));
     if (split < 1) split = 1;
     if (split > kMaxSplit) split = kMaxSplit;
-    const bool try_tc = c->Ahi && !g_force_simt;
+    const bool try_tc = c->Ahi && !lc.force_simt;
     if (try_tc) gru_split_transposed(lc, (const float*)at(g, state), (const float*)c->C4, c->Ahi, c->Alo, rows, (int)d);
     bool have_a4 = false;
     // {first row of the [4d] operand, rows, output, output row, against the states or the inputs}
@@ -540,7 +542,7 @@ struct Run {
     }
     const void* dl = every ? delta : nullptr;
     bool tc = false;
-    if (c->Ahi && !g_force_simt) {
+    if (c->Ahi && !lc.force_simt) {
       lstm_split(lc, (const float*)at(g, state), (const float*)c->C5, (const float*)c->Fg, (const float*)dl, c->Ahi, c->Alo,
                  (float*)c->U, rows, (int)u);
       a.A_hi = c->Ahi; a.A_lo = c->Alo; a.hl_a_sm = 4 * u; a.hl_a_sk = 1;
@@ -560,7 +562,7 @@ struct Run {
     int split = (int)(rows / (c->Ahi ? 512 : 2048));
     if (split < 1) split = 1;
     if (split > kMaxSplit) split = kMaxSplit;
-    const bool try_tc = c->Ahi && !g_force_simt;
+    const bool try_tc = c->Ahi && !lc.force_simt;
     if (try_tc) lstm_split_transposed(lc, (const float*)at(g, state), (const float*)c->C5, c->Ahi, c->Alo, rows, (int)u);
     bool have_a4 = false;
     for (int w = 0; w < 2; ++w) {
@@ -771,9 +773,9 @@ hbp_status hbp_create(const hbp_config* cfg, void* workspace, size_t workspace_b
   c->ws = (char*)workspace;
   c->ws_bytes = workspace_bytes;
   const char* env = std::getenv("HBP_FORCE_SIMT");
-  g_force_simt = env && env[0] == '1';
+  c->force_simt = env && env[0] == '1';
   const char* pm = std::getenv("HBP_GEMM_PAIR");
-  g_gemm_pair = pm && pm[0] == '1';
+  c->gemm_pair = pm && pm[0] == '1';
   if (cudaMemset(c->status, 0, 256) != cudaSuccess) {
     delete c;
     return HBP_ERR_CUDA;
@@ -821,6 +823,8 @@ hbp_status hbp_profile_read(hbp_ctx* ctx, float* ms, int64_t* launches) {
 }
 
 int64_t hbp_launch_count(const hbp_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int32_t hbp_context_modes(const hbp_ctx* ctx) { return ctx ? (ctx->force_simt ? 1 : 0) | (ctx->gemm_pair ? 2 : 0) : 0; }
 
 hbp_status hbp_sync_status(hbp_ctx* ctx, void* cuda_stream) {
   if (!ctx) return HBP_ERR_INVALID_ARG;
@@ -1159,7 +1163,14 @@ hbp_status hbp_cumsumprod_scratch_bytes(int32_t dtype, int32_t L, int64_t rows, 
 hbp_status hbp_cumsumprod(int32_t dtype, int32_t gate, int32_t loss, int32_t L, int64_t rows, int32_t d, const void* u,
                           const void* delta, const void* a, void* g, void* scratch, size_t scratch_bytes,
                           void* cuda_stream) {
+  return hbp_cumsumprod_status(dtype, gate, loss, L, rows, d, u, delta, a, g, scratch, scratch_bytes, nullptr, cuda_stream);
+}
+
+hbp_status hbp_cumsumprod_status(int32_t dtype, int32_t gate, int32_t loss, int32_t L, int64_t rows, int32_t d,
+                                 const void* u, const void* delta, const void* a, void* g, void* scratch,
+                                 size_t scratch_bytes, int32_t* status, void* cuda_stream) {
   size_t need = 0;
+  if ((uintptr_t)status & 3u) return HBP_ERR_SHAPE;
   hbp_status st = hbp_cumsumprod_scratch_bytes(dtype, L, rows, d, &need);
   if (st != HBP_OK) return st;
   if (!delta || !g) return HBP_ERR_INVALID_ARG;
@@ -1178,6 +1189,7 @@ hbp_status hbp_cumsumprod(int32_t dtype, int32_t gate, int32_t loss, int32_t L, 
   s.dtype = dtype; s.L = L; s.l_lo = 0; s.l_hi = L; s.rows = rows; s.d = d;
   s.u = u; s.delta = delta; s.loss = loss; s.a = a; s.gate = gate; s.g = g;
   s.scratch = scratch; s.scratch_bytes = scratch_bytes;
+  s.status = status;
   scan_reverse(lc, s);
   return lc.err == cudaSuccess ? HBP_OK : HBP_ERR_CUDA;
 }

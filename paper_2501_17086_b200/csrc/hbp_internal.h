@@ -58,11 +58,27 @@ struct GemmArgs {
   float* partial = nullptr;
 };
 
-// Counts launches and remembers the first CUDA error.
+// Per-device memo for one-time set-up that CUDA keeps per device (kernel attributes, device properties): a
+// process may drive several GPUs, each from its own context, so nothing of that kind is cached process-wide.
+constexpr int kMaxDevices = 64;
+inline int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+  return dev;
+}
+template <typename T>
+struct PerDevice {
+  T v[kMaxDevices] = {};
+  T& here() { return v[current_device()]; }
+};
+
+// Counts launches and remembers the first CUDA error; carries the kernel-selection modes of the context it runs for.
 struct Launcher {
   cudaStream_t stream = nullptr;
   int64_t* launches = nullptr;
   cudaError_t err = cudaSuccess;
+  bool force_simt = false;  // keep every GEMM and attention product on the CUDA-core kernels (cross-checks)
+  bool gemm_pair = false;   // tensor-core GEMM pairs CTAs (cta_group::2, 256 x 256 tiles) where there are two row blocks
   void count(int n = 1) {
     if (launches) *launches += n;
   }
@@ -82,12 +98,6 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word);
 bool gemm(Launcher& lc, const GemmArgs& g, int* status_word);
 // Number of 64-column slots of partial sums the tensor-core kernel writes per row for N columns.
 int gemm_tc_stats_slots(int N);
-// Set from the environment variable HBP_FORCE_SIMT=1 when a context is created: keeps every GEMM
-// on the CUDA-core kernel (used to cross-check the tensor-core kernel).
-extern bool g_force_simt;
-// Set from the environment variable HBP_GEMM_PAIR=1 when a context is created: the tensor-core GEMM then pairs
-// CTAs (cta_group::2, 256 x 256 tiles) wherever the problem has two row blocks; otherwise single CTAs.
-extern bool g_gemm_pair;
 
 // ---------------------------------------------------------------- scans and elementwise (scan.cu)
 // Internal gate kind beside the public hbp_gate values: a[L][rows][d], one gate per element and step (the

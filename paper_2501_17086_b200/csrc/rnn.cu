@@ -245,7 +245,8 @@ void rnn_forward_step(Launcher& lc, int dtype, const void* W, const void* U, con
                       const double* h_in, double* h_out, void* deriv, void* state_out, int B, int d, int in_dim) {
   const size_t staged = staged_bytes(d + in_dim, d + in_dim);
   if (staged <= kStagedSmemLimit) {
-    static size_t cfg_f = 0, cfg_b = 0;
+    static PerDevice<size_t> cfg_f_on, cfg_b_on;  // per-device kernel attributes
+    size_t &cfg_f = cfg_f_on.here(), &cfg_b = cfg_b_on.here();
     dim3 sgrid((d + kSCols - 1) / kSCols, (B + kSRows - 1) / kSRows);
     if (dtype == HBP_F32 && allow_smem(rnn_step_staged_kernel<float>, staged, &cfg_f)) {
       rnn_step_staged_kernel<float><<<sgrid, 256, staged, lc.stream>>>((const float*)W, (const float*)U, (const float*)x_t,
@@ -281,7 +282,8 @@ void rnn_backward_step(Launcher& lc, int dtype, const void* W, const void* deriv
                        const double* g_in, double* g_out, void* g_store, int B, int d) {
   const size_t staged = staged_bytes(d, d);
   if (staged <= kStagedSmemLimit) {
-    static size_t cfg_f = 0, cfg_b = 0;
+    static PerDevice<size_t> cfg_f_on, cfg_b_on;  // per-device kernel attributes
+    size_t &cfg_f = cfg_f_on.here(), &cfg_b = cfg_b_on.here();
     dim3 sgrid((d + kSCols - 1) / kSCols, (B + kSRows - 1) / kSRows);
     if (dtype == HBP_F32 && allow_smem(rnn_bwd_step_staged_kernel<float>, staged, &cfg_f)) {
       rnn_bwd_step_staged_kernel<float><<<sgrid, 256, staged, lc.stream>>>((const float*)W, (const float*)deriv,

@@ -112,7 +112,10 @@ __global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(co
       for (int k = first; k < issued; ++k) {
         const uint64_t t0 = global_ns();
         while (!mbar_try_wait(full_bar(k % nstages), (uint32_t)((k / nstages) & 1)))
-          if (global_ns() - t0 > WAIT_LIMIT_NS) break;
+          if (global_ns() - t0 > WAIT_LIMIT_NS) {  // a copy that never landed: say so, then leave
+            atomicExch(status, (int)HBP_ERR_TIMEOUT);
+            break;
+          }
       }
     }
     return;
@@ -202,7 +205,8 @@ bool make_map2(CUtensorMap* tm, const void* base, bool f32, int64_t steps, int64
 template <typename T, int NS, bool kElemGate>
 void launch_ring(Launcher& lc, const ScanArgs& s, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& mg,
                  unsigned grid, int nstages, int rows_ps, size_t smem) {
-  static size_t configured = 0;
+  static PerDevice<size_t> configured_on;  // per-device kernel attribute
+  size_t& configured = configured_on.here();
   if (smem > configured) {
     cudaFuncSetAttribute(scan_ring_kernel<T, NS, kElemGate>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     configured = smem;

@@ -9,17 +9,16 @@
 namespace {
 
 constexpr size_t kStaticScratchBytes = (size_t)32 << 20;  // 32 MiB
-constexpr int kMaxDevices = 64;
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 // The array's name is only a host-side handle; the device address is looked up once per device
 // (with that device current) and remembered.
-void* g_scratch_addr[kMaxDevices] = {};
+void* g_scratch_addr[hbp::kMaxDevices] = {};
 
 hbp_status static_scratch(void** out) {
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return HBP_ERR_CUDA;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= hbp::kMaxDevices) return HBP_ERR_CUDA;
   if (!g_scratch_addr[dev]) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {

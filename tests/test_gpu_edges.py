@@ -208,6 +208,35 @@ def test_gemm_single_cta_and_cta_pair_modes_match_oracle(name, ks, mode, monkeyp
     compare(w, gpu, ref, ks, ("exact", kmax))
 
 
+def test_kernel_modes_belong_to_the_context(monkeypatch):
+    """Two contexts created under different settings keep their own modes, and a call through either launches its own
+    kind of kernels however the calls are interleaved: the modes read back as created, the CUDA-core context
+    reproduces its own bits after the others have run, and all agree to the bf16 tolerance."""
+    from paper_2501_17086_b200 import harness
+    from paper_2501_17086_b200.workloads import WORKLOADS, make_inputs
+    w = WORKLOADS["c2_twin"]
+    inp = make_inputs(w, "cuda")
+    monkeypatch.setenv("HBP_FORCE_SIMT", "1")
+    simt = harness.make_context(w)
+    monkeypatch.delenv("HBP_FORCE_SIMT")
+    monkeypatch.setenv("HBP_GEMM_PAIR", "1")
+    pair = harness.make_context(w)
+    monkeypatch.delenv("HBP_GEMM_PAIR")
+    plain = harness.make_context(w)
+    assert (simt.modes, pair.modes, plain.modes) == (1, 2, 0)
+    params = harness.params_for(w, inp)
+    outs = []
+    for ctx in (simt, pair, plain, simt):      # interleaved: a later context's creation or use changes nothing
+        x_all = ctx.forward(params, inp["x0"], None)
+        delta = harness.loss_delta(w, x_all, inp)
+        outs.append(ctx.backward(params, 2, delta, x_all, None).float().clone())
+        ctx.sync_status()
+    assert (simt.modes, pair.modes, plain.modes) == (1, 2, 0)
+    assert torch.equal(outs[0], outs[3])        # the same context computes the same bits before and after the others
+    for o in outs[1:3]:
+        assert float((o - outs[0]).norm() / outs[0].norm()) < 2e-2
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_compare_matches_the_definition(dtype):
     from paper_2501_17086_b200 import binding as B

@@ -11,12 +11,47 @@ from paper_2501_17086_b200.workloads import WORKLOADS, make_inputs
 pytestmark = pytest.mark.gpu
 
 TOL = {"f32": 1e-5, "bf16": 2e-2}
-# Exact BPTT on c3 is ill-conditioned: with a in U(0.9, 0.999) plus 0.5 x orthogonal recurrent weights the step
-# Jacobian a + tanh'(z) W has growth ~1.007 per step, so ||g_0|| / ||g_T|| ~ 1e13 over 4096 steps and the float
-# rounding of the stored states (2.6e-7 between the two forward passes) is amplified through hundreds of
-# factors.  Highway-BP with k <= 8 applies at most 8 block Jacobians and keeps the 1e-5 bar; exact BPTT at the
-# full length is held to this looser bound (it meets 1e-5 on the T = 200 twin).
-TOL_EXACT_LONG_RNN = 5e-4
+RECURRENT = ("rnn_tanh", "gru", "lstm")
+
+
+def _relabelled(w, inp, perm):
+    """The same recurrent network with its hidden units renumbered by ``perm``: a permutation of rows and columns
+    of the weights, of the gate and of the targets.  Mathematically nothing changes (results come back permuted);
+    numerically every sum runs in another order."""
+    p = torch.as_tensor(perm, device=inp["W"].device)
+    n = int(p.numel())
+    out = dict(inp)
+    blocks = {"rnn_tanh": 1, "gru": 3, "lstm": 4}[w.block]
+    W, U = inp["W"], inp["U"]
+    out["W"] = W.reshape(blocks, n, n)[:, p][:, :, p].reshape(W.shape).contiguous()
+    out["U"] = U.reshape(blocks, n, -1)[:, p].reshape(U.shape).contiguous()
+    if "a" in inp:
+        out["a"] = inp["a"][p].contiguous()
+    halves = w.d // n                                   # LSTM: the state is [c | h], both halves renumbered
+    for name in ("Y", "y", "x0"):
+        t = inp[name]
+        out[name] = t.reshape(*t.shape[:-1], halves, n)[..., p].reshape(t.shape).contiguous()
+    return out
+
+
+def _oracle_floor(w, inp, rows, base_exact):
+    """How far two fp64 evaluations of exact backpropagation through the same recurrent network lie apart when only
+    the order of their sums differs (units renumbered): the resolution at which the oracle itself defines the exact
+    gradient.  A recurrence whose forward map amplifies perturbations (c3: ||g_0|| / ||g_T|| ~ 1e13 over 4096 steps)
+    turns the 1e-16 of double rounding into 1e-7 on the late states and 1e-5 on the gradient, whatever the
+    implementation; nothing can be compared with the oracle more finely than that."""
+    n = w.hidden if w.block == "lstm" else w.d
+    perm = np.random.default_rng(w.seed).permutation(n)
+    inv = np.argsort(perm)
+    ref2 = orun.run(w, _relabelled(w, inp, perm), ks=(), rows=rows)
+    halves = w.d // n
+    worst = 0.0
+    for a, b in zip(ref2["exact"], base_exact):
+        a = a.reshape(*a.shape[:-1], halves, n)[..., inv].reshape(b.shape)
+        nb = np.linalg.norm(b)
+        if nb:
+            worst = max(worst, float(np.linalg.norm(a - b) / nb))
+    return worst
 
 
 def _rows_of(w, t, rows):
@@ -29,8 +64,8 @@ def _rows_of(w, t, rows):
 @pytest.mark.parametrize("name,ks,rows", [
     ("c2", (1, 2, 4, 8), [0, 1, 127, 128, 4097, 8191]),
     ("c3", (1, 2, 4, 8), [0, 31]),
-    ("c4", (1, 2, 4), [5]),
-    ("c5", (1, 2), [0, 129, 8200, 16383]),
+    ("c4", (1, 2, 4), [0, 15]),
+    ("c5", (1, 2, 4, 8), [0, 129, 8200, 16383]),
     ("g1", (1, 2, 4), [0, 77, 127]),
     ("g2", (1, 3, 8), [0, 1, 64, 127]),
     ("l1", (1, 2, 4), [0, 77, 127]),
@@ -62,10 +97,28 @@ def test_full_size_sampled_units(name, ks, rows):
     xs_gpu = _rows_of(w, x_all, rows_t).float().cpu().double().numpy()
     for t in grads.values():
         assert torch.isfinite(t).all()
-    del ctx, g_all, x_all, grads
+    # Parameter gradients through the full-size kernels (every token row in the contraction, split-K and layer
+    # groups as the benchmark runs them) with an answer the oracle can give: units are independent, so with delta
+    # zeroed outside the sampled units every other row of g^k is exactly zero and the gradients are the sampled
+    # units' contributions alone.
+    kg = 2
+    units = w.batch if (w.block == "preln_transformer" or w.block in RECURRENT) else w.tokens
+    mask = torch.zeros(units, device="cuda", dtype=delta.dtype)
+    mask[rows_t] = 1
+    if w.block == "preln_transformer":
+        delta_m = (delta.reshape(w.batch, w.seq, w.d) * mask[:, None, None]).reshape(delta.shape).contiguous()
+    else:
+        delta_m = (delta * mask[:, None]).contiguous()      # [N, d] or [steps + 1, B, d]
+    ctx.backward(params, kg, delta_m, x_all, xin, g_all=g_all, grads=grads)
+    ctx.sync_status()
+    others = torch.ones(units, device="cuda", dtype=torch.bool)
+    others[rows_t] = False
+    assert not _rows_of(w, g_all, others.nonzero().flatten()[:64]).any()
+    got_grads = {n: t.double().cpu().numpy() for n, t in grads.items()}
+    del ctx, g_all, x_all, grads, delta_m
     torch.cuda.empty_cache()
 
-    ref = orun.run(w, inp, ks=ks, rows=rows_t.cpu())
+    ref = orun.run(w, inp, ks=ks, rows=rows_t.cpu(), grads_for=(kg,))
     tol = TOL[w.dtype]
 
     def rel(a, b):
@@ -91,12 +144,24 @@ def test_full_size_sampled_units(name, ks, rows):
         worst = worst_over_states(got[k], ref["hbp"][k])
         assert worst < tol, f"k={k}: max rel-L2 {worst:.3e}"
     worst = max(rel(got["exact"][l], ref["exact"][l]) for l in range(w.steps + 1))
-    tol_exact = TOL_EXACT_LONG_RNN if name == "c3" else tol
+    tol_exact = tol
+    if w.block in RECURRENT and w.dtype == "f32":
+        # exact BPTT is compared no more finely than the oracle defines it (see _oracle_floor); 4 x: the floor is
+        # one sample of a quantity that varies with the order of the sums
+        floor = _oracle_floor(w, inp, rows_t.cpu(), ref["exact"])
+        tol_exact = max(tol, 4.0 * floor)
+        print(f"{name}: exact BPTT error {worst:.3e}, oracle floor {floor:.3e}")
     assert worst < tol_exact, f"exact: max rel-L2 {worst:.3e}"
     # tail exactness on the GPU itself (Theorem 2): g^k_l is already exact for l >= steps - k
     kmax = max(ks)
     for l in range(w.steps - kmax, w.steps + 1):
         assert rel(got[kmax][l], got["exact"][l]) < tol_exact
+    # parameter gradients of the sampled units, layer by layer where the weights are stacked
+    for n, v in ref["grads"][kg].items():
+        gp = got_grads["d" + n].reshape(v.shape)
+        parts = zip(gp, v) if v.ndim == 3 else [(gp, v)]
+        worst = max(rel(a, b) for a, b in parts)
+        assert worst < tol, f"d{n} (k={kg}, sampled units through the full-size kernels): {worst:.3e}"
 
 
 def _run_shard(w_shard, inp, rows, delta_rows):
