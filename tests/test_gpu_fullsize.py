@@ -101,7 +101,7 @@ def test_full_size_sampled_units(name, ks, rows):
     # groups as the benchmark runs them) with an answer the oracle can give: units are independent, so with delta
     # zeroed outside the sampled units every other row of g^k is exactly zero and the gradients are the sampled
     # units' contributions alone.
-    kg = 2
+    kg = ks[1]
     units = w.batch if (w.block == "preln_transformer" or w.block in RECURRENT) else w.tokens
     mask = torch.zeros(units, device="cuda", dtype=delta.dtype)
     mask[rows_t] = 1
