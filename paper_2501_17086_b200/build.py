@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhbp.so")
-SOURCES = ["hbp_api.cu", "gemm_simt.cu", "gemm_tc.cu", "scan.cu", "scan_static.cu", "scan_ring.cu", "attention.cu", "attention_tc.cu", "rnn.cu", "gru.cu", "lstm.cu", "diag.cu"]
+SOURCES = ["hbp_api.cu", "gemm_simt.cu", "gemm_tc.cu", "scan.cu", "scan_static.cu", "scan_ring.cu", "attention.cu", "attention_tc.cu", "rnn.cu", "rnn_persistent.cu", "gru.cu", "lstm.cu", "diag.cu"]
 
 
 def _stale() -> bool:

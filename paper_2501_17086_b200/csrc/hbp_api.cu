@@ -49,6 +49,7 @@ struct hbp_ctx {
   char* DACT = nullptr;    // [layers][N][h] gelu'(Z)
   float* xres = nullptr;   // [N][d] float master of the residual stream (bf16 only)
   double* hres = nullptr;  // RNN: 2 x [B][d] double master of the recurrent state (ping-pong)
+  double* Pd = nullptr;    // tanh RNN: [T][B][d] input projections U x_t in double for the one-launch recurrence
   // RNN, float: tf32 high/low splits of the GEMM operands, each written with the contraction index
   // contiguous: A* is g * tanh' as [T*B][d] for the VJP or [d][T*B] for the weight gradients, H* the states
   // h_0..h_{T-1} as [d][T*B], X* the inputs as [in][T*B], W* the recurrent matrix transposed
@@ -183,6 +184,10 @@ size_t carve(hbp_ctx* c, char* base) {
   } else if (f.block == HBP_BLOCK_RNN_TANH) {
     c->C = take(steps * N * d * es);
     c->hres = (double*)take(2 * N * d * 8);
+    if (f.gate != HBP_GATE_CHANNEL_PER_STEP) {
+      const size_t pb = rnn_persistent_proj_bytes(f.L, f.tokens, f.d);
+      if (pb) c->Pd = (double*)take(pb);
+    }
     if (f.dtype == HBP_F32) {
       c->Ahi = (float*)take(steps * N * d * 4); c->Alo = (float*)take(steps * N * d * 4);
       c->Hhi = (float*)take(steps * N * d * 4); c->Hlo = (float*)take(steps * N * d * 4);
@@ -883,13 +888,19 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
     }
   } else if (f.block == HBP_BLOCK_RNN_TANH) {
     const int T = f.L;
-    convert_to_f64(r.lc, f.dtype, x0, ctx->hres, state);
-    for (int t = 0; t < T; ++t) {
-      const double* hin = ctx->hres + (int64_t)(t & 1) * state;
-      double* hout = ctx->hres + (int64_t)((t + 1) & 1) * state;
-      rnn_forward_step(r.lc, f.dtype, params->W, params->U, r.at(inputs, (int64_t)t * N * f.in_dim), r.gate_ptr(t), hin,
-                       hout, r.at(ctx->C, (int64_t)t * state), r.at(xa, (int64_t)(t + 1) * state), (int)N, (int)d,
-                       f.in_dim);
+    // all T steps in one launch where that form applies, else one launch per step
+    const bool one_launch = ctx->Pd && !ctx->force_simt &&
+                            rnn_forward_persistent(r.lc, f.dtype, params->W, params->U, inputs, r.gate_ptr(0), x0, ctx->Pd, xa,
+                                                   ctx->C, T, (int)N, (int)d, f.in_dim);
+    if (!one_launch) {
+      convert_to_f64(r.lc, f.dtype, x0, ctx->hres, state);
+      for (int t = 0; t < T; ++t) {
+        const double* hin = ctx->hres + (int64_t)(t & 1) * state;
+        double* hout = ctx->hres + (int64_t)((t + 1) & 1) * state;
+        rnn_forward_step(r.lc, f.dtype, params->W, params->U, r.at(inputs, (int64_t)t * N * f.in_dim), r.gate_ptr(t), hin,
+                         hout, r.at(ctx->C, (int64_t)t * state), r.at(xa, (int64_t)(t + 1) * state), (int)N, (int)d,
+                         f.in_dim);
+      }
     }
     if (ctx->Ahi) {  // operand splits that do not change between backward calls
       split_tf32_transposed(r.lc, (const float*)xa, nullptr, ctx->Hhi, ctx->Hlo, (int64_t)T * N, (int)d);
@@ -1020,14 +1031,21 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
     // Section 2.2: g_l = delta_l + a_l g_{l+1} + J_l^T g_{l+1}, one step at a time
     PhaseScope ph(r, HBP_PHASE_OTHER);
     if (rnn) {
-      // the sequential recurrence is carried in double beside the stored float gradients
-      convert_to_f64(r.lc, f.dtype, r.at(r.g, (int64_t)steps * r.state), ctx->hres, r.state);
-      for (int t = steps - 1; t >= 0; --t) {
-        const double* gin = ctx->hres + (int64_t)((steps - 1 - t) & 1) * r.state;
-        double* gout = ctx->hres + (int64_t)((steps - t) & 1) * r.state;
-        rnn_backward_step(r.lc, f.dtype, params->W, r.at(ctx->C, (int64_t)t * r.state),
-                          f.loss == HBP_LOSS_EVERY_STEP ? r.at(r.delta, (int64_t)t * r.state) : nullptr, r.gate_ptr(t),
-                          gin, gout, r.at(r.g, (int64_t)t * r.state), (int)r.N, (int)r.d);
+      // the sequential recurrence is carried in double beside the stored float gradients: one launch over all
+      // steps where that form applies, else one launch per step
+      const bool one_launch = ctx->Pd && !ctx->force_simt &&
+                              rnn_backward_persistent(r.lc, f.dtype, params->W, r.gate_ptr(0), ctx->C,
+                                                      f.loss == HBP_LOSS_EVERY_STEP ? r.delta : nullptr, r.g, steps,
+                                                      (int)r.N, (int)r.d);
+      if (!one_launch) {
+        convert_to_f64(r.lc, f.dtype, r.at(r.g, (int64_t)steps * r.state), ctx->hres, r.state);
+        for (int t = steps - 1; t >= 0; --t) {
+          const double* gin = ctx->hres + (int64_t)((steps - 1 - t) & 1) * r.state;
+          double* gout = ctx->hres + (int64_t)((steps - t) & 1) * r.state;
+          rnn_backward_step(r.lc, f.dtype, params->W, r.at(ctx->C, (int64_t)t * r.state),
+                            f.loss == HBP_LOSS_EVERY_STEP ? r.at(r.delta, (int64_t)t * r.state) : nullptr, r.gate_ptr(t),
+                            gin, gout, r.at(r.g, (int64_t)t * r.state), (int)r.N, (int)r.d);
+        }
       }
       if (grads) r.rnn_wgrad(grads);
     } else if (gru) {
