@@ -224,8 +224,19 @@ hbp_status hbp_compare(int32_t dtype, int32_t segments, int64_t elems, const voi
                        void* scratch, size_t scratch_bytes, void* cuda_stream);
 
 /* Copies the context's device status word to the host after synchronising the stream: HBP_OK, or the
- * error a kernel recorded (HBP_ERR_TIMEOUT when a bounded wait gave up).  The only synchronising call. */
+ * error a kernel recorded (HBP_ERR_TIMEOUT when a bounded wait gave up).  An error is reported once: the word is
+ * cleared after a non-zero read, and the context stays usable (a kernel whose wait gave up has released its
+ * tensor memory and ended normally; its outputs are incomplete).  The only synchronising call. */
 hbp_status hbp_sync_status(hbp_ctx* ctx, void* cuda_stream);
+
+/* Diagnostic, not part of the method: exercises the failure path of the tensor-core kernels' bounded waits.
+ * Enqueues one tile of the GEMM kernel whose copy role expects bytes that it never requests, with every wait limited
+ * to limit_ns (1 us .. 1 s) instead of the usual 4 s: the wait runs out, the kernel records HBP_ERR_TIMEOUT in the
+ * context's status word, all of its roles leave, the tensor memory is freed and the kernel ends.  The next
+ * hbp_sync_status returns HBP_ERR_TIMEOUT.  scratch: device memory, 256-byte aligned, >= 128 KiB (contents
+ * irrelevant, may be overwritten).  Nothing waits without a limit at any point. */
+hbp_status hbp_selftest_wait_timeout(hbp_ctx* ctx, void* scratch, size_t scratch_bytes, uint64_t limit_ns,
+                                     void* cuda_stream);
 
 /* Device time per phase of the path, for the backward / exact calls made while profiling is on.  CUDA
  * events are recorded on the call's stream around each phase: the reverse scans (Eq. 9-11), the block VJPs

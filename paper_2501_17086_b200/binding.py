@@ -21,7 +21,7 @@ LOSS_FINAL, LOSS_EVERY_STEP = 0, 1
 
 EXPORTS = ["hbp_workspace_bytes", "hbp_create", "hbp_forward", "hbp_backward", "hbp_exact",
            "hbp_cumsumprod_scratch_bytes", "hbp_cumsumprod", "hbp_cumsumprod_status", "hbp_sync_status", "hbp_launch_count",
-           "hbp_context_modes",
+           "hbp_context_modes", "hbp_selftest_wait_timeout",
            "hbp_profile_enable", "hbp_profile_read", "hbp_cumsumprod_static", "hbp_cumsumprod_static_max_bytes",
            "hbp_compare_scratch_bytes", "hbp_compare", "hbp_iterate", "hbp_add_carry", "hbp_param_grads",
            "hbp_status_string", "hbp_destroy"]
@@ -62,6 +62,7 @@ def _load():
     lib.hbp_cumsumprod_scratch_bytes.argtypes = [i32, i32, i64, i32, C.POINTER(sz)]
     lib.hbp_cumsumprod.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.hbp_cumsumprod_status.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.hbp_selftest_wait_timeout.argtypes = [vp, vp, sz, C.c_uint64, vp]
     lib.hbp_context_modes.argtypes = [vp]
     lib.hbp_context_modes.restype = i32
     lib.hbp_cumsumprod_static.argtypes = [i32, i32, i32, i32, i64, i32, vp, vp, vp, vp, vp]
@@ -164,6 +165,15 @@ class Context:
         _check(lib.hbp_create(C.byref(cfg), C.c_void_p(base), nbytes, C.byref(handle)), "hbp_create")
         self._h = handle
         self._keep = None
+
+    def selftest_wait_timeout(self, limit_ns=1_000_000):
+        """Enqueues a GEMM tile whose pipeline stalls on purpose with every wait limited to ``limit_ns``; the next
+        sync_status() raises HbpError(8)."""
+        scratch = torch.empty((128 << 10) + 256, dtype=torch.uint8, device=self.device)
+        base = (scratch.data_ptr() + 255) // 256 * 256
+        _check(lib.hbp_selftest_wait_timeout(self._h, C.c_void_p(base), 128 << 10, limit_ns, _stream()),
+               "hbp_selftest_wait_timeout")
+        self._keep = scratch
 
     @property
     def modes(self) -> int:

@@ -59,6 +59,8 @@ struct TcParams {
   float* R;
   float2* stats; int64_t stats_sb;
   int* status;
+  uint64_t wait_limit_ns;  // limit of every barrier wait
+  int stall;               // self-test of the bounded waits only: the producer arms its first stage and copies nothing
 };
 
 // ------------------------------------------------------------------------------------------- epilogue math
@@ -201,13 +203,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const CUtensorMap* mA = seg == 0 ? &tmA : (seg == 1 ? &tmA1 : &tmA2);
           const CUtensorMap* mB = seg == 0 ? &tmB : (seg == 1 ? &tmB1 : &tmB2);
           for (int kb = kb_lo; kb < kb_hi; ++kb) {
-            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, p.wait_limit_ns)) { ok = false; break; }
             const uint32_t sA = base + stage * STAGE_BYTES, sB = sA + A_BYTES;
             // pair: all four tile loads of a stage (two per CTA) complete on the leader's barrier
             const uint32_t fb = kPair ? map_to_cta(full_bar(stage), 0) : full_bar(stage);
             if (leader) mbar_expect_tx(full_bar(stage), kPair ? 2 * STAGE_BYTES : STAGE_BYTES);
             issued_mask |= 1u << stage;
             issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+            if (p.stall) { ok = false; break; }  // self-test: bytes are expected that nobody sends
             const int k0 = kb * row_elems;
             auto load = [&](uint32_t dst, const CUtensorMap* tm, int c0, int c1) {
               if (kPair) tma_load_3d_pair(dst, tm, fb, c0, c1, b);
@@ -232,7 +235,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int s = 0; s < STAGES; ++s)
           if (issued_mask & (1u << s)) {
             uint64_t t0 = global_ns();
-            while (!mbar_try_wait(full_bar(s), (issued_parity >> s) & 1u) && global_ns() - t0 < 100000000ull) {
+            const uint64_t lim = p.wait_limit_ns < 100000000ull ? p.wait_limit_ns : 100000000ull;
+            while (!mbar_try_wait(full_bar(s), (issued_parity >> s) & 1u) && global_ns() - t0 < lim) {
             }
           }
       }
@@ -250,14 +254,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
       for (int tile = first_tile; tile < p.num_tiles && ok; tile += tile_step) {
-        if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.status, p.wait_limit_ns)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)acc * BN;
         const int split = (tile / tiles_per_batch) / p.batch;
         const int kb_lo = split * p.kb_per_split, kb_hi = min(p.k_blocks, kb_lo + p.kb_per_split);
         uint32_t first = 1;
         for (int it = (kb_hi - kb_lo) * p.segs; it > 0; --it) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, p.wait_limit_ns)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sA = base + stage * STAGE_BYTES, sB = sA + A_BYTES;
 #pragma unroll
@@ -321,7 +325,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tma_load_3d(buf, &tmE, ebar, colw, row0, b);
         e_pending = true;
       }
-      if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag, p.status)) break;
+      if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag, p.status, p.wait_limit_ns)) break;
       tc_fence_after();
       const uint32_t tsrc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + half * 128);
       if (!staged) {
@@ -349,7 +353,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
           const int col = colw + c * cw;
           if (has_e) {
-            if (!mbar_wait(ebar, e_phase, abort_flag, p.status)) { ok = false; break; }
+            if (!mbar_wait(ebar, e_phase, abort_flag, p.status, p.wait_limit_ns)) { ok = false; break; }
             e_phase ^= 1u;
             e_pending = false;
             if (p.epi == EPI_ADD) {  // float tile: 32 columns
@@ -637,6 +641,8 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   p.R = g.R;
   p.stats = g.stats; p.stats_sb = g.stats_sb;
   p.status = status_word;
+  p.wait_limit_ns = g.wait_limit_ns ? g.wait_limit_ns : WAIT_LIMIT_NS;
+  p.stall = g.test_stall;
   if (pair) {
     const int pairs = p.num_tiles < sms / 2 ? p.num_tiles : sms / 2;
     cudaLaunchConfig_t cfg = {};

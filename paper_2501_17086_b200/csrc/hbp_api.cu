@@ -837,7 +837,33 @@ hbp_status hbp_sync_status(hbp_ctx* ctx, void* cuda_stream) {
   cudaStream_t s = (cudaStream_t)cuda_stream;
   if (cudaMemcpyAsync(&word, ctx->status, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return HBP_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return HBP_ERR_CUDA;
+  if (word != 0) {  // reported once: the next calls start from a clean word
+    if (cudaMemsetAsync(ctx->status, 0, sizeof(int), s) != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) return HBP_ERR_CUDA;
+  }
   return (hbp_status)word;
+}
+
+hbp_status hbp_selftest_wait_timeout(hbp_ctx* ctx, void* scratch, size_t scratch_bytes, uint64_t limit_ns, void* cuda_stream) {
+  if (!ctx || !scratch) return HBP_ERR_INVALID_ARG;
+  if (((uintptr_t)scratch % kAlign) || scratch_bytes < ((size_t)128 << 10)) return HBP_ERR_WORKSPACE;
+  if (limit_ns < 1000 || limit_ns > 1000000000ull) return HBP_ERR_INVALID_ARG;
+  Launcher lc;
+  lc.stream = (cudaStream_t)cuda_stream;
+  lc.launches = &ctx->launches;
+  // one 128 x 256 x 64 bf16 tile; the producer arms the first pipeline stage and issues no copy, so the MMA role's
+  // wait for it runs out after limit_ns
+  char* base = (char*)scratch;
+  GemmArgs g;
+  g.in_dtype = HBP_BF16;
+  g.M = 128; g.N = 256; g.K = 64;
+  g.A = base; g.a_sm = 64; g.a_sk = 1;
+  g.B = base + (16 << 10); g.b_sn = 64; g.b_sk = 1;
+  g.epi = EPI_STORE;
+  g.D = base + (48 << 10); g.ldd = 256;
+  g.wait_limit_ns = limit_ns;
+  g.test_stall = 1;
+  if (!gemm_tc(lc, g, ctx->status)) return HBP_ERR_UNSUPPORTED;
+  return lc.err == cudaSuccess ? HBP_OK : HBP_ERR_CUDA;
 }
 
 hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, const void* inputs, void* x_all,
@@ -891,7 +917,7 @@ hbp_status hbp_forward(hbp_ctx* ctx, const hbp_params* params, const void* x0, c
     // all T steps in one launch where that form applies, else one launch per step
     const bool one_launch = ctx->Pd && !ctx->force_simt &&
                             rnn_forward_persistent(r.lc, f.dtype, params->W, params->U, inputs, r.gate_ptr(0), x0, ctx->Pd, xa,
-                                                   ctx->C, T, (int)N, (int)d, f.in_dim);
+                                                   ctx->C, T, (int)N, (int)d, f.in_dim, ctx->status);
     if (!one_launch) {
       convert_to_f64(r.lc, f.dtype, x0, ctx->hres, state);
       for (int t = 0; t < T; ++t) {
@@ -1036,7 +1062,7 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
       const bool one_launch = ctx->Pd && !ctx->force_simt &&
                               rnn_backward_persistent(r.lc, f.dtype, params->W, r.gate_ptr(0), ctx->C,
                                                       f.loss == HBP_LOSS_EVERY_STEP ? r.delta : nullptr, r.g, steps,
-                                                      (int)r.N, (int)r.d);
+                                                      (int)r.N, (int)r.d, ctx->status);
       if (!one_launch) {
         convert_to_f64(r.lc, f.dtype, r.at(r.g, (int64_t)steps * r.state), ctx->hres, r.state);
         for (int t = steps - 1; t >= 0; --t) {

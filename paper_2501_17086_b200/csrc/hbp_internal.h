@@ -56,6 +56,10 @@ struct GemmArgs {
   int64_t hl_a_sm = 0, hl_a_sk = 0, hl_b_sn = 0, hl_b_sk = 0;
   int splitk = 1;      // > 1: partial sums to `partial` [splitk][batch][M][N], reduced in fixed order
   float* partial = nullptr;
+  // self-test of the tensor-core kernel's bounded waits (hbp_selftest_wait_timeout): a wait limit other than the
+  // default, and a producer that arms its first pipeline stage without issuing the copies
+  uint64_t wait_limit_ns = 0;
+  int test_stall = 0;
 };
 
 // Per-device memo for one-time set-up that CUDA keeps per device (kernel attributes, device properties): a
@@ -177,14 +181,14 @@ void rnn_backward_step(Launcher& lc, int dtype, const void* W, const void* deriv
 void convert_to_f64(Launcher& lc, int dtype, const void* src, double* dst, int64_t elems);
 // The same recurrences as ONE launch over all T steps (rnn_persistent.cu): clusters of 16 CTAs own 4 batch rows
 // each, the recurrent matrix stays in registers, the state moves between the CTAs through distributed shared
-// memory.  P is scratch of rnn_persistent_proj_bytes(...) bytes for U x_t of every step in double (0 = the width is
+// memory.  status: device status word for the kernel's bounded waits.  P is scratch of rnn_persistent_proj_bytes(...) bytes for U x_t of every step in double (0 = the width is
 // not one this form takes).  Both return false when nothing was done for the recurrence (unsupported width, or
 // clusters of 16 cannot be scheduled on this device): the caller then runs the per-step kernels.
 size_t rnn_persistent_proj_bytes(int T, int64_t B, int d);
 bool rnn_forward_persistent(Launcher& lc, int dtype, const void* W, const void* U, const void* X, const void* gate,
-                            const void* x0, double* P, void* x_all, void* deriv, int T, int B, int d, int in_dim);
+                            const void* x0, double* P, void* x_all, void* deriv, int T, int B, int d, int in_dim, int* status);
 bool rnn_backward_persistent(Launcher& lc, int dtype, const void* W, const void* gate, const void* deriv,
-                             const void* delta, void* g_all, int T, int B, int d);
+                             const void* delta, void* g_all, int T, int B, int d, int* status);
 
 // ---------------------------------------------------------------- diagnostics (diag.cu)
 // out[seg][4] = {<a,b>, |a|^2, |b|^2, |a-b|^2} over `elems` elements per segment; scratch holds

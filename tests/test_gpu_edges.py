@@ -208,6 +208,36 @@ def test_gemm_single_cta_and_cta_pair_modes_match_oracle(name, ks, mode, monkeyp
     compare(w, gpu, ref, ks, ("exact", kmax))
 
 
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """The failure path of the tensor-core kernels' waits: a GEMM tile whose copy role expects bytes that nobody
+    sends, every wait limited to 1 ms.  The kernel must end by itself, the status word must read HBP_ERR_TIMEOUT (8)
+    once, and afterwards the same context (same tensor memory, same status word) must compute correctly."""
+    import time
+    from oracle import run as orun
+    from paper_2501_17086_b200 import binding as B, harness
+    from paper_2501_17086_b200.workloads import WORKLOADS, make_inputs
+    w = WORKLOADS["c2_twin"]
+    inp = make_inputs(w, "cuda")
+    ctx = harness.make_context(w)
+    params = harness.params_for(w, inp)
+    x_all = ctx.forward(params, inp["x0"], None)
+    ctx.sync_status()
+    t0 = time.perf_counter()
+    ctx.selftest_wait_timeout(limit_ns=1_000_000)
+    with pytest.raises(B.HbpError) as info:
+        ctx.sync_status()
+    assert info.value.code == 8
+    assert time.perf_counter() - t0 < 5.0           # the waits gave up after milliseconds, not after their usual seconds
+    ctx.sync_status()                               # reported once; the word is clean again
+    # the context is usable: the same kernels, now with their copies, give the right answer
+    delta = harness.loss_delta(w, x_all, inp)
+    g = ctx.backward(params, 2, delta, x_all, None)
+    ctx.sync_status()
+    ref = orun.run(w, inp, ks=(2,))
+    for l in range(w.steps + 1):
+        assert rel(np64(g[l]), ref["hbp"][2][l]) < 2e-2, l
+
+
 def test_kernel_modes_belong_to_the_context(monkeypatch):
     """Two contexts created under different settings keep their own modes, and a call through either launches its own
     kind of kernels however the calls are interleaved: the modes read back as created, the CUDA-core context

@@ -34,24 +34,31 @@ def _relabelled(w, inp, perm):
     return out
 
 
-def _oracle_floor(w, inp, rows, base_exact):
-    """How far two fp64 evaluations of exact backpropagation through the same recurrent network lie apart when only
-    the order of their sums differs (units renumbered): the resolution at which the oracle itself defines the exact
-    gradient.  A recurrence whose forward map amplifies perturbations (c3: ||g_0|| / ||g_T|| ~ 1e13 over 4096 steps)
-    turns the 1e-16 of double rounding into 1e-7 on the late states and 1e-5 on the gradient, whatever the
-    implementation; nothing can be compared with the oracle more finely than that."""
+def _oracle_floor(w, inp, rows, ref, ks):
+    """How far two fp64 evaluations of the same recurrent network lie apart when only the order of their sums
+    differs (units renumbered): the resolution at which the oracle itself defines each gradient.  A recurrence
+    whose forward map amplifies perturbations (c3: ||g_0|| / ||g_T|| ~ 1e13 over 4096 steps) turns the 1e-16 of
+    double rounding into 1e-7 on the late states and 1e-5 on gradients that pass through them, whatever the
+    implementation; nothing can be compared with the oracle more finely than that.  Returns {"exact" | k: floor}."""
     n = w.hidden if w.block == "lstm" else w.d
     perm = np.random.default_rng(w.seed).permutation(n)
     inv = np.argsort(perm)
-    ref2 = orun.run(w, _relabelled(w, inp, perm), ks=(), rows=rows)
+    ref2 = orun.run(w, _relabelled(w, inp, perm), ks=ks, rows=rows)
     halves = w.d // n
-    worst = 0.0
-    for a, b in zip(ref2["exact"], base_exact):
-        a = a.reshape(*a.shape[:-1], halves, n)[..., inv].reshape(b.shape)
-        nb = np.linalg.norm(b)
-        if nb:
-            worst = max(worst, float(np.linalg.norm(a - b) / nb))
-    return worst
+
+    def worst(mine, base):
+        out = 0.0
+        for a, b in zip(mine, base):
+            a = a.reshape(*a.shape[:-1], halves, n)[..., inv].reshape(b.shape)
+            nb = np.linalg.norm(b)
+            if nb:
+                out = max(out, float(np.linalg.norm(a - b) / nb))
+        return out
+
+    floors = {"exact": worst(ref2["exact"], ref["exact"])}
+    for k in ks:
+        floors[k] = worst(ref2["hbp"][k], ref["hbp"][k])
+    return floors
 
 
 def _rows_of(w, t, rows):
@@ -140,17 +147,20 @@ def test_full_size_sampled_units(name, ks, rows):
                 worst = max(worst, rel(got_k[l], ref_k[l]))
         return worst
 
+    # float recurrent workloads: nothing is compared more finely than the oracle defines it (see _oracle_floor);
+    # 4 x: the floor is one sample of a quantity that varies with the order of the sums.  It only matters on c3
+    # (about 2e-5 for exact BPTT, a few 1e-6 for k = 8); on the other workloads it is 1e-15 and the bar stays 1e-5.
+    floors = _oracle_floor(w, inp, rows_t.cpu(), ref, ks) if (w.block in RECURRENT and w.dtype == "f32") else {}
     for k in ks:
         worst = worst_over_states(got[k], ref["hbp"][k])
-        assert worst < tol, f"k={k}: max rel-L2 {worst:.3e}"
+        tol_k = max(tol, 4.0 * floors.get(k, 0.0))
+        if floors:
+            print(f"{name}: k={k} error {worst:.3e}, oracle floor {floors[k]:.3e}")
+        assert worst < tol_k, f"k={k}: max rel-L2 {worst:.3e}"
     worst = max(rel(got["exact"][l], ref["exact"][l]) for l in range(w.steps + 1))
-    tol_exact = tol
-    if w.block in RECURRENT and w.dtype == "f32":
-        # exact BPTT is compared no more finely than the oracle defines it (see _oracle_floor); 4 x: the floor is
-        # one sample of a quantity that varies with the order of the sums
-        floor = _oracle_floor(w, inp, rows_t.cpu(), ref["exact"])
-        tol_exact = max(tol, 4.0 * floor)
-        print(f"{name}: exact BPTT error {worst:.3e}, oracle floor {floor:.3e}")
+    tol_exact = max(tol, 4.0 * floors.get("exact", 0.0))
+    if floors:
+        print(f"{name}: exact BPTT error {worst:.3e}, oracle floor {floors['exact']:.3e}")
     assert worst < tol_exact, f"exact: max rel-L2 {worst:.3e}"
     # tail exactness on the GPU itself (Theorem 2): g^k_l is already exact for l >= steps - k
     kmax = max(ks)
