@@ -114,7 +114,7 @@ __device__ __forceinline__ void residual_chunk(const TcParams& p, int b, int row
 }
 
 // ------------------------------------------------------------------------------------------- kernel
-template <bool kPair>
+template <bool kPair, bool kTf32>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
@@ -183,8 +183,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const uint32_t tmem_base = *tmem_slot;
   const int tiles_per_batch = p.m_tiles * p.n_tiles;
   // per element size: elements per 128-byte row (= K elements per stage), bytes of one MN-major block
-  const int row_elems = p.tf32 ? 32 : 64;
-  const uint32_t mn_block = p.tf32 ? 4096u : 8192u;
+  const int row_elems = kTf32 ? 32 : 64;
+  const uint32_t mn_block = kTf32 ? 4096u : 8192u;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -244,44 +244,60 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && leader) {
-      const uint32_t fmt = p.tf32 ? 2u : 1u;  // operand format: tf32 or bf16
+      const uint32_t fmt = kTf32 ? 2u : 1u;  // operand format: tf32 or bf16
       const uint32_t idesc = (1u << 4) /*fp32 accumulate*/ | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn << 15) |
                              ((uint32_t)p.b_mn << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
-      // one instruction consumes 32 bytes of K: 32 bytes along a K-major row, or 16 rows of an MN-major bf16 block
-      const uint32_t a_step = p.a_mn ? 2048u : 32u, b_step = p.b_mn ? 2048u : 32u;
-      const uint32_t a_lead = p.a_mn ? mn_block : 16u, b_lead = p.b_mn ? mn_block : 16u;
+      // one instruction consumes 32 bytes of K: 32 bytes along a K-major row, or 16 rows of an MN-major bf16 block.
+      // Descriptors differ between stages and k-steps only in their start address (bits 0..13, in 16-byte units):
+      // they are formed once and advanced by adding to the low word.
+      const uint32_t a_step16 = (p.a_mn ? 2048u : 32u) >> 4, b_step16 = (p.b_mn ? 2048u : 32u) >> 4;
+      const uint64_t adesc0 = make_desc(base, p.a_mn ? mn_block : 16u, 1024u);
+      const uint64_t bdesc0 = make_desc(base + A_BYTES, p.b_mn ? mn_block : 16u, 1024u);
+      constexpr uint32_t kStage16 = (uint32_t)STAGE_BYTES >> 4;
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
+      // The tensor core idles whenever this thread takes longer between two MMAs than one MMA runs, so nothing that
+      // has to wait for an answer sits between them: the barrier of the NEXT stage (and of the next tile's
+      // accumulator) is only tested, without blocking, before the current stage's MMAs go out, and the answer is
+      // looked at afterwards; the blocking wait is the fallback when that test said "not yet".
+      bool stage_ready = false, acc_ready = false;
       for (int tile = first_tile; tile < p.num_tiles && ok; tile += tile_step) {
-        if (!mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.status, p.wait_limit_ns)) { ok = false; break; }
+        if (!acc_ready && !mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, p.status, p.wait_limit_ns)) { ok = false; break; }
+        acc_ready = false;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)acc * BN;
         const int split = (tile / tiles_per_batch) / p.batch;
         const int kb_lo = split * p.kb_per_split, kb_hi = min(p.k_blocks, kb_lo + p.kb_per_split);
-        uint32_t first = 1;
-        for (int it = (kb_hi - kb_lo) * p.segs; it > 0; --it) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, p.wait_limit_ns)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t sA = base + stage * STAGE_BYTES, sB = sA + A_BYTES;
+        uint32_t accum = 0;
+        const int n_it = (kb_hi - kb_lo) * p.segs;
+        for (int it = 0; it < n_it; ++it) {
+          if (!stage_ready && !mbar_wait(full_bar(stage), phase, abort_flag, p.status, p.wait_limit_ns)) { ok = false; break; }
+          const int next_stage = stage + 1 == STAGES ? 0 : stage + 1;
+          const uint32_t next_phase = next_stage == 0 ? phase ^ 1u : phase;
+          const bool peek = mbar_test_wait(full_bar(next_stage), next_phase);
+          bool peek_acc = false;
+          if (it == n_it - 1) peek_acc = mbar_test_wait(acce_bar(acc ^ 1), (acc == 1 ? acc_phase ^ 1u : acc_phase) ^ 1u);
+          const uint64_t ad = adesc0 + (uint64_t)((uint32_t)stage * kStage16), bd = bdesc0 + (uint64_t)((uint32_t)stage * kStage16);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
-            const uint64_t ad = make_desc(sA + k * a_step, a_lead, 1024u);
-            const uint64_t bd = make_desc(sB + k * b_step, b_lead, 1024u);
-            const uint32_t accum = (first && k == 0) ? 0u : 1u;
+            const uint64_t adk = ad + (uint64_t)(k * a_step16), bdk = bd + (uint64_t)(k * b_step16);
             if (kPair) {
-              if (p.tf32) tc_mma_tf32_pair(tmem_d, ad, bd, idesc, accum);
-              else tc_mma_pair(tmem_d, ad, bd, idesc, accum);
+              if (kTf32) tc_mma_tf32_pair(tmem_d, adk, bdk, idesc, accum);
+              else tc_mma_pair(tmem_d, adk, bdk, idesc, accum);
             } else {
-              if (p.tf32) tc_mma_tf32(tmem_d, ad, bd, idesc, accum);
-              else tc_mma(tmem_d, ad, bd, idesc, accum);
+              if (kTf32) tc_mma_tf32(tmem_d, adk, bdk, idesc, accum);
+              else tc_mma(tmem_d, adk, bdk, idesc, accum);
             }
+            accum = 1;
           }
-          first = 0;
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
           if (kPair) tc_commit_pair(empty_bar(stage));
           else tc_commit(empty_bar(stage));
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          stage_ready = peek;
+          if (it == n_it - 1) acc_ready = peek_acc;
+          stage = next_stage;
+          phase = next_phase;
         }
         if (!ok) break;
         if (kPair) tc_commit_pair(accf_bar(acc));  // accumulator complete (each CTA holds its 128 rows of it)
@@ -575,9 +591,8 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   if (g.epi == EPI_MUL && !g.E) return false;
   if (g.epi == EPI_RESID && !g.R && !g.E) return false;
 
-  // CTA pairs only on request and when there are at least two 128-row blocks: measured on the MLP shapes the
-  // pair mode halves the MMA thread's waits for operands but its MMAs run slower (about 200 cycles against
-  // about 175 per 128 x 256 x 16 of work per SM), which nets out even
+  // CTA pairs wherever there are at least two 128-row blocks (unless the context asks for single CTAs): a stage is
+  // 32 KB instead of 48 KB for the same flops per SM, so the ring is six stages deep and draws a third less from L2
   const int sms = sm_count();
   const bool pair = lc.gemm_pair && sms >= 2 && g.M > BM;
   const int b_rows = pair ? Mode<true>::kBRows : Mode<false>::kBRows;
@@ -617,8 +632,10 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   static PerDevice<bool> attr_done;  // the shared-memory opt-in is a per-device attribute of the kernel
   bool& attr_set = attr_done.here();
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+    if (cudaFuncSetAttribute(gemm_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return false;
     }
@@ -657,11 +674,13 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<true>, tmA, tmB, tmA1, tmB1, tmA2, tmB2, tmD, tmD2, tmE, p);
+    cudaError_t e = f32 ? cudaLaunchKernelEx(&cfg, gemm_tc_kernel<true, true>, tmA, tmB, tmA1, tmB1, tmA2, tmB2, tmD, tmD2, tmE, p)
+                        : cudaLaunchKernelEx(&cfg, gemm_tc_kernel<true, false>, tmA, tmB, tmA1, tmB1, tmA2, tmB2, tmD, tmD2, tmE, p);
     if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
   } else {
     const int grid = p.num_tiles < sms ? p.num_tiles : sms;
-    gemm_tc_kernel<false><<<grid, THREADS, SMEM_BYTES, lc.stream>>>(tmA, tmB, tmA1, tmB1, tmA2, tmB2, tmD, tmD2, tmE, p);
+    if (f32) gemm_tc_kernel<false, true><<<grid, THREADS, SMEM_BYTES, lc.stream>>>(tmA, tmB, tmA1, tmB1, tmA2, tmB2, tmD, tmD2, tmE, p);
+    else gemm_tc_kernel<false, false><<<grid, THREADS, SMEM_BYTES, lc.stream>>>(tmA, tmB, tmA1, tmB1, tmA2, tmB2, tmD, tmD2, tmE, p);
   }
   lc.count();
   lc.check();

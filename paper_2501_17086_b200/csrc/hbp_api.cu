@@ -26,7 +26,7 @@ struct ProfSeg {
 
 struct hbp_ctx {
   hbp_config cfg;
-  // kernel-selection modes, read from the environment (HBP_FORCE_SIMT=1, HBP_GEMM_PAIR=1) when THIS context is
+  // kernel-selection modes, read from the environment (HBP_FORCE_SIMT=1, HBP_GEMM_PAIR=0) when THIS context is
   // created and kept with it: another context created later under other settings does not change them
   bool force_simt = false, gemm_pair = false;
   bool profiling = false;
@@ -780,7 +780,7 @@ hbp_status hbp_create(const hbp_config* cfg, void* workspace, size_t workspace_b
   const char* env = std::getenv("HBP_FORCE_SIMT");
   c->force_simt = env && env[0] == '1';
   const char* pm = std::getenv("HBP_GEMM_PAIR");
-  c->gemm_pair = pm && pm[0] == '1';
+  c->gemm_pair = !(pm && pm[0] == '0');  // pairs by default
   if (cudaMemset(c->status, 0, 256) != cudaSuccess) {
     delete c;
     return HBP_ERR_CUDA;

@@ -82,7 +82,7 @@ struct Launcher {
   int64_t* launches = nullptr;
   cudaError_t err = cudaSuccess;
   bool force_simt = false;  // keep every GEMM and attention product on the CUDA-core kernels (cross-checks)
-  bool gemm_pair = false;   // tensor-core GEMM pairs CTAs (cta_group::2, 256 x 256 tiles) where there are two row blocks
+  bool gemm_pair = true;    // tensor-core GEMM pairs CTAs (cta_group::2, 256 x 256 tiles) where there are two row blocks
   void count(int n = 1) {
     if (launches) *launches += n;
   }

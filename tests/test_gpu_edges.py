@@ -194,7 +194,7 @@ def test_cuda_core_fallback_matches_oracle(name, ks, monkeypatch):
 @pytest.mark.parametrize("name,ks", [("c2_twin", (2,)), ("c5_twin", (3,)), ("c4_twin", (2,)), ("c3_twin", (2,)), ("gru_twin", (2,))])
 def test_gemm_single_cta_and_cta_pair_modes_match_oracle(name, ks, mode, monkeypatch):
     """HBP_GEMM_PAIR (read when a context is made): 0 keeps the tensor-core GEMM on single CTAs (128 x 256 tiles),
-    1 pairs CTAs (256 x 256 tiles) wherever two row blocks exist; both must meet the bar on every twin."""
+    1 (the default) pairs CTAs (256 x 256 tiles) wherever two row blocks exist; both must meet the bar on every twin."""
     from oracle import run as orun
     from paper_2501_17086_b200.workloads import WORKLOADS, make_inputs
     from test_gpu_parity import compare, run_gpu
@@ -247,12 +247,14 @@ def test_kernel_modes_belong_to_the_context(monkeypatch):
     w = WORKLOADS["c2_twin"]
     inp = make_inputs(w, "cuda")
     monkeypatch.setenv("HBP_FORCE_SIMT", "1")
+    monkeypatch.setenv("HBP_GEMM_PAIR", "0")
     simt = harness.make_context(w)
     monkeypatch.delenv("HBP_FORCE_SIMT")
-    monkeypatch.setenv("HBP_GEMM_PAIR", "1")
-    pair = harness.make_context(w)
     monkeypatch.delenv("HBP_GEMM_PAIR")
+    pair = harness.make_context(w)               # the default: paired CTAs
+    monkeypatch.setenv("HBP_GEMM_PAIR", "0")
     plain = harness.make_context(w)
+    monkeypatch.delenv("HBP_GEMM_PAIR")
     assert (simt.modes, pair.modes, plain.modes) == (1, 2, 0)
     params = harness.params_for(w, inp)
     outs = []
