@@ -52,6 +52,19 @@ constexpr uint32_t make_idesc(int b_mn) {
 }
 constexpr uint32_t IDESC_KK = make_idesc(0), IDESC_KMN = make_idesc(1);
 
+// One lane of a converged warp.  The MMA warps below stay converged through their whole loop - every lane runs the
+// waits and the address arithmetic, which the compiler can then keep on the uniform datapath - and only the
+// tcgen05 instructions themselves are predicated on the elected lane.  Issued from inside an `if (lane == 0)`
+// region instead, with descriptors formed per instruction, one MMA cost the issuing thread about 120 cycles,
+// four times what a 128 x 64 x 16 MMA takes to run; converged and with descriptors formed once, about 50.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t is_leader;
+  asm volatile("{\n\t.reg .pred q;\n\telect.sync _|q, 0xffffffff;\n\tselp.u32 %0, 1, 0, q;\n\t}" : "=r"(is_leader));
+  return is_leader != 0;
+}
+// descriptor `d` moved by `bytes` within shared memory (the start address sits in the low bits, in 16-byte units)
+__device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
+
 // Barrier slots (8 bytes each):
 // 0 big tiles loaded, 1-2 full[2], 3-4 empty[2], 5 scores ready, 6 probabilities ready, 7 all MMAs done,
 // 8 scores copied out of tensor memory (the next block's score MMAs may overwrite them).
@@ -146,63 +159,61 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      // Software pipeline: the score MMAs of block it+1 are issued as soon as the softmax warps have copied the
-      // scores of block it out of tensor memory, so they run under the exp / pack work of block it; the
-      // accumulating MMAs of block it follow once its probabilities are in shared memory.
-      auto issue_scores = [&](int it) {
-        const int buf = it & 1;
-        const uint32_t s0 = sSmall + (2 * buf) * SMALL_BYTES, s1 = s0 + SMALL_BYTES;
+    // Software pipeline: the score MMAs of block it+1 are issued as soon as the softmax warps have copied the
+    // scores of block it out of tensor memory, so they run under the exp / pack work of block it; the
+    // accumulating MMAs of block it follow once its probabilities are in shared memory.
+    const bool leader = elect_one();
+    // descriptors of every tile, formed once (buffer 1 of the small tiles lies 2 * SMALL_BYTES after buffer 0)
+    const uint64_t dBig0 = make_desc(sBig0, 16, 1024), dBig1 = make_desc(sBig1, 16, 1024);
+    const uint64_t dS0kk = make_desc(sSmall, 16, 1024), dS1kk = make_desc(sSmall + SMALL_BYTES, 16, 1024);
+    const uint64_t dS0mn = make_desc(sSmall, 8192, 1024), dS1mn = make_desc(sSmall + SMALL_BYTES, 8192, 1024);
+    const uint64_t dPt = make_desc(sP, 16, 1024), dDSt = make_desc(sDS, 16, 1024);
+    auto issue_scores = [&](int it) {
+      const uint32_t boff = (uint32_t)(it & 1) * (2 * SMALL_BYTES);
+      if (leader) {
         // scores and dP: contraction over the head dimension, both operands K-major
 #pragma unroll
-        for (int k = 0; k < DH / 16; ++k)
-          tc_mma(tS, make_desc(sBig0 + 32 * k, 16, 1024), make_desc(s0 + 32 * k, 16, 1024), IDESC_KK, k != 0);
+        for (int k = 0; k < DH / 16; ++k) tc_mma(tS, desc_add(dBig0, 32 * k), desc_add(dS0kk, boff + 32 * k), IDESC_KK, k != 0);
 #pragma unroll
-        for (int k = 0; k < DH / 16; ++k)
-          tc_mma(tDP, make_desc(sBig1 + 32 * k, 16, 1024), make_desc(s1 + 32 * k, 16, 1024), IDESC_KK, k != 0);
+        for (int k = 0; k < DH / 16; ++k) tc_mma(tDP, desc_add(dBig1, 32 * k), desc_add(dS1kk, boff + 32 * k), IDESC_KK, k != 0);
         tc_commit(bar_at(bars, 5));
-      };
-      bool ok = mbar_wait(bar_at(bars, 0), 0, abort_flag, p.status);
-      ok = ok && mbar_wait(bar_at(bars, 1), 0, abort_flag, p.status);
-      tc_fence_after();
-      if (ok) issue_scores(0);
-      for (int it = 0; it < n_it && ok; ++it) {
-        const int buf = it & 1;
-        const uint32_t itp = (uint32_t)it & 1u;
-        if (it + 1 < n_it) {
-          const int nb = (it + 1) & 1;
-          if (!mbar_wait(bar_at(bars, 1 + nb), (uint32_t)((it + 1) >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
-          if (!mbar_wait(bar_at(bars, 8), itp, abort_flag, p.status)) { ok = false; break; }
-          tc_fence_after();
-          issue_scores(it + 1);
-        }
-        const uint32_t s0 = sSmall + (2 * buf) * SMALL_BYTES, s1 = s0 + SMALL_BYTES;
-        if (!mbar_wait(bar_at(bars, 6), itp, abort_flag, p.status)) { ok = false; break; }
+      }
+    };
+    bool ok = mbar_wait(bar_at(bars, 0), 0, abort_flag, p.status);
+    ok = ok && mbar_wait(bar_at(bars, 1), 0, abort_flag, p.status);
+    tc_fence_after();
+    if (ok) issue_scores(0);
+    for (int it = 0; it < n_it && ok; ++it) {
+      const int buf = it & 1;
+      const uint32_t itp = (uint32_t)it & 1u;
+      if (it + 1 < n_it) {
+        const int nb = (it + 1) & 1;
+        if (!mbar_wait(bar_at(bars, 1 + nb), (uint32_t)((it + 1) >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(bar_at(bars, 8), itp, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
-        // accumulate: contraction over the 64 rows of the small tiles, which are MN-major B operands here
-        const uint32_t acc_on = it != 0 ? 1u : 0u;
+        issue_scores(it + 1);
+      }
+      if (!mbar_wait(bar_at(bars, 6), itp, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      // accumulate: contraction over the 64 rows of the small tiles, which are MN-major B operands here
+      const uint32_t acc_on = it != 0 ? 1u : 0u;
+      const uint32_t boff = (uint32_t)buf * (2 * SMALL_BYTES);
+      if (leader) {
         if (kDKV) {
 #pragma unroll
           for (int k = 0; k < SMALL / 16; ++k)  // dV += P^T dO
-            tc_mma(tAcc1, make_desc(sP + 32 * k, 16, 1024), make_desc(s1 + 2048 * k, 8192, 1024), IDESC_KMN,
-                   acc_on | (k != 0));
-#pragma unroll
-          for (int k = 0; k < SMALL / 16; ++k)  // dK += dS^T Q
-            tc_mma(tAcc0, make_desc(sDS + 32 * k, 16, 1024), make_desc(s0 + 2048 * k, 8192, 1024), IDESC_KMN,
-                   acc_on | (k != 0));
-        } else {
-#pragma unroll
-          for (int k = 0; k < SMALL / 16; ++k)  // dQ += dS K
-            tc_mma(tAcc0, make_desc(sDS + 32 * k, 16, 1024), make_desc(s0 + 2048 * k, 8192, 1024), IDESC_KMN,
-                   acc_on | (k != 0));
+            tc_mma(tAcc1, desc_add(dPt, 32 * k), desc_add(dS1mn, boff + 2048 * k), IDESC_KMN, acc_on | (k != 0));
         }
+#pragma unroll
+        for (int k = 0; k < SMALL / 16; ++k)  // dK += dS^T Q   /   dQ += dS K
+          tc_mma(tAcc0, desc_add(dDSt, 32 * k), desc_add(dS0mn, boff + 2048 * k), IDESC_KMN, acc_on | (k != 0));
         tc_commit(bar_at(bars, 3 + buf));
       }
-      tc_commit(bar_at(bars, 7));
-      if (!ok) {
-        const uint64_t t0 = global_ns();
-        while (!mbar_try_wait(bar_at(bars, 7), 0) && global_ns() - t0 < 100000000ull) {
-        }
+    }
+    if (leader) tc_commit(bar_at(bars, 7));
+    if (!ok) {
+      const uint64_t t0 = global_ns();
+      while (!mbar_try_wait(bar_at(bars, 7), 0) && global_ns() - t0 < 100000000ull) {
       }
     }
   } else {
@@ -397,44 +408,48 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      auto issue_scores = [&](int it) {
-        const uint32_t s0 = sSmall + (2 * (it & 1)) * SMALL_BYTES;
+    // converged warp, one elected lane issues (see elect_one); descriptors formed once
+    const bool leader = elect_one();
+    const uint64_t dQt = make_desc(sQ, 16, 1024), dKkk = make_desc(sSmall, 16, 1024);
+    const uint64_t dVmn = make_desc(sSmall + SMALL_BYTES, 8192, 1024), dPt = make_desc(sP, 16, 1024);
+    auto issue_scores = [&](int it) {
+      const uint32_t boff = (uint32_t)(it & 1) * (2 * SMALL_BYTES);
+      if (leader) {
 #pragma unroll
-        for (int k = 0; k < DH / 16; ++k)
-          tc_mma(tS, make_desc(sQ + 32 * k, 16, 1024), make_desc(s0 + 32 * k, 16, 1024), IDESC_KK, k != 0);
+        for (int k = 0; k < DH / 16; ++k) tc_mma(tS, desc_add(dQt, 32 * k), desc_add(dKkk, boff + 32 * k), IDESC_KK, k != 0);
         tc_commit(bar_at(bars, 5));
         if (it < n_kb) tc_commit(bar_at(bars, 3 + (it & 1)));  // sweep 1: the K tile is free once the scores are formed
-      };
-      bool ok = mbar_wait(bar_at(bars, 0), 0, abort_flag, p.status);
-      ok = ok && mbar_wait(bar_at(bars, 1), 0, abort_flag, p.status);
-      tc_fence_after();
-      if (ok) issue_scores(0);
-      for (int it = 0; it < n_it && ok; ++it) {
-        const int buf = it & 1;
-        if (it + 1 < n_it) {
-          const int nb = (it + 1) & 1;
-          if (!mbar_wait(bar_at(bars, 1 + nb), (uint32_t)((it + 1) >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
-          if (!mbar_wait(bar_at(bars, 8), (uint32_t)it & 1u, abort_flag, p.status)) { ok = false; break; }
-          tc_fence_after();
-          issue_scores(it + 1);
-        }
-        if (it < n_kb) continue;
-        const int j = it - n_kb;
-        if (!mbar_wait(bar_at(bars, 6), (uint32_t)j & 1u, abort_flag, p.status)) { ok = false; break; }
+      }
+    };
+    bool ok = mbar_wait(bar_at(bars, 0), 0, abort_flag, p.status);
+    ok = ok && mbar_wait(bar_at(bars, 1), 0, abort_flag, p.status);
+    tc_fence_after();
+    if (ok) issue_scores(0);
+    for (int it = 0; it < n_it && ok; ++it) {
+      const int buf = it & 1;
+      if (it + 1 < n_it) {
+        const int nb = (it + 1) & 1;
+        if (!mbar_wait(bar_at(bars, 1 + nb), (uint32_t)((it + 1) >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(bar_at(bars, 8), (uint32_t)it & 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t s1 = sSmall + (2 * buf + 1) * SMALL_BYTES;
+        issue_scores(it + 1);
+      }
+      if (it < n_kb) continue;
+      const int j = it - n_kb;
+      if (!mbar_wait(bar_at(bars, 6), (uint32_t)j & 1u, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t boff = (uint32_t)buf * (2 * SMALL_BYTES);
+      if (leader) {
 #pragma unroll
         for (int k = 0; k < SMALL / 16; ++k)  // O += P V: contraction over the 64 keys, V is an MN-major operand
-          tc_mma(tO, make_desc(sP + 32 * k, 16, 1024), make_desc(s1 + 2048 * k, 8192, 1024), IDESC_KMN,
-                 (j != 0 ? 1u : 0u) | (k != 0));
+          tc_mma(tO, desc_add(dPt, 32 * k), desc_add(dVmn, boff + 2048 * k), IDESC_KMN, (j != 0 ? 1u : 0u) | (k != 0));
         tc_commit(bar_at(bars, 3 + buf));
       }
-      tc_commit(bar_at(bars, 7));
-      if (!ok) {
-        const uint64_t t0 = global_ns();
-        while (!mbar_try_wait(bar_at(bars, 7), 0) && global_ns() - t0 < 100000000ull) {
-        }
+    }
+    if (leader) tc_commit(bar_at(bars, 7));
+    if (!ok) {
+      const uint64_t t0 = global_ns();
+      while (!mbar_try_wait(bar_at(bars, 7), 0) && global_ns() - t0 < 100000000ull) {
       }
     }
   } else {

@@ -243,7 +243,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0 && leader) {
+    // The whole warp runs this loop converged (waits, tests and address arithmetic in every lane, which lets the
+    // compiler keep them on the uniform datapath); only the tcgen05 instructions are predicated on one elected lane.
+    if (leader) {
+      uint32_t elected;
+      asm volatile("{\n\t.reg .pred q;\n\telect.sync _|q, 0xffffffff;\n\tselp.u32 %0, 1, 0, q;\n\t}" : "=r"(elected));
+      const bool issuer = elected != 0;
       const uint32_t fmt = kTf32 ? 2u : 1u;  // operand format: tf32 or bf16
       const uint32_t idesc = (1u << 4) /*fp32 accumulate*/ | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn << 15) |
                              ((uint32_t)p.b_mn << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
@@ -279,34 +284,41 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           bool peek_acc = false;
           if (it == n_it - 1) peek_acc = mbar_test_wait(acce_bar(acc ^ 1), (acc == 1 ? acc_phase ^ 1u : acc_phase) ^ 1u);
           const uint64_t ad = adesc0 + (uint64_t)((uint32_t)stage * kStage16), bd = bdesc0 + (uint64_t)((uint32_t)stage * kStage16);
+          if (issuer) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const uint64_t adk = ad + (uint64_t)(k * a_step16), bdk = bd + (uint64_t)(k * b_step16);
-            if (kPair) {
-              if (kTf32) tc_mma_tf32_pair(tmem_d, adk, bdk, idesc, accum);
-              else tc_mma_pair(tmem_d, adk, bdk, idesc, accum);
-            } else {
-              if (kTf32) tc_mma_tf32(tmem_d, adk, bdk, idesc, accum);
-              else tc_mma(tmem_d, adk, bdk, idesc, accum);
+            for (int k = 0; k < 4; ++k) {
+              const uint64_t adk = ad + (uint64_t)(k * a_step16), bdk = bd + (uint64_t)(k * b_step16);
+              const uint32_t acc_k = k == 0 ? accum : 1u;
+              if (kPair) {
+                if (kTf32) tc_mma_tf32_pair(tmem_d, adk, bdk, idesc, acc_k);
+                else tc_mma_pair(tmem_d, adk, bdk, idesc, acc_k);
+              } else {
+                if (kTf32) tc_mma_tf32(tmem_d, adk, bdk, idesc, acc_k);
+                else tc_mma(tmem_d, adk, bdk, idesc, acc_k);
+              }
             }
-            accum = 1;
+            // frees the stage (in both CTAs of a pair) once these MMAs have read it
+            if (kPair) tc_commit_pair(empty_bar(stage));
+            else tc_commit(empty_bar(stage));
           }
-          // frees the stage (in both CTAs of a pair) once these MMAs have read it
-          if (kPair) tc_commit_pair(empty_bar(stage));
-          else tc_commit(empty_bar(stage));
+          accum = 1;
           stage_ready = peek;
           if (it == n_it - 1) acc_ready = peek_acc;
           stage = next_stage;
           phase = next_phase;
         }
         if (!ok) break;
-        if (kPair) tc_commit_pair(accf_bar(acc));  // accumulator complete (each CTA holds its 128 rows of it)
-        else tc_commit(accf_bar(acc));
+        if (issuer) {
+          if (kPair) tc_commit_pair(accf_bar(acc));  // accumulator complete (each CTA holds its 128 rows of it)
+          else tc_commit(accf_bar(acc));
+        }
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
       if (!ok) {  // let issued MMAs finish before the tensor memory is freed
-        if (kPair) tc_commit_pair(drain_bar);
-        else tc_commit(drain_bar);
+        if (issuer) {
+          if (kPair) tc_commit_pair(drain_bar);
+          else tc_commit(drain_bar);
+        }
         uint64_t t0 = global_ns();
         while (!mbar_try_wait(drain_bar, 0) && global_ns() - t0 < 100000000ull) {
         }
