@@ -68,7 +68,8 @@ struct TcParams {
 // sharing exp(-z^2/2) between erf and the density; the tail is formed without cancellation.
 __device__ __forceinline__ void normal_cdf_pdf(float z, float& cdf, float& pdf) {
   const float ax = fabsf(z) * 0.70710678118654752440f;
-  const float t = __frcp_rn(fmaf(0.3275911f, ax, 1.0f));
+  float t;  // 1 / (1 + p |z| / sqrt 2) by the hardware reciprocal (relative error 2^-23: far below the formula's own)
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, ax, 1.0f)));
   const float e = __expf(-0.5f * z * z);
   float poly = fmaf(t, 1.061405429f, -1.453152027f);
   poly = fmaf(t, poly, 1.421413741f);

@@ -72,6 +72,8 @@ WORKLOADS = {
                    init="small", gamma=0.8),
     # c2 with 8 layers: same per-launch tile shapes, small enough for multi-pass profiler captures
     "c2_small": Workload("c2_small", "preln_mlp", "bf16", L=8, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1012),
+    # c5 with 4 layers: same tile shapes per launch, small enough for multi-pass profiler captures
+    "c5_small": Workload("c5_small", "preln_mlp", "bf16", L=4, d=2048, hidden=8192, batch=32, seq=512, tokens=16384, seed=1015),
     # c4 with 4 decoder blocks: same per-launch shapes, small enough for multi-pass profiler captures
     "c4_small": Workload("c4_small", "preln_transformer", "bf16", L=4, d=768, hidden=3072, n_heads=12, head_dim=64,
                          seq=1024, batch=16, tokens=16384, seed=1014),
