@@ -43,6 +43,13 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// A global load that stays where it is written: left to the compiler, a load whose value is first used one loop
+// iteration later is moved down to that use, and its latency is then waited for instead of hidden.
+__device__ __forceinline__ float ld_pinned(const float* ptr) {
+  float v;
+  asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(ptr));
+  return v;
+}
 __device__ __forceinline__ void named_barrier_softmax() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 64, A K-major, B K-major or MN-major
@@ -232,14 +239,29 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
       my_d = grow < p.S ? p.drow[(int64_t)b * p.d_sb + (int64_t)h * p.d_sh + (int64_t)grow * p.d_sq] : 0.0f;
     }
     bool ok = true;  // false after a wait gave up: keep pace with the named barriers, do no more work
+    // dkv: thread t < 64 fetches the log-sum-exp of query t of a block, thread 64 + t its D
+    // dkv: the statistics belong to the block's queries (columns).  Lane c of a warp fetches those of column
+    // ch * 32 + c one block ahead (raw values: nothing waits for the loads) and the lanes exchange them by shuffle in
+    // the element loop: no staging through shared memory, no barrier among the softmax warps per block.
+    auto load_lse = [&](int it) -> float {
+      const int q = (it_beg + it) * SMALL + ch * 32 + lane;
+      return q < p.S ? ld_pinned(p.lse + stat_base + q) : INFINITY;
+    };
+    auto load_dd = [&](int it) -> float {
+      const int q = (it_beg + it) * SMALL + ch * 32 + lane;
+      return q < p.S ? ld_pinned(p.drow + (int64_t)b * p.d_sb + (int64_t)h * p.d_sh + (int64_t)q * p.d_sq) : 0.0f;
+    };
+    float lse_next = (kDKV && n_it > 0) ? load_lse(0) : 0.0f, dd_next = (kDKV && n_it > 0) ? load_dd(0) : 0.0f;
     for (int it = 0; it < n_it; ++it) {
       const int c0 = (it_beg + it) * SMALL;  // first query (dkv) / key (dq) of the small block
-      float* vb = vec + (it & 1) * 128;
-      if (kDKV) {  // statistics of the 64 queries of this block, shared by all rows
-        const int q = c0 + (t & 63);
-        if (t < 64) vb[t] = q < p.S ? p.lse[stat_base + q] * LOG2E : INFINITY;
-        else if (t < 128) vb[t] = q < p.S ? p.drow[(int64_t)b * p.d_sb + (int64_t)h * p.d_sh + (int64_t)q * p.d_sq] : 0.0f;
-        named_barrier_softmax();
+      float col_lse = 0.0f, col_dd = 0.0f;  // dkv: this lane's column statistics of the current block
+      if (kDKV) {
+        col_lse = lse_next * LOG2E;
+        col_dd = dd_next;
+        if (it + 1 < n_it) {
+          lse_next = load_lse(it + 1);
+          dd_next = load_dd(it + 1);
+        }
       }
       if (!ok) continue;
       if (!mbar_wait(bar_at(bars, 5), (uint32_t)it & 1u, abort_flag, p.status)) { ok = false; continue; }
@@ -257,8 +279,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
       if (full) {
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
-          const float lse2 = kDKV ? vb[ch * 32 + c] : my_lse;
-          const float dd = kDKV ? vb[64 + ch * 32 + c] : my_d;
+          const float lse2 = kDKV ? __shfl_sync(0xffffffffu, col_lse, c) : my_lse;
+          const float dd = kDKV ? __shfl_sync(0xffffffffu, col_dd, c) : my_d;
           const float pr = fast_exp2(fmaf(sc[c], scale2, -lse2));
           sc[c] = pr;
           dp[c] = pr * (dp[c] - dd);
@@ -267,8 +289,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
           const int col = c0 + ch * 32 + c;
-          const float lse2 = kDKV ? vb[ch * 32 + c] : my_lse;
-          const float dd = kDKV ? vb[64 + ch * 32 + c] : my_d;
+          const float lse2 = kDKV ? __shfl_sync(0xffffffffu, col_lse, c) : my_lse;
+          const float dd = kDKV ? __shfl_sync(0xffffffffu, col_dd, c) : my_d;
           // dkv: row = key, column = query; dq: row = query, column = key
           const bool vis = kDKV ? ((col >= grow) && (grow < p.S)) : ((col <= grow) && (col < p.S));
           const float pr = vis ? fast_exp2(fmaf(sc[c], scale2, -lse2)) : 0.0f;
