@@ -93,7 +93,6 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
   const uint32_t sP = sSmall + 4 * SMALL_BYTES;            // P^T (dkv only)
   const uint32_t sDS = sP + PS_BYTES;                      // dS^T / dS
   constexpr int VEC_OFF = 2 * BIG_BYTES + 4 * SMALL_BYTES + 2 * PS_BYTES;
-  float* vec = reinterpret_cast<float*>(aligned + VEC_OFF);  // [2 buffers][lse 64 | D 64]
   uint64_t* bar_mem = reinterpret_cast<uint64_t*>(aligned + VEC_OFF + 1024);
   const uint32_t bars = smem_u32(bar_mem);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 10);
