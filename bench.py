@@ -50,20 +50,29 @@ def config_of(w, k):
 # profiles/.  An entry is used only while the kernel's sources still hash to the value recorded with the capture and
 # the workload has the captured shapes; otherwise the bench line carries "traffic": null.
 TRAFFIC = {
-    # gemm_tc_kernel, VJP pair (dA + dY) on c2_small: 1242.949 MB + 895.901 MB for 8 layers x 8192 tokens
-    "gemm_vjp": {"sources": ("gemm_tc.cu", "tc_common.cuh"),
-                 "sha256": "79b4e446ad5f9877",
-                 "shape": ("preln_mlp", "bf16", 1024, 4096), "bytes_per_token_layer": (1242.949e6 + 895.901e6) / (8 * 8192),
-                 "profile": "profiles/gemm_tc_kernel_c2_small.md"},
-    # scan_depth_lnstat_kernel on c2_small: 286.271 MB read + 80.401 MB written for 8 steps x 8192 x 1024 elements
-    # (the writes still in L2 when that small launch ends are not in the counter)
-    "scan_lnstat": {"sources": ("scan.cu",), "sha256": "5efee60609bc121d", "shape": ("preln_mlp", "bf16", 1024, 4096),
-                    "bytes_per_state_element_step": (286.271e6 + 80.401e6) / (8 * 8192 * 1024),
-                    "profile": "profiles/scan_depth_lnstat_kernel_c2_small.md"},
-    # scan_ring_kernel on c3: 268.520 MB read + 217.638 MB written per scan
-    "scan_ring": {"sources": ("scan_ring.cu", "tc_common.cuh"), "sha256": "edb684e7b31e74f9", "shape": ("rnn_tanh", "f32", 512, 0),
-                  "bytes_per_state_element_step": (268.520e6 + 217.638e6) / (4096 * 32 * 512),
-                  "profile": "profiles/scan_ring_kernel_c3.md"},
+    # gemm_tc_kernel, VJP pair (dA + dY): c5_small (4 layers x 16384 tokens): 2119.775 + 1055.853 and 2864.423 + 279.595 MB;
+    # c2_small (8 layers x 8192 tokens): 741.016 + 506.177 and 808.292 + 132.456 MB
+    "gemm_vjp": [
+        {"sources": ("gemm_tc.cu", "tc_common.cuh"), "sha256": "1aac9fae53232ef1", "shape": ("preln_mlp", "bf16", 2048, 8192),
+         "bytes_per_token_layer": (2119.775e6 + 1055.853e6 + 2864.423e6 + 279.595e6) / (4 * 16384),
+         "profile": "profiles/gemm_tc_kernel_c5_small.md"},
+        {"sources": ("gemm_tc.cu", "tc_common.cuh"), "sha256": "1aac9fae53232ef1", "shape": ("preln_mlp", "bf16", 1024, 4096),
+         "bytes_per_token_layer": (741.016e6 + 506.177e6 + 808.292e6 + 132.456e6) / (8 * 8192),
+         "profile": "profiles/gemm_tc_kernel_c2_small.md"}],
+    # scan_depth_lnstat_kernel: c5_small 605.038 MB read + 215.374 MB written for 4 steps x 16384 x 2048 elements; c2_small
+    # 286.270 + 80.477 MB for 8 x 8192 x 1024 (the writes still in L2 when such a small launch ends are not in the counter)
+    "scan_lnstat": [
+        {"sources": ("scan.cu",), "sha256": "5efee60609bc121d", "shape": ("preln_mlp", "bf16", 2048, 8192),
+         "bytes_per_state_element_step": (605.038e6 + 215.374e6) / (4 * 16384 * 2048),
+         "profile": "profiles/scan_depth_lnstat_kernel_c5_small.md"},
+        {"sources": ("scan.cu",), "sha256": "5efee60609bc121d", "shape": ("preln_mlp", "bf16", 1024, 4096),
+         "bytes_per_state_element_step": (286.270e6 + 80.477e6) / (8 * 8192 * 1024),
+         "profile": "profiles/scan_depth_lnstat_kernel_c2_small.md"}],
+    # scan_ring_kernel on c3: 268.606 MB read + 219.337 MB written per scan
+    "scan_ring": [
+        {"sources": ("scan_ring.cu", "tc_common.cuh"), "sha256": "0dae6cd216ff4ebf", "shape": ("rnn_tanh", "f32", 512, 0),
+         "bytes_per_state_element_step": (268.606e6 + 219.337e6) / (4096 * 32 * 512),
+         "profile": "profiles/scan_ring_kernel_c3.md"}],
 }
 
 
@@ -77,16 +86,16 @@ def _sources_hash(names):
 
 
 def measured_traffic(key, w):
-    """Entry of TRAFFIC if it still describes the built kernel and this workload's shapes, else None."""
-    t = TRAFFIC[key]
-    if (w.block, w.dtype, w.d, w.hidden) != t["shape"]:
-        return None
-    try:
-        if _sources_hash(t["sources"]) != t["sha256"]:
-            return None
-    except OSError:
-        return None
-    return t
+    """Entry of TRAFFIC[key] that describes this workload's shapes, if the kernel still is the captured one, else None."""
+    for t in TRAFFIC[key]:
+        if (w.block, w.dtype, w.d, w.hidden) != t["shape"]:
+            continue
+        try:
+            if _sources_hash(t["sources"]) == t["sha256"]:
+                return t
+        except OSError:
+            pass
+    return None
 
 
 def algorithmic_flops(w, k):
