@@ -102,3 +102,12 @@ def test_new_entry_points_reject_bad_arguments_without_a_gpu(B):
     assert lib.hbp_workspace_bytes(C.byref(bad), C.byref(n)) == 2
     gated = B.make_config("gru", "f32", 6, 64, 4, in_dim=8, batch=4, gate=B.GATE_CHANNEL_SHARED)
     assert lib.hbp_workspace_bytes(C.byref(gated), C.byref(n)) == 6              # the cell's gate is the only one
+
+
+def test_diagnostic_entry_points_reject_bad_arguments_without_a_gpu(B):
+    lib = B.lib
+    assert lib.hbp_context_modes(None) == 0
+    assert lib.hbp_selftest_wait_timeout(None, None, 0, 1000000, None) == 1
+    # the scan with a status word: same argument checks as the plain one, plus the word's alignment
+    assert lib.hbp_cumsumprod_status(0, 0, 0, 16, 4, 8, None, None, None, None, None, 0, None, None) == 1
+    assert lib.hbp_cumsumprod_status(0, 0, 0, 16, 4, 8, None, None, None, None, None, 0, C.c_void_p(2), None) == 2

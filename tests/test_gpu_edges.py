@@ -208,6 +208,23 @@ def test_gemm_single_cta_and_cta_pair_modes_match_oracle(name, ks, mode, monkeyp
     compare(w, gpu, ref, ks, ("exact", kmax))
 
 
+def test_scan_with_a_status_word_reports_no_error_and_matches_the_plain_scan():
+    """hbp_cumsumprod_status on the ring scan (the form with bounded waits): same result as hbp_cumsumprod, status 0."""
+    from paper_2501_17086_b200 import binding as B
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    L, rows, d = 700, 4, 128
+    u = torch.randn((L, rows, d), generator=gen, device="cuda")
+    delta = torch.randn((L + 1, rows, d), generator=gen, device="cuda")
+    a = 0.9 + 0.099 * torch.rand((d,), generator=gen, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = B.cumsumprod(u, delta, a, loss=B.LOSS_EVERY_STEP, status=status)
+    want = B.cumsumprod(u, delta, a, loss=B.LOSS_EVERY_STEP)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(got, want)
+
+
 def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     """The failure path of the tensor-core kernels' waits: a GEMM tile whose copy role expects bytes that nobody
     sends, every wait limited to 1 ms.  The kernel must end by itself, the status word must read HBP_ERR_TIMEOUT (8)
