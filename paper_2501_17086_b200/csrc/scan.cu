@@ -146,7 +146,8 @@ __global__ void __launch_bounds__(256) scan_depth_kernel(const ScanArgs s) {
 #pragma unroll
     for (int i = 0; i < V; ++i) old_next[i] = (float)carry[i];
   }
-  for (int l = s.l_hi - 1; l >= s.l_lo; --l) {
+#pragma unroll 4
+  for (int l = s.l_hi - 1; l >= s.l_lo; --l) {  // unrolled: the loads of four steps in flight per thread
     A val[V];
     scan_step<T>(s, l, state_elems, off, ch, carry, val, row);
     if (kShift) {
@@ -184,6 +185,8 @@ __global__ void __launch_bounds__(256) scan_depth_lnstat_kernel(const ScanArgs s
 #pragma unroll
     for (int i = 0; i < V; ++i) old_next[i] = carry[i];
   }
+  // the loads of a step do not depend on the running value: unrolled, those of four steps are in flight per thread
+#pragma unroll 4
   for (int l = s.l_hi - 1; l >= s.l_lo; --l) {
     float dy[V], xh[V], val[V];
     ldv_stream<T>((const T*)s.u + (int64_t)l * state_elems + off).get(dy);
