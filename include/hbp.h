@@ -253,7 +253,11 @@ int64_t hbp_launch_count(const hbp_ctx* ctx);
 /* Kernel-selection modes of a context, fixed when it was created from the environment of that moment:
  * bit 0 = HBP_FORCE_SIMT=1 (every contraction on the CUDA-core kernels, a cross-check of the tensor-core ones),
  * bit 1 = the tensor-core GEMM pairs CTAs (tcgen05 cta_group::2, 256 x 256 tiles): the default; HBP_GEMM_PAIR=0
- * keeps single CTAs (128 x 256 tiles).  The modes belong to the context: contexts created
+ * keeps single CTAs (128 x 256 tiles),
+ * bit 2 = on the float tanh RNN the reverse scan between two all-step VJPs (Eq. 9 followed by Eq. 8) also writes
+ * the next VJP's left operand g_{t+1} * tanh'(z_t), split for the tensor cores, instead of the intermediate
+ * iterate: the default; HBP_SCAN_OPERAND=0 keeps the separate pass (same bits in every result, a cross-check).
+ * The modes belong to the context: contexts created
  * under other settings, before or after, keep their own.  One-time kernel set-up is likewise remembered per
  * device, so one process may hold contexts on several GPUs (each used with its device current). */
 int32_t hbp_context_modes(const hbp_ctx* ctx);

@@ -177,7 +177,8 @@ class Context:
 
     @property
     def modes(self) -> int:
-        """Bit 0: CUDA-core kernels forced; bit 1: paired-CTA GEMM.  Fixed at creation, per context."""
+        """Bit 0: CUDA-core kernels forced; bit 1: paired-CTA GEMM; bit 2: the scan writes the next VJP's operand
+        (float tanh RNN).  Fixed at creation, per context."""
         return int(lib.hbp_context_modes(self._h))
 
     def close(self):

@@ -642,6 +642,7 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
     if (g.epi == EPI_ADD && !make_map_epi(&tmE, g.E, true, g.M, g.N, g.batch, g.lde, g.e_sb)) return false;
   }
 
+  if (g.dry_run) return true;
   static PerDevice<bool> attr_done;  // the shared-memory opt-in is a per-device attribute of the kernel
   bool& attr_set = attr_done.here();
   if (!attr_set) {

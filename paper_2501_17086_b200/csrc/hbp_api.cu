@@ -26,9 +26,9 @@ struct ProfSeg {
 
 struct hbp_ctx {
   hbp_config cfg;
-  // kernel-selection modes, read from the environment (HBP_FORCE_SIMT=1, HBP_GEMM_PAIR=0) when THIS context is
-  // created and kept with it: another context created later under other settings does not change them
-  bool force_simt = false, gemm_pair = false;
+  // kernel-selection modes, read from the environment (HBP_FORCE_SIMT=1, HBP_GEMM_PAIR=0, HBP_SCAN_OPERAND=0) when
+  // THIS context is created and kept with it: another context created later under other settings does not change them
+  bool force_simt = false, gemm_pair = false, scan_operand = true;
   bool profiling = false;
   std::vector<ProfSeg> segs;       // recorded, not yet read
   std::vector<ProfSeg> free_segs;  // event pairs ready for reuse
@@ -278,6 +278,10 @@ struct Run {
     return a;
   }
   bool u_has_delta = false;  // the VJP GEMM already added delta_l to u_l
+  // float tanh RNN: the scan before an all-step VJP may write that VJP's split operand as a by-product
+  bool want_operand = false;       // set by the iteration loop: another all-step VJP follows the next scan
+  mutable bool operand_ready = false;  // set by the scan when it did
+  int rnn_tc = -1;                     // see rnn_operand_from_scan
   bool shifted = false;      // Highway-BP call on a config with gamma > 0 (exact BP ignores the shift)
   bool stats_ok = true;  // every dY GEMM since the last reset also produced the LayerNorm row sums
   bool run_gemm(const GemmArgs& a) { return gemm(lc, a, c->status); }
@@ -421,7 +425,7 @@ struct Run {
 
   // ---- RNN ---------------------------------------------------------------------------------------
   // u_t = (g_{t+1} * tanh'(z_t)) W for every t at once (one GEMM over T*B rows)
-  void rnn_vjp_all() {
+  GemmArgs rnn_vjp_args() const {
     const int T = c->cfg.L;
     GemmArgs a = base_args();
     a.M = (int)(T * N); a.N = (int)d; a.K = (int)d;
@@ -430,14 +434,31 @@ struct Run {
     a.epi = EPI_STORE; a.D = c->U; a.ldd = d;
     if (c->cfg.loss == HBP_LOSS_EVERY_STEP) {  // u_t + delta_t in the epilogue: one tensor less for the scan
       a.epi = EPI_ADD; a.E = delta; a.lde = d;
-      u_has_delta = true;
     }
     if (c->Ahi) {  // float: g * tanh' split for the tf32 tensor-core product; B(n, k) = W[k][n] = W^T[n][k]
-      split_tf32(lc, (const float*)at(g, state), (const float*)c->C, c->Ahi, c->Alo, (int64_t)T * state);
       a.A_hi = c->Ahi; a.A_lo = c->Alo;
       a.B_hi = c->Whi; a.B_lo = c->Wlo; a.hl_b_sn = d; a.hl_b_sk = 1;
     }
+    return a;
+  }
+  void rnn_vjp_all() {
+    const GemmArgs a = rnn_vjp_args();
+    u_has_delta = a.epi == EPI_ADD;
+    if (c->Ahi && !operand_ready)
+      split_tf32(lc, (const float*)at(g, state), (const float*)c->C, c->Ahi, c->Alo, (int64_t)c->cfg.L * state);
+    operand_ready = false;
     run_gemm(a);
+  }
+  // Whether the scan may write the split operand in place of the iterate: only if the tensor-core GEMM is going to
+  // take the product (the CUDA-core kernel reads g itself).  Asked once per call: the answer depends on the
+  // caller's pointers too.
+  bool rnn_operand_from_scan() {
+    if (rnn_tc < 0) {
+      GemmArgs a = rnn_vjp_args();
+      a.dry_run = true;
+      rnn_tc = c->Ahi && c->scan_operand && !lc.force_simt && gemm_tc(lc, a, c->status) ? 1 : 0;
+    }
+    return rnn_tc == 1;
   }
   void rnn_wgrad(const hbp_grads* gr) {
     const int T = c->cfg.L;
@@ -666,6 +687,11 @@ struct Run {
       if (with_u) s.u2 = c->CB;
     }
     s.g = g;
+    if (want_operand && !shifted && lo == 0 && hi == c->steps) {
+      s.op_coef = (const float*)c->C; s.op_hi = c->Ahi; s.op_lo = c->Alo;
+      s.op_skip_g = true;  // an intermediate iterate: only its product with the coefficients is read
+      s.op_done = &operand_ready;
+    }
     if (with_u && c->preln) {
       s.xhat = c->Y; s.rstd = c->rstd;
       if (c->lnpart && stats_ok) s.lnstat = c->lnstat;
@@ -781,6 +807,8 @@ hbp_status hbp_create(const hbp_config* cfg, void* workspace, size_t workspace_b
   c->force_simt = env && env[0] == '1';
   const char* pm = std::getenv("HBP_GEMM_PAIR");
   c->gemm_pair = !(pm && pm[0] == '0');  // pairs by default
+  const char* so = std::getenv("HBP_SCAN_OPERAND");
+  c->scan_operand = !(so && so[0] == '0');  // the scan writes the next VJP's operand by default (float tanh RNN)
   if (cudaMemset(c->status, 0, 256) != cudaSuccess) {
     delete c;
     return HBP_ERR_CUDA;
@@ -829,7 +857,7 @@ hbp_status hbp_profile_read(hbp_ctx* ctx, float* ms, int64_t* launches) {
 
 int64_t hbp_launch_count(const hbp_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
-int32_t hbp_context_modes(const hbp_ctx* ctx) { return ctx ? (ctx->force_simt ? 1 : 0) | (ctx->gemm_pair ? 2 : 0) : 0; }
+int32_t hbp_context_modes(const hbp_ctx* ctx) { return ctx ? (ctx->force_simt ? 1 : 0) | (ctx->gemm_pair ? 2 : 0) | (ctx->scan_operand ? 4 : 0) : 0; }
 
 hbp_status hbp_sync_status(hbp_ctx* ctx, void* cuda_stream) {
   if (!ctx) return HBP_ERR_INVALID_ARG;
@@ -1036,19 +1064,22 @@ static hbp_status backward_common(hbp_ctx* ctx, const hbp_params* params, int32_
   if (!exact) {
     r.shifted = f.gamma != 0.0f;
     // g^0 = CumSumProd(delta, K) (Eq. 10), then k iterations of {all-step VJP (Eq. 8); reverse scan (Eq. 9, 11)}
+    const int iters = k < steps ? k : steps;
     {
       PhaseScope ph(r, HBP_PHASE_OTHER);  // g^0: a scan without VJPs (a broadcast of delta_L when a = 1)
+      r.want_operand = rnn && iters > 0 && r.rnn_operand_from_scan();
       scan_reverse(r.lc, r.scan_args(0, steps, false));
     }
-    const int iters = k < steps ? k : steps;
     for (int it = 0; it < iters; ++it) {
       {
         PhaseScope ph(r, HBP_PHASE_VJP);
         r.vjp_all();
       }
       PhaseScope ph(r, HBP_PHASE_SCAN);
+      r.want_operand = rnn && it + 1 < iters && r.rnn_operand_from_scan();
       r.scan_with_u(0, steps);
     }
+    r.want_operand = false;
     if (grads) {  // Section 4.2: parameter gradients from the final estimate
       PhaseScope ph(r, HBP_PHASE_WGRAD);
       r.wgrad_all(grads);

@@ -60,6 +60,7 @@ struct GemmArgs {
   // default, and a producer that arms its first pipeline stage without issuing the copies
   uint64_t wait_limit_ns = 0;
   int test_stall = 0;
+  bool dry_run = false;  // gemm_tc only: answer whether it would take this product, launch nothing
 };
 
 // Per-device memo for one-time set-up that CUDA keeps per device (kernel attributes, device properties): a
@@ -137,6 +138,15 @@ struct ScanArgs {
   void* scratch = nullptr;  // time-chunked variant only
   size_t scratch_bytes = 0;
   int* status = nullptr;  // device status word for bounded waits (may be null)
+  // Optional by-product for the float tanh RNN, written only by the TMA-ring kernel (which then sets *op_done):
+  // the next all-step VJP's left operand g_{l+1} * coef_l, already split for the 3 x tf32 product, into rows
+  // l = l_lo-1 .. l_hi-1 (l >= 0) of op_hi / op_lo ([L][rows][d] float, like op_coef).  With op_skip_g the kernel
+  // leaves g alone (an intermediate iterate nobody reads).
+  const float* op_coef = nullptr;
+  float* op_hi = nullptr;
+  float* op_lo = nullptr;
+  bool op_skip_g = false;
+  bool* op_done = nullptr;
 };
 size_t scan_scratch_bytes(int dtype, int L, int64_t rows, int d);
 void scan_reverse(Launcher& lc, const ScanArgs& s);

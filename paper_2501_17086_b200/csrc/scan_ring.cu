@@ -54,24 +54,36 @@ __device__ __forceinline__ void unpack_word<bf16>(uint32_t w, float* f) {
 // NS additive streams (0..2: u and/or a per-step delta), kElemGate: a gate value per element and step.
 // m0, m1: maps of the additive streams, mg: map of the gate; all [steps][rows * d] with boxes of
 // {512 bytes, rows_ps}.  Row y of every map is step y.
-template <typename T, int NS, bool kElemGate>
-__global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(const ScanArgs s,
+// kOp (float only): a further stream mc, the coefficients of the next all-step VJP, read one step lower than the
+// others (step l takes row l - 1), so that beside g_l the kernel can write row l - 1 of that product's left operand
+// g_l * coef_{l-1}, split into its two tf32 terms: the operand never makes a round trip through g.  The serial chain
+// is the critical path here (one warp per scheduler, thousands of dependent steps), so the consumers only leave the
+// float g_l in place of the u_l they took from the ring, and four further warps - again one per scheduler - turn a
+// finished stage into operand rows and give the stage back to the producer.
+template <typename T, int NS, bool kElemGate, bool kOp>
+__global__ void __launch_bounds__((kConsumerWarps * (kOp ? 2 : 1) + 1) * 32) scan_ring_kernel(const ScanArgs s,
                                                                              const __grid_constant__ CUtensorMap m0,
                                                                              const __grid_constant__ CUtensorMap m1,
                                                                              const __grid_constant__ CUtensorMap mg,
+                                                                             const __grid_constant__ CUtensorMap mc,
                                                                              int nstages, int rows_ps) {
   typedef typename RingAcc<T>::type A;
   constexpr int EPT = 4 / (int)sizeof(T);  // channels per lane: one 32-bit word
-  constexpr int STREAMS = NS + (kElemGate ? 1 : 0);
+  static_assert(!kOp || EPT == 1, "the operand by-product is a float path");
+  constexpr int STREAMS = NS + (kElemGate ? 1 : 0) + (kOp ? 1 : 0);
+  constexpr int OP_STREAM = STREAMS - 1;
   const int kRows = rows_ps;                       // steps per ring stage
   const int kStageBytes = rows_ps * kRowBytes;  // per stream
   extern __shared__ __align__(128) unsigned char ring_raw[];
   unsigned char* ring = reinterpret_cast<unsigned char*>(((uintptr_t)ring_raw + 127) & ~(uintptr_t)127);
   uint64_t* bars = reinterpret_cast<uint64_t*>(ring + (size_t)nstages * STREAMS * kStageBytes);
-  int* abort_flag = reinterpret_cast<int*>(bars + 2 * nstages);
+  constexpr int kBarsPerStage = 2 + (kOp ? kConsumerWarps : 0);
+  int* abort_flag = reinterpret_cast<int*>(bars + kBarsPerStage * nstages);
   int* local_status = abort_flag + 1;
   auto full_bar = [&](int i) { return smem_u32(bars + i); };
   auto empty_bar = [&](int i) { return smem_u32(bars + nstages + i); };
+  // kOp: consumer warp w has left its g values in stage i
+  auto done_bar = [&](int i, int w) { return smem_u32(bars + 2 * nstages + i * kConsumerWarps + w); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t state = s.rows * s.d;
@@ -84,6 +96,8 @@ __global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(co
     for (int i = 0; i < nstages; ++i) {
       mbar_init(full_bar(i), 1);
       mbar_init(empty_bar(i), kConsumerWarps);
+      if (kOp)
+        for (int w = 0; w < kConsumerWarps; ++w) mbar_init(done_bar(i, w), 1);
     }
     *abort_flag = 0;
     *local_status = 0;
@@ -105,6 +119,7 @@ __global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(co
         if (NS >= 1) tma_load_2d(dst, &m0, full_bar(slot), x0, y);
         if (NS >= 2) tma_load_2d(dst + kStageBytes, &m1, full_bar(slot), x0, y);
         if (kElemGate) tma_load_2d(dst + NS * kStageBytes, &mg, full_bar(slot), x0, y);
+        if (kOp) tma_load_2d(dst + OP_STREAM * kStageBytes, &mc, full_bar(slot), x0, y - 1);  // rows below 0: zero fill
         issued = k + 1;
       }
       // nothing of this block may still be in flight when it ends (only reachable with work left after an abort)
@@ -117,6 +132,47 @@ __global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(co
             break;
           }
       }
+    }
+    return;
+  }
+
+  if (kOp && warp > kConsumerWarps) {
+    // ---- operand warps: warp w takes the words of consumer warp w; row l - 1 of the operand is g_l * coef_{l-1} ----
+    const int cw = warp - kConsumerWarps - 1;
+    const int word = cw * 32 + lane;
+    const int64_t e0 = (int64_t)x0 + word;
+    const bool live = e0 < state;
+    const int l_min = s.l_lo > 1 ? s.l_lo : 1;
+    auto put = [&](int64_t row, float gl, float coef) {
+      const float v = gl * coef;
+      const float h = round_tf32(v);
+      s.op_hi[row * state + e0] = h;
+      s.op_lo[row * state + e0] = round_tf32(v - h);
+    };
+    if (live && s.l_hi >= 1)  // the top row comes from the carry-in
+      put(s.l_hi - 1, ((const float*)s.g)[(int64_t)s.l_hi * state + e0], s.op_coef[(int64_t)(s.l_hi - 1) * state + e0]);
+    for (int k = 0; k < niter; ++k) {
+      const int slot = k % nstages;
+      if (!mbar_wait(done_bar(slot, cw), (uint32_t)((k / nstages) & 1), abort_flag, status)) break;
+      const unsigned char* stg = ring + (size_t)slot * STREAMS * kStageBytes + word * 4;
+      const int l_base = s.l_hi - (k + 1) * kRows;
+#pragma unroll 1
+      for (int sb = kRows / kSubRows - 1; sb >= 0; --sb) {
+        const unsigned char* sub = stg + sb * kSubRows * kRowBytes;
+        float gg[kSubRows], cc[kSubRows];
+#pragma unroll
+        for (int r = 0; r < kSubRows; ++r) {
+          gg[r] = *reinterpret_cast<const float*>(sub + r * kRowBytes);
+          cc[r] = *reinterpret_cast<const float*>(sub + OP_STREAM * kStageBytes + r * kRowBytes);
+        }
+#pragma unroll
+        for (int r = kSubRows - 1; r >= 0; --r) {
+          const int l = l_base + sb * kSubRows + r;
+          if (live && l >= l_min) put(l - 1, gg[r], cc[r]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_bar(slot));
     }
     return;
   }
@@ -138,6 +194,7 @@ __global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(co
     for (int e = 0; e < EPT; ++e) a0[e] = to_f(((const T*)s.a)[(e0 + e) % s.d]);
   }
   T* gp = g + (int64_t)(s.l_hi - 1) * state + e0;  // where the next step's value goes
+  const bool store_g = !(kOp && s.op_skip_g);
   // kSub rows of one stage, later steps first; `check` = the stage reaches below the first step
   auto sub_block = [&](const unsigned char* stg, int l_top, auto check) {
     constexpr bool kCheck = decltype(check)::value;
@@ -163,11 +220,13 @@ __global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(co
       if (kCheck && l_top - (kSubRows - 1 - r) < s.l_lo) break;
 #pragma unroll
       for (int e = 0; e < EPT; ++e) carry[e] = (A)aa[r][e] * carry[e] + (A)uu[r][e];
-      if (live) {
+      if (live && store_g) {
         if (EPT == 1) *gp = from_f<T>((float)carry[0]);
         else *reinterpret_cast<__nv_bfloat162*>(gp) = __floats2bfloat162_rn((float)carry[0], (float)carry[EPT - 1]);
       }
       gp -= state;
+      // the float the store above holds, left where u_l was for the operand warps
+      if (kOp) *reinterpret_cast<float*>(const_cast<unsigned char*>(stg) + r * kRowBytes) = (float)carry[0];
     }
   };
   for (int k = 0; k < niter; ++k) {
@@ -185,7 +244,7 @@ __global__ void __launch_bounds__((kConsumerWarps + 1) * 32) scan_ring_kernel(co
         sub_block(stg + sb * kSubRows * kRowBytes, l_base + sb * kSubRows + kSubRows - 1, std::true_type());
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(empty_bar(slot));
+    if (lane == 0) mbar_arrive(kOp ? done_bar(slot, warp) : empty_bar(slot));
   }
 }
 
@@ -202,30 +261,41 @@ bool make_map2(CUtensorMap* tm, const void* base, bool f32, int64_t steps, int64
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <typename T, int NS, bool kElemGate>
-void launch_ring(Launcher& lc, const ScanArgs& s, const CUtensorMap& m0, const CUtensorMap& m1, const CUtensorMap& mg,
-                 unsigned grid, int nstages, int rows_ps, size_t smem) {
+struct RingMaps {
+  CUtensorMap m0, m1, mg, mc;
+};
+
+template <typename T, int NS, bool kElemGate, bool kOp>
+void launch_ring(Launcher& lc, const ScanArgs& s, const RingMaps& m, unsigned grid, int nstages, int rows_ps, size_t smem) {
   static PerDevice<size_t> configured_on;  // per-device kernel attribute
   size_t& configured = configured_on.here();
   if (smem > configured) {
-    cudaFuncSetAttribute(scan_ring_kernel<T, NS, kElemGate>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaFuncSetAttribute(scan_ring_kernel<T, NS, kElemGate, kOp>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     configured = smem;
   }
-  scan_ring_kernel<T, NS, kElemGate><<<grid, (kConsumerWarps + 1) * 32, smem, lc.stream>>>(s, m0, m1, mg, nstages, rows_ps);
+  scan_ring_kernel<T, NS, kElemGate, kOp>
+      <<<grid, (kConsumerWarps * (kOp ? 2 : 1) + 1) * 32, smem, lc.stream>>>(s, m.m0, m.m1, m.mg, m.mc, nstages, rows_ps);
   lc.count();
   lc.check();
 }
 
 template <typename T>
-void dispatch_ring(Launcher& lc, const ScanArgs& s, int ns, bool eg, const CUtensorMap& m0, const CUtensorMap& m1,
-                   const CUtensorMap& mg, unsigned grid, int nstages, int rows_ps, size_t smem) {
+void dispatch_ring(Launcher& lc, const ScanArgs& s, int ns, bool eg, bool op, const RingMaps& m, unsigned grid, int nstages,
+                   int rows_ps, size_t smem) {
+  if constexpr (std::is_same<T, float>::value) {
+    if (op) {  // never together with an element gate (see scan_ring)
+      if (ns == 1) launch_ring<T, 1, false, true>(lc, s, m, grid, nstages, rows_ps, smem);
+      else launch_ring<T, 2, false, true>(lc, s, m, grid, nstages, rows_ps, smem);
+      return;
+    }
+  }
   if (eg) {
-    if (ns == 0) launch_ring<T, 0, true>(lc, s, m0, m1, mg, grid, nstages, rows_ps, smem);
-    else if (ns == 1) launch_ring<T, 1, true>(lc, s, m0, m1, mg, grid, nstages, rows_ps, smem);
-    else launch_ring<T, 2, true>(lc, s, m0, m1, mg, grid, nstages, rows_ps, smem);
+    if (ns == 0) launch_ring<T, 0, true, false>(lc, s, m, grid, nstages, rows_ps, smem);
+    else if (ns == 1) launch_ring<T, 1, true, false>(lc, s, m, grid, nstages, rows_ps, smem);
+    else launch_ring<T, 2, true, false>(lc, s, m, grid, nstages, rows_ps, smem);
   } else {
-    if (ns == 1) launch_ring<T, 1, false>(lc, s, m0, m1, mg, grid, nstages, rows_ps, smem);
-    else launch_ring<T, 2, false>(lc, s, m0, m1, mg, grid, nstages, rows_ps, smem);
+    if (ns == 1) launch_ring<T, 1, false, false>(lc, s, m, grid, nstages, rows_ps, smem);
+    else launch_ring<T, 2, false, false>(lc, s, m, grid, nstages, rows_ps, smem);
   }
 }
 
@@ -254,7 +324,9 @@ bool scan_ring(Launcher& lc, const ScanArgs& s) {
   }
   const bool eg = s.a && s.gate == kGateElement;
   if (ns == 0 && !eg) return false;  // nothing to stream: a pure broadcast
-  const int nstreams = ns + (eg ? 1 : 0);
+  // the operand by-product: float, a constant gate, and at least one additive stream to ride along with
+  const bool op = f32 && !eg && ns >= 1 && s.op_coef && s.op_hi && s.op_lo;
+  const int nstreams = ns + (eg ? 1 : 0) + (op ? 1 : 0);
   const int sms = sm_count();
   int per_sm = (int)((grid + sms - 1) / sms);
   if (per_sm > 4) per_sm = 4;
@@ -267,16 +339,19 @@ bool scan_ring(Launcher& lc, const ScanArgs& s) {
   if (nstages > niter) nstages = niter;
   if (nstages > kMaxStages) nstages = kMaxStages;
   if (nstages < 2) return false;
-  CUtensorMap m0, m1, mg;
-  if (ns >= 1 && !make_map2(&m0, streams[0], f32, stream_rows[0], state, rows_ps)) return false;
-  if (ns >= 2 && !make_map2(&m1, streams[1], f32, stream_rows[1], state, rows_ps)) return false;
-  if (eg && !make_map2(&mg, s.a, f32, s.L, state, rows_ps)) return false;
-  if (ns == 0) m0 = mg;  // unused maps still have to be valid objects
-  if (ns < 2) m1 = m0;
-  if (!eg) mg = m0;
-  const size_t smem = (size_t)nstages * nstreams * rows_ps * kRowBytes + (size_t)nstages * 16 + 16 + 128;
-  if (f32) dispatch_ring<float>(lc, s, ns, eg, m0, m1, mg, grid, nstages, rows_ps, smem);
-  else dispatch_ring<bf16>(lc, s, ns, eg, m0, m1, mg, grid, nstages, rows_ps, smem);
+  RingMaps m;
+  if (ns >= 1 && !make_map2(&m.m0, streams[0], f32, stream_rows[0], state, rows_ps)) return false;
+  if (ns >= 2 && !make_map2(&m.m1, streams[1], f32, stream_rows[1], state, rows_ps)) return false;
+  if (eg && !make_map2(&m.mg, s.a, f32, s.L, state, rows_ps)) return false;
+  if (op && !make_map2(&m.mc, s.op_coef, true, s.L, state, rows_ps)) return false;
+  if (ns == 0) m.m0 = m.mg;  // unused maps still have to be valid objects
+  if (ns < 2) m.m1 = m.m0;
+  if (!eg) m.mg = m.m0;
+  if (!op) m.mc = m.m0;
+  const size_t smem = (size_t)nstages * nstreams * rows_ps * kRowBytes + (size_t)nstages * (op ? 16 + 8 * kConsumerWarps : 16) + 16 + 128;
+  if (f32) dispatch_ring<float>(lc, s, ns, eg, op, m, grid, nstages, rows_ps, smem);
+  else dispatch_ring<bf16>(lc, s, ns, eg, false, m, grid, nstages, rows_ps, smem);
+  if (op && s.op_done) *s.op_done = true;
   return true;
 }
 
