@@ -51,22 +51,36 @@ __device__ __forceinline__ void unpack_word<bf16>(uint32_t w, float* f) {
   f[1] = __uint_as_float(w & 0xffff0000u);
 }
 
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tm), "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+
+struct RingMaps {
+  CUtensorMap m0, m1, mg, mc;  // loads: the additive streams, the element gate, the operand's coefficients
+  CUtensorMap og, oh, ol;      // stores: g, and the two terms of the operand
+};
+
 // NS additive streams (0..2: u and/or a per-step delta), kElemGate: a gate value per element and step.
 // m0, m1: maps of the additive streams, mg: map of the gate; all [steps][rows * d] with boxes of
 // {512 bytes, rows_ps}.  Row y of every map is step y.
+//
+// Results leave the way the inputs came: a consumer puts g_l where it took u_l (or the gate, when there is no
+// additive stream) from the ring, and when a stage is done the block's one control lane sends it to global memory as
+// one TMA box, waits until the box has been read, and refills the slot with loads.  The serial chain (one warp per
+// scheduler, thousands of dependent steps) so never issues a global store.  Only a stage that reaches below the
+// first step (or, for the operand, below row 0) is stored by the threads themselves: a TMA store may not start at
+// a negative coordinate, and rows outside [l_lo, l_hi) are not this call's to write.
+//
 // kOp (float only): a further stream mc, the coefficients of the next all-step VJP, read one step lower than the
-// others (step l takes row l - 1), so that beside g_l the kernel can write row l - 1 of that product's left operand
-// g_l * coef_{l-1}, split into its two tf32 terms: the operand never makes a round trip through g.  The serial chain
-// is the critical path here (one warp per scheduler, thousands of dependent steps), so the consumers only leave the
-// float g_l in place of the u_l they took from the ring, and four further warps - again one per scheduler - turn a
-// finished stage into operand rows and give the stage back to the producer.
+// others (step l takes row l - 1), so that the kernel can write row l - 1 of that product's left operand
+// g_l * coef_{l-1}, split into its two tf32 terms: the operand never makes a round trip through g.  Four further
+// warps - again one per scheduler - turn a stage the consumers have finished into operand rows, in place over g_l
+// and the coefficients; g itself is then stored only on request (by the consumers' own stores).
 template <typename T, int NS, bool kElemGate, bool kOp>
 __global__ void __launch_bounds__((kConsumerWarps * (kOp ? 2 : 1) + 1) * 32) scan_ring_kernel(const ScanArgs s,
-                                                                             const __grid_constant__ CUtensorMap m0,
-                                                                             const __grid_constant__ CUtensorMap m1,
-                                                                             const __grid_constant__ CUtensorMap mg,
-                                                                             const __grid_constant__ CUtensorMap mc,
-                                                                             int nstages, int rows_ps) {
+                                                                                            const __grid_constant__ RingMaps m,
+                                                                                            int nstages, int rows_ps) {
   typedef typename RingAcc<T>::type A;
   constexpr int EPT = 4 / (int)sizeof(T);  // channels per lane: one 32-bit word
   static_assert(!kOp || EPT == 1, "the operand by-product is a float path");
@@ -80,10 +94,10 @@ __global__ void __launch_bounds__((kConsumerWarps * (kOp ? 2 : 1) + 1) * 32) sca
   constexpr int kBarsPerStage = 2 + (kOp ? kConsumerWarps : 0);
   int* abort_flag = reinterpret_cast<int*>(bars + kBarsPerStage * nstages);
   int* local_status = abort_flag + 1;
-  auto full_bar = [&](int i) { return smem_u32(bars + i); };
-  auto empty_bar = [&](int i) { return smem_u32(bars + nstages + i); };
+  auto full_bar = [&](int i) { return smem_u32(bars + i); };            // the loads of stage i have landed
+  auto done_bar = [&](int i) { return smem_u32(bars + nstages + i); };  // the results of stage i are in place
   // kOp: consumer warp w has left its g values in stage i
-  auto done_bar = [&](int i, int w) { return smem_u32(bars + 2 * nstages + i * kConsumerWarps + w); };
+  auto chain_bar = [&](int i, int w) { return smem_u32(bars + 2 * nstages + i * kConsumerWarps + w); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t state = s.rows * s.d;
@@ -91,13 +105,16 @@ __global__ void __launch_bounds__((kConsumerWarps * (kOp ? 2 : 1) + 1) * 32) sca
   const int nsteps = s.l_hi - s.l_lo;
   const int niter = (nsteps + kRows - 1) / kRows;
   int* status = s.status ? s.status : local_status;
+  const bool store_g = !(kOp && s.op_skip_g);
+  // the lowest first step of a stage that still goes out as a box (see above)
+  const int l_box = kOp ? (s.l_lo > 1 ? s.l_lo : 1) : s.l_lo;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < nstages; ++i) {
       mbar_init(full_bar(i), 1);
-      mbar_init(empty_bar(i), kConsumerWarps);
+      mbar_init(done_bar(i), kConsumerWarps);
       if (kOp)
-        for (int w = 0; w < kConsumerWarps; ++w) mbar_init(done_bar(i, w), 1);
+        for (int w = 0; w < kConsumerWarps; ++w) mbar_init(chain_bar(i, w), 1);
     }
     *abort_flag = 0;
     *local_status = 0;
@@ -107,24 +124,40 @@ __global__ void __launch_bounds__((kConsumerWarps * (kOp ? 2 : 1) + 1) * 32) sca
   __syncthreads();
 
   if (warp == kConsumerWarps) {
-    // ---- producer: one lane keeps the ring full ----------------------------------------------------
+    // ---- control: one lane keeps the ring full and sends finished stages out ---------------------------------
     if (lane == 0) {
-      int issued = 0;
-      for (int k = 0; k < niter; ++k) {
+      auto load_stage = [&](int k) {
         const int slot = k % nstages;
-        if (k >= nstages && !mbar_wait(empty_bar(slot), (uint32_t)((k / nstages - 1) & 1), abort_flag, status)) break;
         mbar_expect_tx(full_bar(slot), STREAMS * kStageBytes);
         const int y = s.l_hi - (k + 1) * kRows;  // may start below step 0 in the last stage: zero fill
         const uint32_t dst = smem_u32(ring + (size_t)slot * STREAMS * kStageBytes);
-        if (NS >= 1) tma_load_2d(dst, &m0, full_bar(slot), x0, y);
-        if (NS >= 2) tma_load_2d(dst + kStageBytes, &m1, full_bar(slot), x0, y);
-        if (kElemGate) tma_load_2d(dst + NS * kStageBytes, &mg, full_bar(slot), x0, y);
-        if (kOp) tma_load_2d(dst + OP_STREAM * kStageBytes, &mc, full_bar(slot), x0, y - 1);  // rows below 0: zero fill
-        issued = k + 1;
+        if (NS >= 1) tma_load_2d(dst, &m.m0, full_bar(slot), x0, y);
+        if (NS >= 2) tma_load_2d(dst + kStageBytes, &m.m1, full_bar(slot), x0, y);
+        if (kElemGate) tma_load_2d(dst + NS * kStageBytes, &m.mg, full_bar(slot), x0, y);
+        if (kOp) tma_load_2d(dst + OP_STREAM * kStageBytes, &m.mc, full_bar(slot), x0, y - 1);  // rows below 0: zero fill
+      };
+      int issued = 0, taken = 0;
+      for (; issued < niter && issued < nstages; ++issued) load_stage(issued);
+      for (int k = 0; k < niter; ++k) {
+        const int slot = k % nstages;
+        if (!mbar_wait(done_bar(slot), (uint32_t)((k / nstages) & 1), abort_flag, status)) break;
+        taken = k + 1;
+        const int l_base = s.l_hi - (k + 1) * kRows;
+        if (l_base >= l_box) {
+          const uint32_t src = smem_u32(ring + (size_t)slot * STREAMS * kStageBytes);
+          if (kOp) {
+            tma_store_2d(&m.oh, src, x0, l_base - 1);
+            tma_store_2d(&m.ol, src + OP_STREAM * kStageBytes, x0, l_base - 1);
+          } else {
+            tma_store_2d(&m.og, src, x0, l_base);
+          }
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          tma_store_wait_read();  // the slot may be overwritten once the box has been read out of it
+        }
+        if (issued < niter) load_stage(issued++);
       }
-      // nothing of this block may still be in flight when it ends (only reachable with work left after an abort)
-      const int first = issued > nstages ? issued - nstages : 0;
-      for (int k = first; k < issued; ++k) {
+      // nothing of this block may still be in flight when it ends: loads that no one took (only after an abort) ...
+      for (int k = taken; k < issued; ++k) {
         const uint64_t t0 = global_ns();
         while (!mbar_try_wait(full_bar(k % nstages), (uint32_t)((k / nstages) & 1)))
           if (global_ns() - t0 > WAIT_LIMIT_NS) {  // a copy that never landed: say so, then leave
@@ -132,6 +165,7 @@ __global__ void __launch_bounds__((kConsumerWarps * (kOp ? 2 : 1) + 1) * 32) sca
             break;
           }
       }
+      tma_store_wait_all();  // ... and the boxes on their way out
     }
     return;
   }
@@ -142,37 +176,51 @@ __global__ void __launch_bounds__((kConsumerWarps * (kOp ? 2 : 1) + 1) * 32) sca
     const int word = cw * 32 + lane;
     const int64_t e0 = (int64_t)x0 + word;
     const bool live = e0 < state;
-    const int l_min = s.l_lo > 1 ? s.l_lo : 1;
-    auto put = [&](int64_t row, float gl, float coef) {
+    auto split = [](float gl, float coef, float& h, float& l) {
       const float v = gl * coef;
-      const float h = round_tf32(v);
-      s.op_hi[row * state + e0] = h;
-      s.op_lo[row * state + e0] = round_tf32(v - h);
+      h = round_tf32(v);
+      l = round_tf32(v - h);
     };
-    if (live && s.l_hi >= 1)  // the top row comes from the carry-in
-      put(s.l_hi - 1, ((const float*)s.g)[(int64_t)s.l_hi * state + e0], s.op_coef[(int64_t)(s.l_hi - 1) * state + e0]);
+    if (live && s.l_hi >= 1) {  // the top row comes from the carry-in
+      float h, l;
+      split(((const float*)s.g)[(int64_t)s.l_hi * state + e0], s.op_coef[(int64_t)(s.l_hi - 1) * state + e0], h, l);
+      s.op_hi[(int64_t)(s.l_hi - 1) * state + e0] = h;
+      s.op_lo[(int64_t)(s.l_hi - 1) * state + e0] = l;
+    }
     for (int k = 0; k < niter; ++k) {
       const int slot = k % nstages;
-      if (!mbar_wait(done_bar(slot, cw), (uint32_t)((k / nstages) & 1), abort_flag, status)) break;
-      const unsigned char* stg = ring + (size_t)slot * STREAMS * kStageBytes + word * 4;
+      if (!mbar_wait(chain_bar(slot, cw), (uint32_t)((k / nstages) & 1), abort_flag, status)) break;
+      unsigned char* stg = ring + (size_t)slot * STREAMS * kStageBytes + word * 4;
       const int l_base = s.l_hi - (k + 1) * kRows;
+      const bool box = l_base >= l_box;  // else: this stage reaches below the first row, its rows go out one by one
 #pragma unroll 1
       for (int sb = kRows / kSubRows - 1; sb >= 0; --sb) {
-        const unsigned char* sub = stg + sb * kSubRows * kRowBytes;
-        float gg[kSubRows], cc[kSubRows];
+        unsigned char* sub = stg + sb * kSubRows * kRowBytes;
+        float hh[kSubRows], ll[kSubRows];
 #pragma unroll
-        for (int r = 0; r < kSubRows; ++r) {
-          gg[r] = *reinterpret_cast<const float*>(sub + r * kRowBytes);
-          cc[r] = *reinterpret_cast<const float*>(sub + OP_STREAM * kStageBytes + r * kRowBytes);
-        }
+        for (int r = 0; r < kSubRows; ++r)
+          split(*reinterpret_cast<const float*>(sub + r * kRowBytes),
+                *reinterpret_cast<const float*>(sub + OP_STREAM * kStageBytes + r * kRowBytes), hh[r], ll[r]);
+        if (box) {
 #pragma unroll
-        for (int r = kSubRows - 1; r >= 0; --r) {
-          const int l = l_base + sb * kSubRows + r;
-          if (live && l >= l_min) put(l - 1, gg[r], cc[r]);
+          for (int r = 0; r < kSubRows; ++r) {
+            *reinterpret_cast<float*>(sub + r * kRowBytes) = hh[r];
+            *reinterpret_cast<float*>(sub + OP_STREAM * kStageBytes + r * kRowBytes) = ll[r];
+          }
+        } else {
+#pragma unroll
+          for (int r = kSubRows - 1; r >= 0; --r) {
+            const int l = l_base + sb * kSubRows + r;
+            if (live && l >= l_box) {
+              s.op_hi[(int64_t)(l - 1) * state + e0] = hh[r];
+              s.op_lo[(int64_t)(l - 1) * state + e0] = ll[r];
+            }
+          }
         }
       }
+      fence_async_smem();  // the box is read by the async proxy
       __syncwarp();
-      if (lane == 0) mbar_arrive(empty_bar(slot));
+      if (lane == 0) mbar_arrive(done_bar(slot));
     }
     return;
   }
@@ -194,10 +242,10 @@ __global__ void __launch_bounds__((kConsumerWarps * (kOp ? 2 : 1) + 1) * 32) sca
     for (int e = 0; e < EPT; ++e) a0[e] = to_f(((const T*)s.a)[(e0 + e) % s.d]);
   }
   T* gp = g + (int64_t)(s.l_hi - 1) * state + e0;  // where the next step's value goes
-  const bool store_g = !(kOp && s.op_skip_g);
-  // kSub rows of one stage, later steps first; `check` = the stage reaches below the first step
-  auto sub_block = [&](const unsigned char* stg, int l_top, auto check) {
-    constexpr bool kCheck = decltype(check)::value;
+  // kSub rows of one stage, later steps first.  direct = the threads store g themselves (a stage that reaches below
+  // the first step, where they also stop there; or g wanted beside the operand)
+  auto sub_block = [&](unsigned char* stg, int l_top, auto direct_t, auto check_t) {
+    constexpr bool kDirect = decltype(direct_t)::value, kCheck = decltype(check_t)::value;
     float uu[kSubRows][EPT], aa[kSubRows][EPT];
 #pragma unroll
     for (int r = 0; r < kSubRows; ++r) {
@@ -220,31 +268,42 @@ __global__ void __launch_bounds__((kConsumerWarps * (kOp ? 2 : 1) + 1) * 32) sca
       if (kCheck && l_top - (kSubRows - 1 - r) < s.l_lo) break;
 #pragma unroll
       for (int e = 0; e < EPT; ++e) carry[e] = (A)aa[r][e] * carry[e] + (A)uu[r][e];
-      if (live && store_g) {
-        if (EPT == 1) *gp = from_f<T>((float)carry[0]);
-        else *reinterpret_cast<__nv_bfloat162*>(gp) = __floats2bfloat162_rn((float)carry[0], (float)carry[EPT - 1]);
+      uint32_t out;  // g_l as it is stored: one float, or two bf16
+      if (EPT == 1) {
+        out = __float_as_uint((float)carry[0]);
+      } else {
+        const __nv_bfloat162 b2 = __floats2bfloat162_rn((float)carry[0], (float)carry[EPT - 1]);
+        out = *reinterpret_cast<const uint32_t*>(&b2);
       }
+      if (kDirect && live) *reinterpret_cast<uint32_t*>(gp) = out;
       gp -= state;
-      // the float the store above holds, left where u_l was for the operand warps
-      if (kOp) *reinterpret_cast<float*>(const_cast<unsigned char*>(stg) + r * kRowBytes) = (float)carry[0];
+      // left in the first stream's place: for the box that goes out, or for the operand warps
+      if (!kDirect || kOp) *reinterpret_cast<uint32_t*>(stg + r * kRowBytes) = out;
     }
   };
   for (int k = 0; k < niter; ++k) {
     const int slot = k % nstages;
     if (!mbar_wait(full_bar(slot), (uint32_t)((k / nstages) & 1), abort_flag, status)) break;
-    const unsigned char* stg = ring + (size_t)slot * STREAMS * kStageBytes + word * 4;
+    unsigned char* stg = ring + (size_t)slot * STREAMS * kStageBytes + word * 4;
     const int l_base = s.l_hi - (k + 1) * kRows;
-    if (l_base >= s.l_lo) {
+    if (l_base < s.l_lo) {
+#pragma unroll 1
+      for (int sb = kRows / kSubRows - 1; sb >= 0; --sb) {
+        if (store_g) sub_block(stg + sb * kSubRows * kRowBytes, l_base + sb * kSubRows + kSubRows - 1, std::true_type(), std::true_type());
+        else sub_block(stg + sb * kSubRows * kRowBytes, l_base + sb * kSubRows + kSubRows - 1, std::false_type(), std::true_type());
+      }
+    } else if (kOp ? store_g : l_base < l_box) {
 #pragma unroll 1
       for (int sb = kRows / kSubRows - 1; sb >= 0; --sb)
-        sub_block(stg + sb * kSubRows * kRowBytes, l_base + sb * kSubRows + kSubRows - 1, std::false_type());
+        sub_block(stg + sb * kSubRows * kRowBytes, l_base + sb * kSubRows + kSubRows - 1, std::true_type(), std::false_type());
     } else {
 #pragma unroll 1
       for (int sb = kRows / kSubRows - 1; sb >= 0; --sb)
-        sub_block(stg + sb * kSubRows * kRowBytes, l_base + sb * kSubRows + kSubRows - 1, std::true_type());
+        sub_block(stg + sb * kSubRows * kRowBytes, l_base + sb * kSubRows + kSubRows - 1, std::false_type(), std::false_type());
     }
+    if (!kOp) fence_async_smem();  // the box is read by the async proxy
     __syncwarp();
-    if (lane == 0) mbar_arrive(kOp ? done_bar(slot, warp) : empty_bar(slot));
+    if (lane == 0) mbar_arrive(kOp ? chain_bar(slot, warp) : done_bar(slot));
   }
 }
 
@@ -261,10 +320,6 @@ bool make_map2(CUtensorMap* tm, const void* base, bool f32, int64_t steps, int64
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-struct RingMaps {
-  CUtensorMap m0, m1, mg, mc;
-};
-
 template <typename T, int NS, bool kElemGate, bool kOp>
 void launch_ring(Launcher& lc, const ScanArgs& s, const RingMaps& m, unsigned grid, int nstages, int rows_ps, size_t smem) {
   static PerDevice<size_t> configured_on;  // per-device kernel attribute
@@ -274,7 +329,7 @@ void launch_ring(Launcher& lc, const ScanArgs& s, const RingMaps& m, unsigned gr
     configured = smem;
   }
   scan_ring_kernel<T, NS, kElemGate, kOp>
-      <<<grid, (kConsumerWarps * (kOp ? 2 : 1) + 1) * 32, smem, lc.stream>>>(s, m.m0, m.m1, m.mg, m.mc, nstages, rows_ps);
+      <<<grid, (kConsumerWarps * (kOp ? 2 : 1) + 1) * 32, smem, lc.stream>>>(s, m, nstages, rows_ps);
   lc.count();
   lc.check();
 }
@@ -348,6 +403,11 @@ bool scan_ring(Launcher& lc, const ScanArgs& s) {
   if (ns < 2) m.m1 = m.m0;
   if (!eg) m.mg = m.m0;
   if (!op) m.mc = m.m0;
+  // the ways out: g [L + 1 rows], and the operand's two terms [L rows]
+  if (!make_map2(&m.og, s.g, f32, (int64_t)s.L + 1, state, rows_ps)) return false;
+  if (op && (!make_map2(&m.oh, s.op_hi, true, s.L, state, rows_ps) || !make_map2(&m.ol, s.op_lo, true, s.L, state, rows_ps)))
+    return false;
+  if (!op) m.oh = m.ol = m.og;
   const size_t smem = (size_t)nstages * nstreams * rows_ps * kRowBytes + (size_t)nstages * (op ? 16 + 8 * kConsumerWarps : 16) + 16 + 128;
   if (f32) dispatch_ring<float>(lc, s, ns, eg, op, m, grid, nstages, rows_ps, smem);
   else dispatch_ring<bf16>(lc, s, ns, eg, false, m, grid, nstages, rows_ps, smem);
