@@ -74,7 +74,8 @@ __device__ __forceinline__ uint64_t desc_add(uint64_t d, uint32_t bytes) { retur
 
 // Barrier slots (8 bytes each):
 // 0 big tiles loaded, 1-2 full[2], 3-4 empty[2], 5 scores ready, 6 probabilities ready, 7 all MMAs done,
-// 8 scores copied out of tensor memory (the next block's score MMAs may overwrite them).
+// 8 scores copied out of tensor memory (the next block's score MMAs may overwrite them), 9 / 10 full / empty of the
+// dQ kernel's third buffer.
 __device__ __forceinline__ uint32_t bar_at(uint32_t bars, int i) { return bars + 8u * i; }
 
 template <bool kDKV>
@@ -95,7 +96,12 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
   constexpr int VEC_OFF = 2 * BIG_BYTES + 4 * SMALL_BYTES + 2 * PS_BYTES;
   uint64_t* bar_mem = reinterpret_cast<uint64_t*>(aligned + VEC_OFF + 1024);
   const uint32_t bars = smem_u32(bar_mem);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 10);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 12);
+  // The dQ kernel does not stage P, so the place of P^T holds a third buffer of small tiles: its K / V tiles come a
+  // block earlier, which is what its MMA warp was waiting for.  Slots of the buffers' barriers: full 1, 2, 9; empty 3, 4, 10.
+  constexpr int NBUF = kDKV ? 2 : 3;
+  auto full_bar = [&](int buf) { return bar_at(bars, buf < 2 ? 1 + buf : 9); };
+  auto empty_bar = [&](int buf) { return bar_at(bars, buf < 2 ? 3 + buf : 10); };
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -117,6 +123,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
     mbar_init(bar_at(bars, 6), SOFTMAX_WARPS);
     mbar_init(bar_at(bars, 7), 1);
     mbar_init(bar_at(bars, 8), SOFTMAX_WARPS);
+    mbar_init(bar_at(bars, 9), 1);
+    mbar_init(bar_at(bars, 10), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -140,22 +148,22 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
       tma_load_4d(sBig0, &tmBig0, bar_at(bars, 0), 0, big0, h, b);
       tma_load_4d(sBig1, &tmBig1, bar_at(bars, 0), 0, big0, h, b);
       bool ok = true;
-      int last_buf_parity[2] = {-1, -1};
+      int last_buf_parity[3] = {-1, -1, -1};
       for (int it = 0; it < n_it && ok; ++it) {
-        const int buf = it & 1;
-        const uint32_t ph = (uint32_t)(it >> 1) & 1u;
-        if (!mbar_wait(bar_at(bars, 3 + buf), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        const int buf = it % NBUF;
+        const uint32_t ph = (uint32_t)(it / NBUF) & 1u;
+        if (!mbar_wait(empty_bar(buf), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
         const int r0 = (it_beg + it) * SMALL;
-        mbar_expect_tx(bar_at(bars, 1 + buf), 2 * SMALL_BYTES);
+        mbar_expect_tx(full_bar(buf), 2 * SMALL_BYTES);
         last_buf_parity[buf] = (int)ph;
-        tma_load_4d(sSmall + (2 * buf) * SMALL_BYTES, &tmSmall0, bar_at(bars, 1 + buf), 0, r0, h, b);
-        tma_load_4d(sSmall + (2 * buf + 1) * SMALL_BYTES, &tmSmall1, bar_at(bars, 1 + buf), 0, r0, h, b);
+        tma_load_4d(sSmall + (2 * buf) * SMALL_BYTES, &tmSmall0, full_bar(buf), 0, r0, h, b);
+        tma_load_4d(sSmall + (2 * buf + 1) * SMALL_BYTES, &tmSmall1, full_bar(buf), 0, r0, h, b);
       }
       if (!ok) {  // leave no copy of ours in flight
-        for (int buf = 0; buf < 2; ++buf)
+        for (int buf = 0; buf < NBUF; ++buf)
           if (last_buf_parity[buf] >= 0) {
             const uint64_t t0 = global_ns();
-            while (!mbar_try_wait(bar_at(bars, 1 + buf), (uint32_t)last_buf_parity[buf]) &&
+            while (!mbar_try_wait(full_bar(buf), (uint32_t)last_buf_parity[buf]) &&
                    global_ns() - t0 < 100000000ull) {
             }
           }
@@ -175,7 +183,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
     const uint64_t dS0mn = make_desc(sSmall, 8192, 1024), dS1mn = make_desc(sSmall + SMALL_BYTES, 8192, 1024);
     const uint64_t dPt = make_desc(sP, 16, 1024), dDSt = make_desc(sDS, 16, 1024);
     auto issue_scores = [&](int it) {
-      const uint32_t boff = (uint32_t)(it & 1) * (2 * SMALL_BYTES);
+      const uint32_t boff = (uint32_t)(it % NBUF) * (2 * SMALL_BYTES);
       if (leader) {
         // scores and dP: contraction over the head dimension, both operands K-major
 #pragma unroll
@@ -186,15 +194,15 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
       }
     };
     bool ok = mbar_wait(bar_at(bars, 0), 0, abort_flag, p.status);
-    ok = ok && mbar_wait(bar_at(bars, 1), 0, abort_flag, p.status);
+    ok = ok && mbar_wait(full_bar(0), 0, abort_flag, p.status);
     tc_fence_after();
     if (ok) issue_scores(0);
     for (int it = 0; it < n_it && ok; ++it) {
-      const int buf = it & 1;
+      const int buf = it % NBUF;
       const uint32_t itp = (uint32_t)it & 1u;
       if (it + 1 < n_it) {
-        const int nb = (it + 1) & 1;
-        if (!mbar_wait(bar_at(bars, 1 + nb), (uint32_t)((it + 1) >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+        const int nb = (it + 1) % NBUF;
+        if (!mbar_wait(full_bar(nb), (uint32_t)((it + 1) / NBUF) & 1u, abort_flag, p.status)) { ok = false; break; }
         if (!mbar_wait(bar_at(bars, 8), itp, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         issue_scores(it + 1);
@@ -213,7 +221,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
 #pragma unroll
         for (int k = 0; k < SMALL / 16; ++k)  // dK += dS^T Q   /   dQ += dS K
           tc_mma(tAcc0, desc_add(dDSt, 32 * k), desc_add(dS0mn, boff + 2048 * k), IDESC_KMN, acc_on | (k != 0));
-        tc_commit(bar_at(bars, 3 + buf));
+        tc_commit(empty_bar(buf));
       }
     }
     if (leader) tc_commit(bar_at(bars, 7));
@@ -298,7 +306,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmBig0, const __grid_cons
         }
       }
       // the accumulating MMAs of the previous block read the probability tiles: wait until they are done
-      if (it > 0 && !mbar_wait(bar_at(bars, 3 + ((it - 1) & 1)), (uint32_t)((it - 1) >> 1) & 1u, abort_flag, p.status)) {
+      if (it > 0 && !mbar_wait(empty_bar((it - 1) % NBUF), (uint32_t)((it - 1) / NBUF) & 1u, abort_flag, p.status)) {
         ok = false;
         continue;
       }

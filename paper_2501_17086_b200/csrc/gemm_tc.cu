@@ -27,17 +27,16 @@ namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;
 constexpr int A_BYTES = BM * BK * 2;
-// Single CTA: a 128 x 256 tile, stages of {A 128 x 64, B 256 x 64}.  CTA pair (two CTAs of a cluster on one
-// 256 x 256 tile, tcgen05 cta_group::2): each CTA stages its own 128 rows of A and its own 128 of the 256
-// columns of B, so a stage is 32 KB instead of 48 KB for the same flops per SM, and six stages fit.
+// Single CTA: a 128 x 256 tile, stages of {A 128 x 64, B 256 x 64} (B 64 or 128 rows for a product at most that wide).
+// CTA pair (two CTAs of a cluster on one 256 x 256 tile, tcgen05 cta_group::2): each CTA stages its own 128 rows of A
+// and its own 128 of the 256 columns of B, so a stage is 32 KB instead of 48 KB for the same flops per SM, and six
+// stages fit.
 template <bool kPair>
 struct Mode {
-  static constexpr int kStages = kPair ? 6 : 4;
   static constexpr int kBRows = kPair ? 128 : 256;
-  static constexpr int kBBytes = kBRows * BK * 2;
-  static constexpr int kStageBytes = A_BYTES + kBBytes;
   static constexpr int kTileM = kPair ? 256 : 128;
 };
+constexpr int PAIR_STAGES = 6, PAIR_STAGE_BYTES = A_BYTES + 128 * BK * 2;
 constexpr int RING_BYTES = 4 * (A_BYTES + 256 * BK * 2);  // = 6 stages of the pair mode
 constexpr int EPI_WARPS = 8, THREADS = 64 + 32 * EPI_WARPS;
 constexpr uint32_t TMEM_COLS = 512;
@@ -49,6 +48,8 @@ struct TcParams {
   int m_tiles, n_tiles, num_tiles, k_blocks;
   int a_mn, b_mn;  // 1: the operand is MN-major
   int tf32;        // operands are float, multiplied as tf32 (else bf16)
+  int n_mma;       // columns one MMA covers: 256, or 64 / 128 for a narrow single-CTA product (N <= 128), whose B tiles,
+                   // instructions and epilogue then leave the padding columns out
   int segs;        // K segments, each with its own pair of operand maps (3 for the split-float product)
   int splits, kb_per_split;  // split-K: tile z index = split * batch + b; each split covers kb_per_split k-blocks
   int epi, d_f32;
@@ -122,7 +123,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
                const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmD2,
                const __grid_constant__ CUtensorMap tmE, const TcParams p) {
-  constexpr int STAGES = Mode<kPair>::kStages, STAGE_BYTES = Mode<kPair>::kStageBytes;
+  // single CTAs size their stages by the B tile they load (a narrow product: 64 or 128 rows instead of 256), so the
+  // same 192 KB ring is 4, 6 or 8 stages deep: the bytes in flight, not the stage count, hide the load latency
+  constexpr int MAX_STAGES = 8;
+  const int STAGE_BYTES = kPair ? PAIR_STAGE_BYTES : A_BYTES + p.n_mma * 128;
+  const int STAGES = kPair ? PAIR_STAGES : RING_BYTES / STAGE_BYTES;
   constexpr int B_ROWS = Mode<kPair>::kBRows, TILE_M = Mode<kPair>::kTileM;
   // pair mode: rank of this CTA in its pair; the even CTA (leader) owns the pipeline's full barriers and
   // issues the MMAs, its peer's tile loads signal the leader's barriers
@@ -134,18 +139,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   // the swizzled tiles need 1024-byte alignment
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* aligned = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t epi_base = base + STAGES * STAGE_BYTES;  // EPI_WARPS x 4 KB, each 1024-byte aligned
-  uint64_t* bars = reinterpret_cast<uint64_t*>(aligned + STAGES * STAGE_BYTES + EPI_WARPS * EPI_BUF_BYTES);
-  // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty, [2S+4] drain,
-  // [2S+5 .. 2S+5+EPI_WARPS) one per epilogue warp for its staged operand loads
+  const uint32_t epi_base = base + RING_BYTES;  // EPI_WARPS x 4 KB, each 1024-byte aligned
+  uint64_t* bars = reinterpret_cast<uint64_t*>(aligned + RING_BYTES + EPI_WARPS * EPI_BUF_BYTES);
+  // with S = MAX_STAGES: bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty,
+  // [2S+4] drain, [2S+5 .. 2S+5+EPI_WARPS) one per epilogue warp for its staged operand loads
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
-  auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
-  auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
-  const uint32_t drain_bar = bar0 + 8u * (2 * STAGES + 4);
-  auto epi_bar = [&](int w) { return bar0 + 8u * (2 * STAGES + 5 + w); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5 + EPI_WARPS);
+  auto empty_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };
+  auto accf_bar = [&](int a) { return bar0 + 8u * (2 * MAX_STAGES + a); };
+  auto acce_bar = [&](int a) { return bar0 + 8u * (2 * MAX_STAGES + 2 + a); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * MAX_STAGES + 4);
+  auto epi_bar = [&](int w) { return bar0 + 8u * (2 * MAX_STAGES + 5 + w); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_STAGES + 5 + EPI_WARPS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -208,7 +213,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t sA = base + stage * STAGE_BYTES, sB = sA + A_BYTES;
             // pair: all four tile loads of a stage (two per CTA) complete on the leader's barrier
             const uint32_t fb = kPair ? map_to_cta(full_bar(stage), 0) : full_bar(stage);
-            if (leader) mbar_expect_tx(full_bar(stage), kPair ? 2 * STAGE_BYTES : STAGE_BYTES);
+            if (leader) mbar_expect_tx(full_bar(stage), kPair ? 2 * STAGE_BYTES : A_BYTES + p.n_mma * 128);
             issued_mask |= 1u << stage;
             issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
             if (p.stall) { ok = false; break; }  // self-test: bytes are expected that nobody sends
@@ -223,7 +228,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               load(sA, mA, k0, m0);
             }
             if (p.b_mn) {
-              for (int i = 0; i < B_ROWS / row_elems; ++i) load(sB + i * mn_block, mB, n0 + row_elems * i, k0);
+              for (int i = 0; i < (kPair ? B_ROWS : p.n_mma) / row_elems; ++i) load(sB + i * mn_block, mB, n0 + row_elems * i, k0);
             } else {
               load(sB, mB, k0, n0);
             }
@@ -252,14 +257,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const bool issuer = elected != 0;
       const uint32_t fmt = kTf32 ? 2u : 1u;  // operand format: tf32 or bf16
       const uint32_t idesc = (1u << 4) /*fp32 accumulate*/ | (fmt << 7) | (fmt << 10) | ((uint32_t)p.a_mn << 15) |
-                             ((uint32_t)p.b_mn << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+                             ((uint32_t)p.b_mn << 16) | ((uint32_t)((kPair ? BN : p.n_mma) >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
       // one instruction consumes 32 bytes of K: 32 bytes along a K-major row, or 16 rows of an MN-major bf16 block.
       // Descriptors differ between stages and k-steps only in their start address (bits 0..13, in 16-byte units):
       // they are formed once and advanced by adding to the low word.
       const uint32_t a_step16 = (p.a_mn ? 2048u : 32u) >> 4, b_step16 = (p.b_mn ? 2048u : 32u) >> 4;
       const uint64_t adesc0 = make_desc(base, p.a_mn ? mn_block : 16u, 1024u);
       const uint64_t bdesc0 = make_desc(base + A_BYTES, p.b_mn ? mn_block : 16u, 1024u);
-      constexpr uint32_t kStage16 = (uint32_t)STAGE_BYTES >> 4;
+      const uint32_t kStage16 = (uint32_t)STAGE_BYTES >> 4;
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
@@ -337,7 +342,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool staged = p.epi != EPI_RESID;
     const bool has_e = p.epi == EPI_MUL || p.epi == EPI_STORE_LN || p.epi == EPI_ADD;
     const int cw = p.d_f32 ? 32 : 64;      // accumulator columns per staged chunk (128 bytes of output per row)
-    const int nchunks = 128 / cw;
+    // columns of this warp's half that the MMAs write: a narrow product leaves the rest of the tile out
+    const int my_cols = min(128, max(0, (kPair ? BN : p.n_mma) - half * 128));
+    const int nchunks = (my_cols + cw - 1) / cw;
     const uint32_t acce_target[2] = {kPair ? map_to_cta(acce_bar(0), 0) : acce_bar(0),
                                      kPair ? map_to_cta(acce_bar(1), 0) : acce_bar(1)};
     auto release_acc = [&](int a) {
@@ -349,7 +356,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int b = tile / tiles_per_batch, r = tile % tiles_per_batch;
       const int m0 = (r / p.n_tiles) * TILE_M + (int)rank * BM, n0 = (r % p.n_tiles) * BN;  // this CTA's 128 rows
       const int row0 = m0 + quarter * 32, colw = n0 + half * 128;
-      if (has_e && lane == 0) {  // the buffer is free here: fetch the first chunk of E while the MMAs still run
+      if (has_e && lane == 0 && nchunks > 0) {  // the buffer is free here: fetch the first chunk of E while the MMAs still run
         mbar_expect_tx(ebar, EPI_BUF_BYTES);
         tma_load_3d(buf, &tmE, ebar, colw, row0, b);
         e_pending = true;
@@ -357,9 +364,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!mbar_wait(accf_bar(acc), acc_phase, abort_flag, p.status, p.wait_limit_ns)) break;
       tc_fence_after();
       const uint32_t tsrc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN + half * 128);
-      if (!staged) {
+      if (nchunks == 0) {  // nothing of a narrow product in this half: only hand the accumulator back
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) release_acc(acc);
+      } else if (!staged) {
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < (my_cols + 31) / 32; ++c) {
           float v[32];
           tc_ld32(tsrc + c * 32, v);
           residual_chunk(p, b, row0 + lane, colw + c * 32, v);
@@ -607,8 +618,12 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   // CTA pairs wherever there are at least two 128-row blocks (unless the context asks for single CTAs): a stage is
   // 32 KB instead of 48 KB for the same flops per SM, so the ring is six stages deep and draws a third less from L2
   const int sms = sm_count();
-  const bool pair = lc.gemm_pair && sms >= 2 && g.M > BM;
-  const int b_rows = pair ? Mode<true>::kBRows : Mode<false>::kBRows;
+  // A product at most 128 columns wide runs on single CTAs with MMAs of 64 or 128 columns, so that most of the tile is
+  // not padding (64-wide recurrent states).  The LayerNorm row sums keep the full tile: their slots are per 64 columns.
+  const bool narrow = g.N <= 128 && g.epi != EPI_STORE_LN;
+  const bool pair = lc.gemm_pair && sms >= 2 && g.M > BM && !narrow;
+  const int n_mma = !narrow ? BN : (g.N <= 64 ? 64 : 128);
+  const int b_rows = pair ? Mode<true>::kBRows : n_mma;
   CUtensorMap tmA, tmB;
   if (!make_map(&tmA, A0, g.M, g.K, g.batch, a_sm, a_sk, g.a_sb, a_mn, BM, f32)) return false;
   if (!make_map(&tmB, B0, g.N, g.K, g.batch, b_sn, b_sk, g.b_sb, b_mn, b_rows, f32)) return false;
@@ -663,6 +678,7 @@ bool gemm_tc(Launcher& lc, const GemmArgs& g, int* status_word) {
   p.k_blocks = k_blocks;
   p.a_mn = a_mn; p.b_mn = b_mn;
   p.tf32 = f32; p.segs = f32 ? 3 : 1;
+  p.n_mma = n_mma;
   p.splits = splits; p.kb_per_split = kb_per_split;
   p.epi = g.epi; p.d_f32 = out_f32;
   p.D = g.D; p.ldd = g.ldd; p.d_sb = g.d_sb;
