@@ -50,14 +50,14 @@ def config_of(w, k):
 # profiles/.  An entry is used only while the kernel's sources still hash to the value recorded with the capture and
 # the workload has the captured shapes; otherwise the bench line carries "traffic": null.
 TRAFFIC = {
-    # gemm_tc_kernel, VJP pair (dA + dY): c5_small (4 layers x 16384 tokens): 2119.775 + 1055.853 and 2864.423 + 279.595 MB;
-    # c2_small (8 layers x 8192 tokens): 741.016 + 506.177 and 808.292 + 132.456 MB
+    # gemm_tc_kernel, VJP pair (dA + dY): c5_small (4 layers x 16384 tokens): 2050.448 + 1063.307 and 2531.918 + 292.011 MB;
+    # c2_small (8 layers x 8192 tokens): 738.928 + 506.633 and 809.241 + 133.026 MB
     "gemm_vjp": [
-        {"sources": ("gemm_tc.cu", "tc_common.cuh"), "sha256": "1aac9fae53232ef1", "shape": ("preln_mlp", "bf16", 2048, 8192),
-         "bytes_per_token_layer": (2119.775e6 + 1055.853e6 + 2864.423e6 + 279.595e6) / (4 * 16384),
+        {"sources": ("gemm_tc.cu", "tc_common.cuh"), "sha256": "a0699ad7953dac89", "shape": ("preln_mlp", "bf16", 2048, 8192),
+         "bytes_per_token_layer": (2050.448e6 + 1063.307e6 + 2531.918e6 + 292.011e6) / (4 * 16384),
          "profile": "profiles/gemm_tc_kernel_c5_small.md"},
-        {"sources": ("gemm_tc.cu", "tc_common.cuh"), "sha256": "1aac9fae53232ef1", "shape": ("preln_mlp", "bf16", 1024, 4096),
-         "bytes_per_token_layer": (741.016e6 + 506.177e6 + 808.292e6 + 132.456e6) / (8 * 8192),
+        {"sources": ("gemm_tc.cu", "tc_common.cuh"), "sha256": "a0699ad7953dac89", "shape": ("preln_mlp", "bf16", 1024, 4096),
+         "bytes_per_token_layer": (738.928e6 + 506.633e6 + 809.241e6 + 133.026e6) / (8 * 8192),
          "profile": "profiles/gemm_tc_kernel_c2_small.md"}],
     # scan_depth_lnstat_kernel: c5_small 605.158 MB read + 214.451 MB written for 4 steps x 16384 x 2048 elements; c2_small
     # 286.292 + 81.457 MB for 8 x 8192 x 1024 (the writes still in L2 when such a small launch ends are not in the counter)
