@@ -57,6 +57,9 @@ WORKLOADS = {
     "c1": Workload("c1", "mlp", "f32", L=8, d=64, hidden=256, tokens=32, seed=1001, loss="final_half_sse"),
     "c2": Workload("c2", "preln_mlp", "bf16", L=64, d=1024, hidden=4096, batch=16, seq=512, tokens=8192, seed=1002),
     "c3": Workload("c3", "rnn_tanh", "f32", L=4096, d=512, in_dim=256, batch=32, tokens=32, seed=1003, loss="every_mse"),
+    # a 128-wide tanh RNN with many row tiles per SM (196608 rows): the GEMM form for products at most 128 columns
+    # wide and the time scan that writes the next VJP's operand, at a size where their rings wrap many times
+    "r1": Workload("r1", "rnn_tanh", "f32", L=1024, d=128, in_dim=64, batch=192, tokens=192, seed=1010, loss="every_mse"),
     "c4": Workload("c4", "preln_transformer", "bf16", L=24, d=768, hidden=3072, n_heads=12, head_dim=64,
                    seq=1024, batch=16, tokens=16384, seed=1004),
     "c5": Workload("c5", "preln_mlp", "bf16", L=128, d=2048, hidden=8192, batch=32, seq=512, tokens=16384, seed=1005),

@@ -77,11 +77,12 @@ def _rows_of(w, t, rows):
     ("g2", (1, 3, 8), [0, 1, 64, 127]),
     ("l1", (1, 2, 4), [0, 77, 127]),
     ("p2", (1, 2, 4), [0, 1, 127, 128, 4097, 8191]),
+    ("r1", (1, 2, 5), [0, 95, 191]),
 ])
 def test_full_size_sampled_units(name, ks, rows):
     from paper_2501_17086_b200 import harness
     w = WORKLOADS[name]
-    need_gb = {"c2": 30, "c3": 4, "c4": 40, "c5": 150, "g1": 4, "g2": 1, "l1": 6, "p2": 34}[name]
+    need_gb = {"c2": 30, "c3": 4, "c4": 40, "c5": 150, "g1": 4, "g2": 1, "l1": 6, "p2": 34, "r1": 2}[name]
     free, _ = torch.cuda.mem_get_info()
     if free < need_gb * 2**30:
         pytest.skip(f"needs about {need_gb} GB of free device memory")
