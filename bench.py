@@ -40,10 +40,18 @@ def parse():
     return ap.parse_args()
 
 
-def config_of(w, k):
+L2_BYTES = 126e6
+
+
+def config_of(w, k, touched_bytes=None):
+    """touched_bytes: what one step reads and writes at least once (states, gradients, delta, the cached activations
+    and scratch in the workspace); above a few L2 sizes nothing survives in L2 from one step to the next."""
+    if touched_bytes is None or touched_bytes > 2 * L2_BYTES:
+        l2 = "inputs_larger_than_l2 (no flush needed)"
+    else:
+        l2 = f"NOT larger than L2 (a step touches {touched_bytes / 1e6:.0f} MB): a latency case, not a bandwidth figure"
     return {"workload": f"{w.name}: {w.block} L={w.L} d={w.d} hidden={w.hidden} tokens={w.tokens} {w.dtype}",
-            "k": k, "steps_of_scan": w.steps, "with_param_grads": True,
-            "l2": "inputs_larger_than_l2 (no flush needed)", "seed": w.seed}
+            "k": k, "steps_of_scan": w.steps, "with_param_grads": True, "l2": l2, "seed": w.seed}
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per unit of work from the ncu captures summarised under
@@ -295,6 +303,7 @@ def measure(env, wname, k, steps, warmup, headline, detail):
     grads = ctx.new_grads(with_gate=True)
     g_all = ctx.new_states()
 
+    touched = sum(t.numel() * t.element_size() for t in (x_all, g_all, delta, ctx.workspace))
     step = lambda: ctx.backward(params, k, delta, x_all, xin, g_all=g_all, grads=grads)
     for _ in range(max(3, warmup)):
         step()
@@ -415,12 +424,12 @@ def measure(env, wname, k, steps, warmup, headline, detail):
     if headline:
         line = {"metric": METRIC, "value": ms_step, "unit": UNIT, "n_gpus": world, "steps": steps,
                 "warmup": max(3, warmup), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
-                "vs_baseline": None, "dtype": w.dtype, "data": "synthetic", "config": config_of(w, k),
-                "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
+                "vs_baseline": None, "dtype": w.dtype, "data": "synthetic", "config": config_of(w, k, touched),
+                "working_set_gb": touched / 1e9, "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
                 "roofline": roofline, "scan_roofline": scan_roof, "phases_ms_per_step": phases, "tflops": tflops,
                 "replicas_tokens_per_s": world * w.tokens * (w.L if w.block in ("rnn_tanh", "gru", "lstm") else 1) / (ms_step * 1e-3)}
     else:
-        line = {"config": config_of(w, k), "ms_per_step": ms_step, "steps": steps, "gpu_launches": launches,
+        line = {"config": config_of(w, k, touched), "ms_per_step": ms_step, "steps": steps, "gpu_launches": launches,
                 "phases_ms_per_step": phases, "tflops": tflops,
                 "roofline": {x: roofline.get(x) for x in ("kernel", "achieved", "peak", "unit", "frac", "frac_of_burst", "algorithmic_frac")},
                 "scan_roofline": {x: scan_roof.get(x) for x in ("kernel", "achieved", "peak", "unit", "frac", "tensors_counted")}}
