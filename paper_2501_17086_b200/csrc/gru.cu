@@ -11,7 +11,7 @@
 // gates) and stores as C4 = [c_r | c_z | c_nr | c_n] per row.  The input-weight gradient uses
 // [c_r | c_z | c_n] instead of the first three.  Like the tanh RNN, the recurrence itself and exact
 // backpropagation through time are carried in double beside the stored values.
-#include "hbp_internal.h"
+#include "tc_common.cuh"
 
 namespace hbp {
 
@@ -19,11 +19,12 @@ namespace {
 
 constexpr int kTile = 32;
 
-// acc[gate][j] += sum_k src[m_j][k] * Wm[gate * d + n][k] over k in [0, kdim)
+// acc[gate][j] += sum_k src[m_j][k] * Wm[gate * d + n][k] over k in [k_lo, k_hi) (k_lo a multiple of the tile)
 template <typename T, bool kSrcDouble>
 __device__ __forceinline__ void gru_accumulate(const void* __restrict__ src, const T* __restrict__ Wm, int kdim, int B,
                                                int d, int m0, int n0, double (*Hs)[kTile + 1],
-                                               float (*Ws)[kTile][kTile + 1], double acc[3][4]) {
+                                               float (*Ws)[kTile][kTile + 1], double (*acc)[4], int k_lo, int k_hi) {
+  if (k_lo >= k_hi) return;
   const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
   // The next tile's global loads are issued into registers before the current tile is multiplied, so the loop
   // waits for memory once, not once per tile.
@@ -42,8 +43,8 @@ __device__ __forceinline__ void gru_accumulate(const void* __restrict__ src, con
       for (int q = 0; q < 3; ++q) wreg[q][j] = (k < kdim && n < d) ? to_f(Wm[((int64_t)q * d + n) * kdim + k]) : 0.0f;
     }
   };
-  fetch(0);
-  for (int k0 = 0; k0 < kdim; k0 += kTile) {
+  fetch(k_lo);
+  for (int k0 = k_lo; k0 < k_hi; k0 += kTile) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int i = ty + 8 * j;
@@ -52,7 +53,7 @@ __device__ __forceinline__ void gru_accumulate(const void* __restrict__ src, con
       for (int q = 0; q < 3; ++q) Ws[q][i][tx] = wreg[q][j];
     }
     __syncthreads();
-    if (k0 + kTile < kdim) fetch(k0 + kTile);
+    if (k0 + kTile < k_hi) fetch(k0 + kTile);
 #pragma unroll 8
     for (int kk = 0; kk < kTile; ++kk) {
       double w[3];
@@ -71,7 +72,7 @@ __device__ __forceinline__ void gru_accumulate(const void* __restrict__ src, con
 
 __device__ __forceinline__ double sigmoid_d(double v) { return 1.0 / (1.0 + exp(-v)); }
 
-template <typename T>
+template <typename T, bool kCluster>
 __global__ void __launch_bounds__(256) gru_step_kernel(const T* __restrict__ W, const T* __restrict__ U,
                                                        const T* __restrict__ x_t, const double* __restrict__ h_in,
                                                        double* __restrict__ h_out, T* __restrict__ zc,
@@ -79,15 +80,31 @@ __global__ void __launch_bounds__(256) gru_step_kernel(const T* __restrict__ W, 
                                                        int in_dim) {
   __shared__ double Hs[kTile][kTile + 1];
   __shared__ float Ws[3][kTile][kTile + 1];
+  extern __shared__ double red[];  // partial sums of the cluster's other ranks (see cluster_splitk_reduce)
   const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
   const int n0 = blockIdx.x * kTile, m0 = blockIdx.y * kTile;
-  double rec[3][4], pre[3][4];
+  double acc[24];  // [rec | pre][gate][row]
 #pragma unroll
-  for (int q = 0; q < 3; ++q)
+  for (int i = 0; i < 24; ++i) acc[i] = 0.0;
+  double (*rec)[4] = reinterpret_cast<double (*)[4]>(acc);
+  double (*pre)[4] = reinterpret_cast<double (*)[4]>(acc + 12);
+  // the previous state of this thread's outputs, fetched before the products so that the epilogue does not wait for it
+  double hprev[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) rec[q][j] = pre[q][j] = 0.0;
-  gru_accumulate<T, true>(h_in, W, d, B, d, m0, n0, Hs, Ws, rec);
-  gru_accumulate<T, false>(x_t, U, in_dim, B, d, m0, n0, Hs, Ws, pre);
+  for (int j = 0; j < 4; ++j) {
+    const int m = m0 + ty + 8 * j, n = n0 + tx;
+    hprev[j] = (m < B && n < d) ? h_in[(int64_t)m * d + n] : 0.0;
+  }
+  // the CTAs of a cluster share the k-tiles of both products out and add their partial sums
+  // (a kernel that reads the cluster registers is launched as a cluster even alone, which costs microseconds per launch:
+  // the form without a split does not touch them)
+  const int ks = kCluster ? (int)tc::cluster_nctarank() : 1, rank = kCluster ? (int)tc::cluster_ctarank() : 0;
+  const int nt_h = (d + kTile - 1) / kTile, nt_x = (in_dim + kTile - 1) / kTile;
+  gru_accumulate<T, true>(h_in, W, d, B, d, m0, n0, Hs, Ws, rec, (nt_h * rank / ks) * kTile,
+                          min(d, (nt_h * (rank + 1) / ks) * kTile));
+  gru_accumulate<T, false>(x_t, U, in_dim, B, d, m0, n0, Hs, Ws, pre, (nt_x * rank / ks) * kTile,
+                           min(in_dim, (nt_x * (rank + 1) / ks) * kTile));
+  if (kCluster && !tc::cluster_splitk_reduce(acc, red)) return;
   const int n = n0 + tx;
   if (n >= d) return;
 #pragma unroll
@@ -102,7 +119,7 @@ __global__ void __launch_bounds__(256) gru_step_kernel(const T* __restrict__ W, 
     const double e = exp(-2.0 * fabs(an));
     const double nn = copysign((1.0 - e) / (1.0 + e), an);
     const double dn = 4.0 * e / ((1.0 + e) * (1.0 + e));  // 1 - tanh(an)^2
-    const double h = h_in[idx];
+    const double h = hprev[j];
     const double hn = z * h + z1 * nn;
     const double cn = z1 * dn;
     h_out[idx] = hn;
@@ -118,19 +135,25 @@ __global__ void __launch_bounds__(256) gru_step_kernel(const T* __restrict__ W, 
 
 // Exact backpropagation through one GRU step in double:
 //     g_t = delta_t + z_t * g_{t+1} + (g_{t+1} * [c_r | c_z | c_nr]) W.
-template <typename T>
+template <typename T, bool kCluster>
 __global__ void __launch_bounds__(256) gru_bwd_step_kernel(const T* __restrict__ W, const T* __restrict__ zc,
                                                            const T* __restrict__ c4, const T* __restrict__ delta,
                                                            const double* __restrict__ g_in, double* __restrict__ g_out,
                                                            T* __restrict__ g_store, int B, int d) {
   __shared__ double Hs[kTile][kTile + 1];
   __shared__ float Ws[kTile][kTile + 1];
+  __shared__ double red[(tc::kMaxClusterSplit - 1) * 4 * 256];
   const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
   const int n0 = blockIdx.x * kTile, m0 = blockIdx.y * kTile;
   double acc[4] = {0.0, 0.0, 0.0, 0.0};
   // the next tile's operands are fetched into registers before the current tile is multiplied; tiles are numbered
-  // through the three gate blocks
+  // through the three gate blocks.  The CTAs of a cluster share the tiles out (one step has too few output tiles to
+  // fill the GPU) and add their partial sums at the end.
   const int tiles_per_gate = (d + kTile - 1) / kTile, ntiles = 3 * tiles_per_gate;
+  // (a kernel that reads the cluster registers is launched as a cluster even alone, which costs microseconds per launch:
+  // the form without a split does not touch them)
+  const int ks = kCluster ? (int)tc::cluster_nctarank() : 1, rank = kCluster ? (int)tc::cluster_ctarank() : 0;
+  const int t_lo = ntiles * rank / ks, t_hi = ntiles * (rank + 1) / ks;
   double hreg[4];
   float wreg[4];
   auto fetch = [&](int t) {
@@ -144,16 +167,16 @@ __global__ void __launch_bounds__(256) gru_bwd_step_kernel(const T* __restrict__
       wreg[j] = (kk < d && n < d) ? to_f(W[((int64_t)q * d + kk) * d + n]) : 0.0f;
     }
   };
-  fetch(0);
+  if (t_lo < t_hi) fetch(t_lo);
   {
-    for (int t = 0; t < ntiles; ++t) {
+    for (int t = t_lo; t < t_hi; ++t) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         Hs[ty + 8 * j][tx] = hreg[j];
         Ws[tx][ty + 8 * j] = wreg[j];
       }
       __syncthreads();
-      if (t + 1 < ntiles) fetch(t + 1);
+      if (t + 1 < t_hi) fetch(t + 1);
 #pragma unroll
       for (int kk = 0; kk < kTile; ++kk) {
         const double w = (double)Ws[tx][kk];
@@ -163,6 +186,7 @@ __global__ void __launch_bounds__(256) gru_bwd_step_kernel(const T* __restrict__
       __syncthreads();
     }
   }
+  if (kCluster && !tc::cluster_splitk_reduce(acc, red)) return;
   const int n = n0 + tx;
   if (n >= d) return;
 #pragma unroll
@@ -241,12 +265,31 @@ __global__ void __launch_bounds__(256) gru_split_transposed_kernel(const float* 
 void gru_forward_step(Launcher& lc, int dtype, const void* W, const void* U, const void* x_t, const double* h_in,
                       double* h_out, void* zc, void* c4, void* state_out, int B, int d, int in_dim) {
   dim3 grid((d + kTile - 1) / kTile, (B + kTile - 1) / kTile);
-  if (dtype == HBP_F32)
-    gru_step_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)U, (const float*)x_t, h_in, h_out,
-                                                        (float*)zc, (float*)c4, (float*)state_out, B, d, in_dim);
-  else
-    gru_step_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)U, (const bf16*)x_t, h_in, h_out,
-                                                       (bf16*)zc, (bf16*)c4, (bf16*)state_out, B, d, in_dim);
+  // at most two ways: a rank hands 24 partial sums per thread over, 48 KB of the leader's shared memory per peer
+  const int ks = tc::cluster_split_for((int)(grid.x * grid.y), (int)grid.x, tc::sm_count(), 2, 4);
+  const size_t smem = (size_t)(ks - 1) * 24 * 256 * sizeof(double);
+  static PerDevice<bool> attr_done;  // per-device kernel attribute
+  if (ks > 1 && !attr_done.here()) {
+    cudaFuncSetAttribute(gru_step_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 24 * 256 * (int)sizeof(double));
+    cudaFuncSetAttribute(gru_step_kernel<bf16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 24 * 256 * (int)sizeof(double));
+    attr_done.here() = true;
+  }
+  if (ks == 1) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
+    if (dtype == HBP_F32) gru_step_kernel<float, false><<<grid, 256, smem, lc.stream>>>((const float*)W, (const float*)U, (const float*)x_t, h_in, h_out,
+                           (float*)zc, (float*)c4, (float*)state_out, B, d, in_dim);
+    else gru_step_kernel<bf16, false><<<grid, 256, smem, lc.stream>>>((const bf16*)W, (const bf16*)U, (const bf16*)x_t, h_in, h_out,
+                           (bf16*)zc, (bf16*)c4, (bf16*)state_out, B, d, in_dim);
+  } else {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr;
+    tc::cluster_launch_config(cfg, attr, grid, ks, smem, lc.stream);
+    cudaError_t e;
+    if (dtype == HBP_F32) e = cudaLaunchKernelEx(&cfg, gru_step_kernel<float, true>, (const float*)W, (const float*)U, (const float*)x_t, h_in, h_out,
+                           (float*)zc, (float*)c4, (float*)state_out, B, d, in_dim);
+    else e = cudaLaunchKernelEx(&cfg, gru_step_kernel<bf16, true>, (const bf16*)W, (const bf16*)U, (const bf16*)x_t, h_in, h_out,
+                           (bf16*)zc, (bf16*)c4, (bf16*)state_out, B, d, in_dim);
+    if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
+  }
   lc.count();
   lc.check();
 }
@@ -254,12 +297,23 @@ void gru_forward_step(Launcher& lc, int dtype, const void* W, const void* U, con
 void gru_backward_step(Launcher& lc, int dtype, const void* W, const void* zc, const void* c4, const void* delta,
                        const double* g_in, double* g_out, void* g_store, int B, int d) {
   dim3 grid((d + kTile - 1) / kTile, (B + kTile - 1) / kTile);
-  if (dtype == HBP_F32)
-    gru_bwd_step_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)zc, (const float*)c4,
-                                                            (const float*)delta, g_in, g_out, (float*)g_store, B, d);
-  else
-    gru_bwd_step_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)zc, (const bf16*)c4,
-                                                           (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, d);
+  const int ks = tc::cluster_split_for((int)(grid.x * grid.y), 3 * (int)grid.x, tc::sm_count());
+  if (ks == 1) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
+    if (dtype == HBP_F32) gru_bwd_step_kernel<float, false><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)zc, (const float*)c4,
+                           (const float*)delta, g_in, g_out, (float*)g_store, B, d);
+    else gru_bwd_step_kernel<bf16, false><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)zc, (const bf16*)c4,
+                           (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, d);
+  } else {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr;
+    tc::cluster_launch_config(cfg, attr, grid, ks, 0, lc.stream);
+    cudaError_t e;
+    if (dtype == HBP_F32) e = cudaLaunchKernelEx(&cfg, gru_bwd_step_kernel<float, true>, (const float*)W, (const float*)zc, (const float*)c4,
+                           (const float*)delta, g_in, g_out, (float*)g_store, B, d);
+    else e = cudaLaunchKernelEx(&cfg, gru_bwd_step_kernel<bf16, true>, (const bf16*)W, (const bf16*)zc, (const bf16*)c4,
+                           (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, d);
+    if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
+  }
   lc.count();
   lc.check();
 }

@@ -7,7 +7,7 @@
 // computed once, in double, by the forward step and stored as C5 = [c_i | c_f | c_g | c_o | c_h] per row.  The
 // parameter gradients contract the same four-block operand with h and with x_t.  As for the other recurrent cells,
 // the recurrence itself and exact backpropagation through time are carried in double beside the stored values.
-#include "hbp_internal.h"
+#include "tc_common.cuh"
 
 namespace hbp {
 
@@ -15,11 +15,13 @@ namespace {
 
 constexpr int kTile = 32;
 
-// acc[q][j] += sum_k src[m_j][k] * Wm[q * u + n][k] over k in [0, kdim); src rows are src_ld apart
+// acc[q][j] += sum_k src[m_j][k] * Wm[q * u + n][k] over k in [k_lo, k_hi) (k_lo a multiple of the tile); src rows are
+// src_ld apart
 template <typename T, bool kSrcDouble>
 __device__ __forceinline__ void lstm_accumulate(const void* __restrict__ src, int64_t src_ld, const T* __restrict__ Wm,
                                                 int kdim, int B, int u, int m0, int n0, double (*Hs)[kTile + 1],
-                                                float (*Ws)[kTile][kTile + 1], double acc[4][4]) {
+                                                float (*Ws)[kTile][kTile + 1], double (*acc)[4], int k_lo, int k_hi) {
+  if (k_lo >= k_hi) return;
   const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
   // The next tile's global loads are issued into registers before the current tile is multiplied, so the loop
   // waits for memory once, not once per tile.
@@ -38,8 +40,8 @@ __device__ __forceinline__ void lstm_accumulate(const void* __restrict__ src, in
       for (int q = 0; q < 4; ++q) wreg[q][j] = (k < kdim && n < u) ? to_f(Wm[((int64_t)q * u + n) * kdim + k]) : 0.0f;
     }
   };
-  fetch(0);
-  for (int k0 = 0; k0 < kdim; k0 += kTile) {
+  fetch(k_lo);
+  for (int k0 = k_lo; k0 < k_hi; k0 += kTile) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int i = ty + 8 * j;
@@ -48,7 +50,7 @@ __device__ __forceinline__ void lstm_accumulate(const void* __restrict__ src, in
       for (int q = 0; q < 4; ++q) Ws[q][i][tx] = wreg[q][j];
     }
     __syncthreads();
-    if (k0 + kTile < kdim) fetch(k0 + kTile);
+    if (k0 + kTile < k_hi) fetch(k0 + kTile);
 #pragma unroll 8
     for (int kk = 0; kk < kTile; ++kk) {
       double w[4];
@@ -73,7 +75,7 @@ __device__ __forceinline__ void tanh_and_slope(double v, double& t, double& s) {
   s = 4.0 * e / ((1.0 + e) * (1.0 + e));
 }
 
-template <typename T>
+template <typename T, bool kCluster>
 __global__ void __launch_bounds__(256) lstm_step_kernel(const T* __restrict__ W, const T* __restrict__ U,
                                                         const T* __restrict__ x_t, const double* __restrict__ s_in,
                                                         double* __restrict__ s_out, T* __restrict__ fg,
@@ -81,15 +83,30 @@ __global__ void __launch_bounds__(256) lstm_step_kernel(const T* __restrict__ W,
                                                         int in_dim) {
   __shared__ double Hs[kTile][kTile + 1];
   __shared__ float Ws[4][kTile][kTile + 1];
+  extern __shared__ double red[];  // partial sums of the cluster's other ranks (see cluster_splitk_reduce)
   const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
   const int n0 = blockIdx.x * kTile, m0 = blockIdx.y * kTile;
-  double acc[4][4];
+  double flat[16];  // [gate][row]
 #pragma unroll
-  for (int q = 0; q < 4; ++q)
+  for (int i = 0; i < 16; ++i) flat[i] = 0.0;
+  double (*acc)[4] = reinterpret_cast<double (*)[4]>(flat);
+  // the CTAs of a cluster share the k-tiles of both products out and add their partial sums
+  // (a kernel that reads the cluster registers is launched as a cluster even alone, which costs microseconds per launch:
+  // the form without a split does not touch them)
+  const int ks = kCluster ? (int)tc::cluster_nctarank() : 1, rank = kCluster ? (int)tc::cluster_ctarank() : 0;
+  // the previous cell state of this thread's outputs, fetched before the products so that the epilogue does not wait
+  double cprev[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[q][j] = 0.0;
-  lstm_accumulate<T, true>(s_in + u, 2 * u, W, u, B, u, m0, n0, Hs, Ws, acc);   // W h: h is the second half of the state
-  lstm_accumulate<T, false>(x_t, in_dim, U, in_dim, B, u, m0, n0, Hs, Ws, acc);  // + U x_t
+  for (int j = 0; j < 4; ++j) {
+    const int m = m0 + ty + 8 * j, n = n0 + tx;
+    cprev[j] = (m < B && n < u) ? s_in[(int64_t)m * 2 * u + n] : 0.0;
+  }
+  const int nt_h = (u + kTile - 1) / kTile, nt_x = (in_dim + kTile - 1) / kTile;
+  lstm_accumulate<T, true>(s_in + u, 2 * u, W, u, B, u, m0, n0, Hs, Ws, acc, (nt_h * rank / ks) * kTile,
+                           min(u, (nt_h * (rank + 1) / ks) * kTile));   // W h: h is the second half of the state
+  lstm_accumulate<T, false>(x_t, in_dim, U, in_dim, B, u, m0, n0, Hs, Ws, acc, (nt_x * rank / ks) * kTile,
+                            min(in_dim, (nt_x * (rank + 1) / ks) * kTile));  // + U x_t
+  if (kCluster && !tc::cluster_splitk_reduce(flat, red)) return;
   const int n = n0 + tx;
   if (n >= u) return;
 #pragma unroll
@@ -101,7 +118,7 @@ __global__ void __launch_bounds__(256) lstm_step_kernel(const T* __restrict__ W,
     const double o = sigmoid_d(acc[3][j]), o1 = sigmoid_d(-acc[3][j]);
     double g, dg, tc, dtc;
     tanh_and_slope(acc[2][j], g, dg);
-    const double c = s_in[(int64_t)m * 2 * u + n];
+    const double c = cprev[j];
     const double cn = f * c + i * g;
     tanh_and_slope(cn, tc, dtc);
     const double hn = o * tc;
@@ -147,16 +164,24 @@ __device__ __forceinline__ void operand_quad(const T* __restrict__ g_row, const 
 }
 
 // Exact backpropagation through one step in double: g_t = delta_t + [f * g_c, 0] + [u_c, u_h].
-template <typename T>
+template <typename T, bool kCluster>
 __global__ void __launch_bounds__(256) lstm_bwd_step_kernel(const T* __restrict__ W, const T* __restrict__ fg,
                                                             const T* __restrict__ c5, const T* __restrict__ delta,
                                                             const double* __restrict__ g_in, double* __restrict__ g_out,
                                                             T* __restrict__ g_store, int B, int u) {
   __shared__ double Hs[kTile][kTile + 1];
   __shared__ float Ws[kTile][kTile + 1];
+  __shared__ double red[(tc::kMaxClusterSplit - 1) * 4 * 256];
   const int tx = threadIdx.x % kTile, ty = threadIdx.x / kTile;
   const int n0 = blockIdx.x * kTile, m0 = blockIdx.y * kTile;
   double acc[4] = {0.0, 0.0, 0.0, 0.0};
+  // the CTAs of a cluster share the k-tiles out (one step has too few output tiles to fill the GPU) and add their
+  // partial sums at the end
+  const int ntiles = (4 * u + kTile - 1) / kTile;
+  // (a kernel that reads the cluster registers is launched as a cluster even alone, which costs microseconds per launch:
+  // the form without a split does not touch them)
+  const int ks = kCluster ? (int)tc::cluster_nctarank() : 1, rank = kCluster ? (int)tc::cluster_ctarank() : 0;
+  const int k_lo = (ntiles * rank / ks) * kTile, k_hi = min(4 * u, (ntiles * (rank + 1) / ks) * kTile);
   // the next tile's operands are fetched into registers before the current tile is multiplied
   double hreg[4];
   float wreg[4];
@@ -170,15 +195,15 @@ __global__ void __launch_bounds__(256) lstm_bwd_step_kernel(const T* __restrict_
       wreg[j] = (kk < 4 * u && n < u) ? to_f(W[(int64_t)kk * u + n]) : 0.0f;
     }
   };
-  fetch(0);
-  for (int k0 = 0; k0 < 4 * u; k0 += kTile) {  // u is a multiple of 4, not of the tile: blocks may straddle gates
+  if (k_lo < k_hi) fetch(k_lo);
+  for (int k0 = k_lo; k0 < k_hi; k0 += kTile) {  // u is a multiple of 4, not of the tile: blocks may straddle gates
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       Hs[ty + 8 * j][tx] = hreg[j];
       Ws[tx][ty + 8 * j] = wreg[j];
     }
     __syncthreads();
-    if (k0 + kTile < 4 * u) fetch(k0 + kTile);
+    if (k0 + kTile < k_hi) fetch(k0 + kTile);
 #pragma unroll
     for (int kk = 0; kk < kTile; ++kk) {
       const double w = (double)Ws[tx][kk];
@@ -187,6 +212,7 @@ __global__ void __launch_bounds__(256) lstm_bwd_step_kernel(const T* __restrict_
     }
     __syncthreads();
   }
+  if (kCluster && !tc::cluster_splitk_reduce(acc, red)) return;
   const int n = n0 + tx;
   if (n >= u) return;
 #pragma unroll
@@ -284,12 +310,31 @@ __global__ void __launch_bounds__(256) lstm_split_transposed_kernel(const float*
 void lstm_forward_step(Launcher& lc, int dtype, const void* W, const void* U, const void* x_t, const double* s_in,
                        double* s_out, void* fg, void* c5, void* state_out, int B, int u, int in_dim) {
   dim3 grid((u + kTile - 1) / kTile, (B + kTile - 1) / kTile);
-  if (dtype == HBP_F32)
-    lstm_step_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)U, (const float*)x_t, s_in, s_out,
-                                                         (float*)fg, (float*)c5, (float*)state_out, B, u, in_dim);
-  else
-    lstm_step_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)U, (const bf16*)x_t, s_in, s_out,
-                                                        (bf16*)fg, (bf16*)c5, (bf16*)state_out, B, u, in_dim);
+  // at most two ways: a rank hands 16 partial sums per thread over, 32 KB of the leader's shared memory per peer
+  const int ks = tc::cluster_split_for((int)(grid.x * grid.y), (int)grid.x, tc::sm_count(), 2, 4);
+  const size_t smem = (size_t)(ks - 1) * 16 * 256 * sizeof(double);
+  static PerDevice<bool> attr_done;  // per-device kernel attribute
+  if (ks > 1 && !attr_done.here()) {
+    cudaFuncSetAttribute(lstm_step_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 256 * (int)sizeof(double));
+    cudaFuncSetAttribute(lstm_step_kernel<bf16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 256 * (int)sizeof(double));
+    attr_done.here() = true;
+  }
+  if (ks == 1) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
+    if (dtype == HBP_F32) lstm_step_kernel<float, false><<<grid, 256, smem, lc.stream>>>((const float*)W, (const float*)U, (const float*)x_t, s_in, s_out,
+                           (float*)fg, (float*)c5, (float*)state_out, B, u, in_dim);
+    else lstm_step_kernel<bf16, false><<<grid, 256, smem, lc.stream>>>((const bf16*)W, (const bf16*)U, (const bf16*)x_t, s_in, s_out,
+                           (bf16*)fg, (bf16*)c5, (bf16*)state_out, B, u, in_dim);
+  } else {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr;
+    tc::cluster_launch_config(cfg, attr, grid, ks, smem, lc.stream);
+    cudaError_t e;
+    if (dtype == HBP_F32) e = cudaLaunchKernelEx(&cfg, lstm_step_kernel<float, true>, (const float*)W, (const float*)U, (const float*)x_t, s_in, s_out,
+                           (float*)fg, (float*)c5, (float*)state_out, B, u, in_dim);
+    else e = cudaLaunchKernelEx(&cfg, lstm_step_kernel<bf16, true>, (const bf16*)W, (const bf16*)U, (const bf16*)x_t, s_in, s_out,
+                           (bf16*)fg, (bf16*)c5, (bf16*)state_out, B, u, in_dim);
+    if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
+  }
   lc.count();
   lc.check();
 }
@@ -297,12 +342,23 @@ void lstm_forward_step(Launcher& lc, int dtype, const void* W, const void* U, co
 void lstm_backward_step(Launcher& lc, int dtype, const void* W, const void* fg, const void* c5, const void* delta,
                         const double* g_in, double* g_out, void* g_store, int B, int u) {
   dim3 grid((u + kTile - 1) / kTile, (B + kTile - 1) / kTile);
-  if (dtype == HBP_F32)
-    lstm_bwd_step_kernel<float><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)fg, (const float*)c5,
-                                                             (const float*)delta, g_in, g_out, (float*)g_store, B, u);
-  else
-    lstm_bwd_step_kernel<bf16><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)fg, (const bf16*)c5,
-                                                            (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, u);
+  const int ks = tc::cluster_split_for((int)(grid.x * grid.y), (4 * u + kTile - 1) / kTile, tc::sm_count());
+  if (ks == 1) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
+    if (dtype == HBP_F32) lstm_bwd_step_kernel<float, false><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)fg, (const float*)c5,
+                           (const float*)delta, g_in, g_out, (float*)g_store, B, u);
+    else lstm_bwd_step_kernel<bf16, false><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)fg, (const bf16*)c5,
+                           (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, u);
+  } else {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr;
+    tc::cluster_launch_config(cfg, attr, grid, ks, 0, lc.stream);
+    cudaError_t e;
+    if (dtype == HBP_F32) e = cudaLaunchKernelEx(&cfg, lstm_bwd_step_kernel<float, true>, (const float*)W, (const float*)fg, (const float*)c5,
+                           (const float*)delta, g_in, g_out, (float*)g_store, B, u);
+    else e = cudaLaunchKernelEx(&cfg, lstm_bwd_step_kernel<bf16, true>, (const bf16*)W, (const bf16*)fg, (const bf16*)c5,
+                           (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, u);
+    if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
+  }
   lc.count();
   lc.check();
 }
