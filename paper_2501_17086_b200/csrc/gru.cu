@@ -274,12 +274,8 @@ void gru_forward_step(Launcher& lc, int dtype, const void* W, const void* U, con
     cudaFuncSetAttribute(gru_step_kernel<bf16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 24 * 256 * (int)sizeof(double));
     attr_done.here() = true;
   }
-  if (ks == 1) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
-    if (dtype == HBP_F32) gru_step_kernel<float, false><<<grid, 256, smem, lc.stream>>>((const float*)W, (const float*)U, (const float*)x_t, h_in, h_out,
-                           (float*)zc, (float*)c4, (float*)state_out, B, d, in_dim);
-    else gru_step_kernel<bf16, false><<<grid, 256, smem, lc.stream>>>((const bf16*)W, (const bf16*)U, (const bf16*)x_t, h_in, h_out,
-                           (bf16*)zc, (bf16*)c4, (bf16*)state_out, B, d, in_dim);
-  } else {
+  bool launched = false;
+  if (ks > 1) {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr;
     tc::cluster_launch_config(cfg, attr, grid, ks, smem, lc.stream);
@@ -288,7 +284,14 @@ void gru_forward_step(Launcher& lc, int dtype, const void* W, const void* U, con
                            (float*)zc, (float*)c4, (float*)state_out, B, d, in_dim);
     else e = cudaLaunchKernelEx(&cfg, gru_step_kernel<bf16, true>, (const bf16*)W, (const bf16*)U, (const bf16*)x_t, h_in, h_out,
                            (bf16*)zc, (bf16*)c4, (bf16*)state_out, B, d, in_dim);
-    if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
+    launched = e == cudaSuccess;
+    if (!launched) cudaGetLastError();  // clusters of this size cannot be placed here: run unsplit
+  }
+  if (!launched) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
+    if (dtype == HBP_F32) gru_step_kernel<float, false><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)U, (const float*)x_t, h_in, h_out,
+                           (float*)zc, (float*)c4, (float*)state_out, B, d, in_dim);
+    else gru_step_kernel<bf16, false><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)U, (const bf16*)x_t, h_in, h_out,
+                           (bf16*)zc, (bf16*)c4, (bf16*)state_out, B, d, in_dim);
   }
   lc.count();
   lc.check();
@@ -298,12 +301,8 @@ void gru_backward_step(Launcher& lc, int dtype, const void* W, const void* zc, c
                        const double* g_in, double* g_out, void* g_store, int B, int d) {
   dim3 grid((d + kTile - 1) / kTile, (B + kTile - 1) / kTile);
   const int ks = tc::cluster_split_for((int)(grid.x * grid.y), 3 * (int)grid.x, tc::sm_count());
-  if (ks == 1) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
-    if (dtype == HBP_F32) gru_bwd_step_kernel<float, false><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)zc, (const float*)c4,
-                           (const float*)delta, g_in, g_out, (float*)g_store, B, d);
-    else gru_bwd_step_kernel<bf16, false><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)zc, (const bf16*)c4,
-                           (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, d);
-  } else {
+  bool launched = false;
+  if (ks > 1) {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr;
     tc::cluster_launch_config(cfg, attr, grid, ks, 0, lc.stream);
@@ -312,7 +311,14 @@ void gru_backward_step(Launcher& lc, int dtype, const void* W, const void* zc, c
                            (const float*)delta, g_in, g_out, (float*)g_store, B, d);
     else e = cudaLaunchKernelEx(&cfg, gru_bwd_step_kernel<bf16, true>, (const bf16*)W, (const bf16*)zc, (const bf16*)c4,
                            (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, d);
-    if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
+    launched = e == cudaSuccess;
+    if (!launched) cudaGetLastError();  // clusters of this size cannot be placed here: run unsplit
+  }
+  if (!launched) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
+    if (dtype == HBP_F32) gru_bwd_step_kernel<float, false><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)zc, (const float*)c4,
+                           (const float*)delta, g_in, g_out, (float*)g_store, B, d);
+    else gru_bwd_step_kernel<bf16, false><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)zc, (const bf16*)c4,
+                           (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, d);
   }
   lc.count();
   lc.check();

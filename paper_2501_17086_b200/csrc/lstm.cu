@@ -319,12 +319,8 @@ void lstm_forward_step(Launcher& lc, int dtype, const void* W, const void* U, co
     cudaFuncSetAttribute(lstm_step_kernel<bf16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * 256 * (int)sizeof(double));
     attr_done.here() = true;
   }
-  if (ks == 1) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
-    if (dtype == HBP_F32) lstm_step_kernel<float, false><<<grid, 256, smem, lc.stream>>>((const float*)W, (const float*)U, (const float*)x_t, s_in, s_out,
-                           (float*)fg, (float*)c5, (float*)state_out, B, u, in_dim);
-    else lstm_step_kernel<bf16, false><<<grid, 256, smem, lc.stream>>>((const bf16*)W, (const bf16*)U, (const bf16*)x_t, s_in, s_out,
-                           (bf16*)fg, (bf16*)c5, (bf16*)state_out, B, u, in_dim);
-  } else {
+  bool launched = false;
+  if (ks > 1) {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr;
     tc::cluster_launch_config(cfg, attr, grid, ks, smem, lc.stream);
@@ -333,7 +329,14 @@ void lstm_forward_step(Launcher& lc, int dtype, const void* W, const void* U, co
                            (float*)fg, (float*)c5, (float*)state_out, B, u, in_dim);
     else e = cudaLaunchKernelEx(&cfg, lstm_step_kernel<bf16, true>, (const bf16*)W, (const bf16*)U, (const bf16*)x_t, s_in, s_out,
                            (bf16*)fg, (bf16*)c5, (bf16*)state_out, B, u, in_dim);
-    if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
+    launched = e == cudaSuccess;
+    if (!launched) cudaGetLastError();  // clusters of this size cannot be placed here: run unsplit
+  }
+  if (!launched) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
+    if (dtype == HBP_F32) lstm_step_kernel<float, false><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)U, (const float*)x_t, s_in, s_out,
+                           (float*)fg, (float*)c5, (float*)state_out, B, u, in_dim);
+    else lstm_step_kernel<bf16, false><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)U, (const bf16*)x_t, s_in, s_out,
+                           (bf16*)fg, (bf16*)c5, (bf16*)state_out, B, u, in_dim);
   }
   lc.count();
   lc.check();
@@ -343,12 +346,8 @@ void lstm_backward_step(Launcher& lc, int dtype, const void* W, const void* fg, 
                         const double* g_in, double* g_out, void* g_store, int B, int u) {
   dim3 grid((u + kTile - 1) / kTile, (B + kTile - 1) / kTile);
   const int ks = tc::cluster_split_for((int)(grid.x * grid.y), (4 * u + kTile - 1) / kTile, tc::sm_count());
-  if (ks == 1) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
-    if (dtype == HBP_F32) lstm_bwd_step_kernel<float, false><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)fg, (const float*)c5,
-                           (const float*)delta, g_in, g_out, (float*)g_store, B, u);
-    else lstm_bwd_step_kernel<bf16, false><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)fg, (const bf16*)c5,
-                           (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, u);
-  } else {
+  bool launched = false;
+  if (ks > 1) {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr;
     tc::cluster_launch_config(cfg, attr, grid, ks, 0, lc.stream);
@@ -357,7 +356,14 @@ void lstm_backward_step(Launcher& lc, int dtype, const void* W, const void* fg, 
                            (const float*)delta, g_in, g_out, (float*)g_store, B, u);
     else e = cudaLaunchKernelEx(&cfg, lstm_bwd_step_kernel<bf16, true>, (const bf16*)W, (const bf16*)fg, (const bf16*)c5,
                            (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, u);
-    if (e != cudaSuccess && lc.err == cudaSuccess) lc.err = e;
+    launched = e == cudaSuccess;
+    if (!launched) cudaGetLastError();  // clusters of this size cannot be placed here: run unsplit
+  }
+  if (!launched) {  // no cluster: the plain launch path is the cheaper one, and these launches are latency-bound
+    if (dtype == HBP_F32) lstm_bwd_step_kernel<float, false><<<grid, 256, 0, lc.stream>>>((const float*)W, (const float*)fg, (const float*)c5,
+                           (const float*)delta, g_in, g_out, (float*)g_store, B, u);
+    else lstm_bwd_step_kernel<bf16, false><<<grid, 256, 0, lc.stream>>>((const bf16*)W, (const bf16*)fg, (const bf16*)c5,
+                           (const bf16*)delta, g_in, g_out, (bf16*)g_store, B, u);
   }
   lc.count();
   lc.check();
