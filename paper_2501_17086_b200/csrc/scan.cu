@@ -562,9 +562,21 @@ __global__ void __launch_bounds__(256) gate_grad_kernel(const T* __restrict__ g,
   const int64_t per = (rows + gridDim.x - 1) / gridDim.x;
   const int64_t r0 = (int64_t)blockIdx.x * per, r1 = min(rows, r0 + per);
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    float acc = 0.0f;
-    for (int64_t r = r0; r < r1; ++r) acc = fmaf(to_f(g[r * d + c]), to_f(x[r * d + c]), acc);
-    partial[(int64_t)blockIdx.x * d + c] = acc;
+    // four running sums over interleaved rows: eight loads in flight per thread instead of two, fixed order
+    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    int64_t r = r0;
+    for (; r + 4 <= r1; r += 4) {
+      float gv[4], xv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        gv[i] = to_f(g[(r + i) * d + c]);
+        xv[i] = to_f(x[(r + i) * d + c]);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[i] = fmaf(gv[i], xv[i], acc[i]);
+    }
+    for (; r < r1; ++r) acc[0] = fmaf(to_f(g[r * d + c]), to_f(x[r * d + c]), acc[0]);
+    partial[(int64_t)blockIdx.x * d + c] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
   }
 }
 
