@@ -11,7 +11,7 @@
 // gates) and stores as C4 = [c_r | c_z | c_nr | c_n] per row.  The input-weight gradient uses
 // [c_r | c_z | c_n] instead of the first three.  Like the tanh RNN, the recurrence itself and exact
 // backpropagation through time are carried in double beside the stored values.
-#include "tc_common.cuh"
+#include "cluster_split.cuh"
 
 namespace hbp {
 

@@ -7,7 +7,7 @@
 // computed once, in double, by the forward step and stored as C5 = [c_i | c_f | c_g | c_o | c_h] per row.  The
 // parameter gradients contract the same four-block operand with h and with x_t.  As for the other recurrent cells,
 // the recurrence itself and exact backpropagation through time are carried in double beside the stored values.
-#include "tc_common.cuh"
+#include "cluster_split.cuh"
 
 namespace hbp {
 
